@@ -1,0 +1,147 @@
+/*
+ * aser.h -- C ABI of the B200 (sm_100a) library for the forward pass of an
+ * ASER-quantized linear layer (Activation Smoothing + Error Reconstruction,
+ * arXiv 2411.07762):
+ *
+ *     Y = dequant( Q4(W diag(s)) . Q8(diag(s)^-1 X) ) + L_B (L_A X~),   X~ = diag(s)^-1 X
+ *
+ * which is the paper's inference pass "W_q X + L_A L_B X" on the smoothed
+ * activation M^-1 X (Sec. 4.2, last paragraph before Algorithm 1).
+ *
+ * NAMES.  Token-major storage: X [M tokens, K], W [N, K], Y = X W^T [M, N].
+ *   s    [K]   fp32  diagonal of the paper's smoothing matrix M (Sec. 4.2, Eq. 10)
+ *   L_A  [r,K] fp16  DOWN projection  V_r^T S^-1   (the paper calls this one L_B)
+ *   L_B  [N,r] fp16  UP projection    U_r Sigma_r  (the paper calls this one L_A)
+ *   T    [M,r] bf16  T = X~ L_A^T, the intermediate between the two kernels
+ *
+ * CONVENTIONS.  Every function returns 0 (ASER_OK) or a negative ASER_ERR_*;
+ * on error nothing has been launched unless stated.  Every data pointer is a
+ * DEVICE pointer owned by the caller unless its name ends in _host; arrays are
+ * row-major and contiguous; pointers must be 16-byte aligned.  The library
+ * allocates no memory, never synchronises (except aser_check_status), and
+ * enqueues all work on the cudaStream_t passed as `stream` (NULL = the legacy
+ * default stream).  NaN/Inf inputs give unspecified values but never a fault.
+ * Shapes: M >= 0, K % 128 == 0, N % 8 == 0, r % 16 == 0, 0 <= r <= 256.
+ * M == 0 is a no-op that returns ASER_OK.
+ */
+#ifndef ASER_H_
+#define ASER_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ASER_OK                  0
+#define ASER_ERR_NULL           -1  /* a required pointer is NULL */
+#define ASER_ERR_ALIGN          -2  /* a pointer is not 16-byte aligned */
+#define ASER_ERR_SHAPE          -3  /* unsupported M, N, K or r */
+#define ASER_ERR_WORKSPACE      -4  /* workspace NULL or smaller than aser_workspace_bytes() */
+#define ASER_ERR_LAUNCH         -5  /* CUDA reported an error; text in aser_last_error() */
+#define ASER_ERR_DEVICE_TIMEOUT -6  /* a bounded in-kernel wait gave up (see aser_check_status) */
+#define ASER_ERR_DEVICE         -7  /* current device is not compute capability 10.x */
+
+/*
+ * aser_pack_w4 -- offline weight quantization (Sec. 4.2 Eq. 9/11: Q(W_s) of the
+ * smoothed weight W M; Sec. 5.1: per-channel round-to-nearest).
+ *   ws = fp32(W[n,k]) * s[k]            (one fp32 multiply; s == NULL means ones)
+ *   w_scale[n] = max_k |ws| / 7         (fp32 division)
+ *   q = clamp(rne(ws / w_scale[n]), -8, 7)   (fp32 division, half-to-even)
+ * A zero row gets scale 0 and codes 0.
+ * Output Wq [N, K/2] is the CANONICAL packed form: byte j of row n holds
+ * (q[n,2j] & 0xF) | (q[n,2j+1] << 4).  Bit-exact with the definition above.
+ */
+int aser_pack_w4(const void* W_f16, const float* s, int N, int K,
+                 uint8_t* Wq, float* w_scale, void* stream);
+
+/*
+ * aser_repack_w4 / aser_unrepack_w4 -- pure permutation between the canonical
+ * packed form and the layout the tensor-core kernel streams ("Wk").  Wk has
+ * aser_repacked_bytes(N, K) bytes: N is padded to a multiple of 128 with zero
+ * codes; each (128-row, 128-column) block is stored contiguously.  The paper
+ * has no counterpart (it fixes no storage format).  unrepack is the exact
+ * inverse on the first N rows.
+ */
+size_t aser_repacked_bytes(int N, int K);
+int aser_repack_w4(const uint8_t* Wq, int N, int K, void* Wk, void* stream);
+int aser_unrepack_w4(const void* Wk, int N, int K, uint8_t* Wq, void* stream);
+
+/*
+ * aser_quant_act -- fused activation kernel: smoothing (Sec. 4.2, the M^-1 X
+ * factor of Eq. 9), per-token int8 round-to-nearest (Sec. 5.1) and the down
+ * projection of the reconstruction branch (Sec. 4.1, V_r^T S^-1 applied to X~).
+ *   x~ = fp32(X[m,k]) / s[k]                       (fp32 division; s == NULL means ones)
+ *   a_scale[m] = max_k |x~| / 127                  (fp32 division; zero row -> 0, codes 0)
+ *   Xq[m,k] = clamp(rne(x~ / a_scale[m]), -127, 127)
+ *   T[m,j]  = bf16( sum_k L_A[j,k] * x~[m,k] )     (fp32 accumulation; x~ may be rounded to
+ *                                                   fp16 first when tensor cores are used)
+ * Xq and a_scale are bit-exact with the definition.  r == 0: LA_f16 and T_bf16 are ignored.
+ */
+int aser_quant_act(const void* X_f16, const float* s, const void* LA_f16,
+                   int M, int K, int r,
+                   int8_t* Xq, float* a_scale, void* T_bf16, void* stream);
+
+/*
+ * aser_linear_w4a8_lr -- integer GEMM, dequantisation and up projection
+ * (Sec. 4.2: W_q X + L_A L_B X in the paper's letters):
+ *   acc[m,n] = sum_k Xq[m,k] * q[n,k]                               (exact int32)
+ *   Y[m,n]   = fp16( acc * a_scale[m] * w_scale[n] + sum_j L_B[n,j] * T[m,j] )   (fp32)
+ * Wk is the repacked weight (aser_repack_w4).  acc_debug, when not NULL, receives the
+ * int32 accumulators [M,N] (bit-exact); pass NULL in timed runs.  workspace must hold
+ * aser_workspace_bytes(M,N,K,r) bytes, must have been zeroed once with
+ * aser_workspace_init, and may be reused by later calls on the same stream; two calls
+ * that overlap in time need separate workspaces.
+ * aser_linear_w4a8 is the same without the low-rank term (the plain W4A8 control).
+ */
+int aser_linear_w4a8_lr(const int8_t* Xq, const float* a_scale, const void* Wk,
+                        const float* w_scale, const void* T_bf16, const void* LB_f16,
+                        int M, int N, int K, int r, void* Y_f16, int32_t* acc_debug,
+                        void* workspace, size_t workspace_bytes, void* stream);
+int aser_linear_w4a8(const int8_t* Xq, const float* a_scale, const void* Wk,
+                     const float* w_scale, int M, int N, int K, void* Y_f16,
+                     int32_t* acc_debug, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * aser_linear_w4a8_lr_simt -- the same operation on CUDA cores (dp4a) from the
+ * CANONICAL packed weights; slow, used as an on-device cross-check.  r == 0 (with
+ * NULL T/LB) gives the plain product.  Needs no workspace.
+ */
+int aser_linear_w4a8_lr_simt(const int8_t* Xq, const float* a_scale, const uint8_t* Wq,
+                             const float* w_scale, const void* T_bf16, const void* LB_f16,
+                             int M, int N, int K, int r, void* Y_f16, int32_t* acc_debug,
+                             void* stream);
+
+/* Workspace: split-K partial sums, tile counters and a status word. */
+size_t aser_workspace_bytes(int M, int N, int K, int r);
+int aser_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+/*
+ * aser_check_status -- synchronises `stream`, reads the status word and returns
+ * ASER_OK or ASER_ERR_DEVICE_TIMEOUT (a kernel's bounded wait gave up; its output is
+ * invalid).  Clears the word.  Debugging aid, not part of the hot path.
+ */
+int aser_check_status(void* workspace, void* stream);
+
+/*
+ * aser_forward_host -- one whole forward pass from HOST buffers: copies X (fp16 [M,K],
+ * ideally pinned) to the device staging buffer X_dev, runs aser_quant_act and
+ * aser_linear_w4a8_lr (the plain kernel when r == 0), and copies Y back to Y_host,
+ * all enqueued on `stream`; returns without synchronising.  Device-side operands and
+ * staging buffers are the caller's.
+ */
+int aser_forward_host(const void* X_host_f16, void* Y_host_f16,
+                      void* X_dev, int8_t* Xq_dev, float* a_scale_dev, void* T_dev, void* Y_dev,
+                      const float* s, const void* LA_f16, const void* Wk, const float* w_scale,
+                      const void* LB_f16, int M, int N, int K, int r,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
+/* Text of the last CUDA error seen by the calling thread ("" if none). */
+const char* aser_last_error(void);
+/* Library version: major * 1000 + minor. */
+int aser_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ASER_H_ */

@@ -1,0 +1,235 @@
+"""ctypes binding: same names as the C ABI, argument marshalling only."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+lib_path = os.path.join(_HERE, "libaser.so")
+
+EXPORTED_SYMBOLS = (
+    "aser_pack_w4", "aser_repacked_bytes", "aser_repack_w4", "aser_unrepack_w4",
+    "aser_quant_act", "aser_linear_w4a8_lr", "aser_linear_w4a8", "aser_linear_w4a8_lr_simt",
+    "aser_workspace_bytes", "aser_workspace_init", "aser_check_status", "aser_forward_host",
+    "aser_last_error", "aser_version",
+)
+
+if not os.path.exists(lib_path):
+    raise ImportError(
+        f"{lib_path} is missing: build it with `python -m paper_2411_07762_b200.build` "
+        "(there is no fallback path)")
+lib = C.CDLL(lib_path)
+
+_P, _I, _Z = C.c_void_p, C.c_int, C.c_size_t
+lib.aser_pack_w4.argtypes = [_P, _P, _I, _I, _P, _P, _P]
+lib.aser_repacked_bytes.argtypes = [_I, _I]
+lib.aser_repacked_bytes.restype = _Z
+lib.aser_repack_w4.argtypes = [_P, _I, _I, _P, _P]
+lib.aser_unrepack_w4.argtypes = [_P, _I, _I, _P, _P]
+lib.aser_quant_act.argtypes = [_P, _P, _P, _I, _I, _I, _P, _P, _P, _P]
+lib.aser_linear_w4a8_lr.argtypes = [_P, _P, _P, _P, _P, _P, _I, _I, _I, _I, _P, _P, _P, _Z, _P]
+lib.aser_linear_w4a8.argtypes = [_P, _P, _P, _P, _I, _I, _I, _P, _P, _P, _Z, _P]
+lib.aser_linear_w4a8_lr_simt.argtypes = [_P, _P, _P, _P, _P, _P, _I, _I, _I, _I, _P, _P, _P]
+lib.aser_workspace_bytes.argtypes = [_I, _I, _I, _I]
+lib.aser_workspace_bytes.restype = _Z
+lib.aser_workspace_init.argtypes = [_P, _Z, _P]
+lib.aser_check_status.argtypes = [_P, _P]
+lib.aser_forward_host.argtypes = [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P,
+                                  _I, _I, _I, _I, _P, _Z, _P]
+lib.aser_last_error.restype = C.c_char_p
+lib.aser_version.restype = _I
+
+
+class AserError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where} failed with code {code}: {last_error()}")
+
+
+def last_error() -> str:
+    return lib.aser_last_error().decode()
+
+
+def version() -> int:
+    return lib.aser_version()
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _chk(rc: int, where: str):
+    if rc != 0:
+        raise AserError(rc, where)
+
+
+def _dev(t: torch.Tensor, dtype, name: str):
+    if not t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise TypeError(f"{name}: need a contiguous CUDA tensor of {dtype}")
+    return t
+
+
+def pack_w4(W: torch.Tensor, s: torch.Tensor | None):
+    """W fp16 [N,K], s fp32 [K] or None -> (Wq uint8 [N,K/2] canonical, w_scale fp32 [N])."""
+    _dev(W, torch.float16, "W")
+    N, K = W.shape
+    Wq = torch.empty((N, K // 2), dtype=torch.uint8, device=W.device)
+    w_scale = torch.empty((N,), dtype=torch.float32, device=W.device)
+    _chk(lib.aser_pack_w4(_ptr(W), _ptr(s), N, K, _ptr(Wq), _ptr(w_scale), _stream()), "aser_pack_w4")
+    return Wq, w_scale
+
+
+def repacked_bytes(N: int, K: int) -> int:
+    return int(lib.aser_repacked_bytes(N, K))
+
+
+def repack_w4(Wq: torch.Tensor) -> torch.Tensor:
+    _dev(Wq, torch.uint8, "Wq")
+    N, K = Wq.shape[0], Wq.shape[1] * 2
+    Wk = torch.empty((repacked_bytes(N, K),), dtype=torch.uint8, device=Wq.device)
+    _chk(lib.aser_repack_w4(_ptr(Wq), N, K, _ptr(Wk), _stream()), "aser_repack_w4")
+    return Wk
+
+
+def unrepack_w4(Wk: torch.Tensor, N: int, K: int) -> torch.Tensor:
+    _dev(Wk, torch.uint8, "Wk")
+    Wq = torch.empty((N, K // 2), dtype=torch.uint8, device=Wk.device)
+    _chk(lib.aser_unrepack_w4(_ptr(Wk), N, K, _ptr(Wq), _stream()), "aser_unrepack_w4")
+    return Wq
+
+
+def quant_act(X: torch.Tensor, s: torch.Tensor | None, L_A: torch.Tensor | None,
+              out=None):
+    """X fp16 [M,K] -> (Xq int8 [M,K], a_scale fp32 [M], T bf16 [M,r])."""
+    _dev(X, torch.float16, "X")
+    M, K = X.shape
+    r = 0 if L_A is None else L_A.shape[0]
+    if out is None:
+        Xq = torch.empty((M, K), dtype=torch.int8, device=X.device)
+        a_scale = torch.empty((M,), dtype=torch.float32, device=X.device)
+        T = torch.empty((M, r), dtype=torch.bfloat16, device=X.device)
+    else:
+        Xq, a_scale, T = out
+    _chk(lib.aser_quant_act(_ptr(X), _ptr(s), _ptr(L_A) if r else None, M, K, r, _ptr(Xq),
+                            _ptr(a_scale), _ptr(T) if r else None, _stream()), "aser_quant_act")
+    return Xq, a_scale, T
+
+
+def workspace_bytes(M: int, N: int, K: int, r: int) -> int:
+    return int(lib.aser_workspace_bytes(M, N, K, r))
+
+
+def new_workspace(M: int, N: int, K: int, r: int, device="cuda") -> torch.Tensor:
+    """Allocate (with torch) and zero a workspace for the given problem size."""
+    nbytes = max(256, workspace_bytes(M, N, K, r))
+    ws = torch.empty((nbytes,), dtype=torch.uint8, device=device)
+    _chk(lib.aser_workspace_init(_ptr(ws), nbytes, _stream()), "aser_workspace_init")
+    return ws
+
+
+def check_status(ws: torch.Tensor) -> None:
+    _chk(lib.aser_check_status(_ptr(ws), _stream()), "aser_check_status")
+
+
+def linear_w4a8_lr(Xq, a_scale, Wk, w_scale, T, L_B, N: int, ws: torch.Tensor,
+                   Y=None, acc_debug=None):
+    M, K = Xq.shape
+    r = 0 if L_B is None else L_B.shape[1]
+    if Y is None:
+        Y = torch.empty((M, N), dtype=torch.float16, device=Xq.device)
+    _chk(lib.aser_linear_w4a8_lr(_ptr(Xq), _ptr(a_scale), _ptr(Wk), _ptr(w_scale),
+                                 _ptr(T) if r else None, _ptr(L_B) if r else None, M, N, K, r,
+                                 _ptr(Y), _ptr(acc_debug), _ptr(ws), ws.numel(), _stream()),
+         "aser_linear_w4a8_lr")
+    return Y
+
+
+def linear_w4a8(Xq, a_scale, Wk, w_scale, N: int, ws: torch.Tensor, Y=None, acc_debug=None):
+    M, K = Xq.shape
+    if Y is None:
+        Y = torch.empty((M, N), dtype=torch.float16, device=Xq.device)
+    _chk(lib.aser_linear_w4a8(_ptr(Xq), _ptr(a_scale), _ptr(Wk), _ptr(w_scale), M, N, K, _ptr(Y),
+                              _ptr(acc_debug), _ptr(ws), ws.numel(), _stream()), "aser_linear_w4a8")
+    return Y
+
+
+def linear_w4a8_lr_simt(Xq, a_scale, Wq, w_scale, T, L_B, Y=None, acc_debug=None):
+    M, K = Xq.shape
+    N = Wq.shape[0]
+    r = 0 if L_B is None else L_B.shape[1]
+    if Y is None:
+        Y = torch.empty((M, N), dtype=torch.float16, device=Xq.device)
+    _chk(lib.aser_linear_w4a8_lr_simt(_ptr(Xq), _ptr(a_scale), _ptr(Wq), _ptr(w_scale),
+                                      _ptr(T) if r else None, _ptr(L_B) if r else None, M, N, K, r,
+                                      _ptr(Y), _ptr(acc_debug), _stream()),
+         "aser_linear_w4a8_lr_simt")
+    return Y
+
+
+class AserLinear:
+    """Device-resident operands of one ASER-quantized linear layer plus preallocated
+    intermediates for up to `max_tokens` tokens.  __call__ runs aser_quant_act followed by
+    aser_linear_w4a8_lr on the current stream."""
+
+    def __init__(self, W: torch.Tensor, s: torch.Tensor | None, L_A: torch.Tensor | None,
+                 L_B: torch.Tensor | None, max_tokens: int):
+        self.N, self.K = W.shape
+        self.r = 0 if L_A is None else L_A.shape[0]
+        self.s, self.L_A, self.L_B = s, L_A, L_B
+        self.Wq, self.w_scale = pack_w4(W, s)
+        self.Wk = repack_w4(self.Wq)
+        dev = W.device
+        self.max_tokens = max_tokens
+        self.Xq = torch.empty((max_tokens, self.K), dtype=torch.int8, device=dev)
+        self.a_scale = torch.empty((max_tokens,), dtype=torch.float32, device=dev)
+        self.T = torch.empty((max_tokens, max(self.r, 1)), dtype=torch.bfloat16, device=dev)
+        self.Y = torch.empty((max_tokens, self.N), dtype=torch.float16, device=dev)
+        self.X_dev = torch.empty((max_tokens, self.K), dtype=torch.float16, device=dev)
+        self.ws = new_workspace(max_tokens, self.N, self.K, self.r, dev)
+
+    def quant(self, X: torch.Tensor):
+        M = X.shape[0]
+        r = self.r
+        _chk(lib.aser_quant_act(_ptr(X), _ptr(self.s), _ptr(self.L_A) if r else None, M, self.K, r,
+                                _ptr(self.Xq), _ptr(self.a_scale), _ptr(self.T) if r else None,
+                                _stream()), "aser_quant_act")
+
+    def linear(self, M: int, lowrank: bool = True, acc_debug=None):
+        r = self.r if lowrank else 0
+        if r:
+            _chk(lib.aser_linear_w4a8_lr(_ptr(self.Xq), _ptr(self.a_scale), _ptr(self.Wk),
+                                         _ptr(self.w_scale), _ptr(self.T), _ptr(self.L_B), M, self.N,
+                                         self.K, r, _ptr(self.Y), _ptr(acc_debug), _ptr(self.ws),
+                                         self.ws.numel(), _stream()), "aser_linear_w4a8_lr")
+        else:
+            _chk(lib.aser_linear_w4a8(_ptr(self.Xq), _ptr(self.a_scale), _ptr(self.Wk),
+                                      _ptr(self.w_scale), M, self.N, self.K, _ptr(self.Y),
+                                      _ptr(acc_debug), _ptr(self.ws), self.ws.numel(), _stream()),
+                 "aser_linear_w4a8")
+
+    def __call__(self, X: torch.Tensor, lowrank: bool = True) -> torch.Tensor:
+        M = X.shape[0]
+        assert M <= self.max_tokens
+        self.quant(X)
+        self.linear(M, lowrank)
+        return self.Y[:M]
+
+    def forward_host(self, X_host: torch.Tensor, Y_host: torch.Tensor):
+        """Host fp16 X [M,K] (pinned) -> host fp16 Y [M,N] through aser_forward_host."""
+        forward_host(self, X_host, Y_host)
+
+
+def forward_host(layer: AserLinear, X_host: torch.Tensor, Y_host: torch.Tensor):
+    M = X_host.shape[0]
+    r = layer.r
+    _chk(lib.aser_forward_host(_ptr(X_host), _ptr(Y_host), _ptr(layer.X_dev), _ptr(layer.Xq),
+                               _ptr(layer.a_scale), _ptr(layer.T), _ptr(layer.Y), _ptr(layer.s),
+                               _ptr(layer.L_A) if r else None, _ptr(layer.Wk), _ptr(layer.w_scale),
+                               _ptr(layer.L_B) if r else None, M, layer.N, layer.K, r,
+                               _ptr(layer.ws), layer.ws.numel(), _stream()), "aser_forward_host")

@@ -1,0 +1,255 @@
+// extern "C" boundary of the ASER linear library: argument validation and dispatch.
+// No kernel lives here.
+#include <stdio.h>
+#include <string.h>
+
+#include "aser_common.cuh"
+
+namespace aser {
+
+static thread_local char g_last_error[512] = "";
+
+int record_cuda_error(cudaError_t e, const char* where) {
+    snprintf(g_last_error, sizeof(g_last_error), "%s: %s (%s)", where, cudaGetErrorString(e),
+             cudaGetErrorName(e));
+    return ASER_ERR_LAUNCH;
+}
+
+int check_launch(const char* where) {
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return record_cuda_error(e, where);
+    return ASER_OK;
+}
+
+namespace {
+
+int fail(int code, const char* msg) {
+    snprintf(g_last_error, sizeof(g_last_error), "%s", msg);
+    return code;
+}
+
+bool shape_ok(int M, int N, int K, int r) {
+    return M >= 0 && N >= 0 && K > 0 && K % 128 == 0 && K <= 32768 && N % 8 == 0 && r >= 0 &&
+           r <= 256 && r % 16 == 0;
+}
+
+// The kernels are built for sm_100a only; refuse to launch anywhere else.
+int check_device() {
+    static thread_local int cached_dev = -1;
+    static thread_local int cached_rc = ASER_OK;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return record_cuda_error(e, "cudaGetDevice");
+    if (dev == cached_dev) return cached_rc;
+    int major = 0;
+    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) return record_cuda_error(e, "cudaDeviceGetAttribute");
+    cached_dev = dev;
+    cached_rc = (major == 10) ? ASER_OK
+                              : fail(ASER_ERR_DEVICE, "device is not compute capability 10.x");
+    return cached_rc;
+}
+
+#define ASER_REQUIRE_PTR(p)                                                   \
+    do {                                                                      \
+        if ((p) == nullptr) return fail(ASER_ERR_NULL, #p " is NULL");        \
+        if (misaligned16(p)) return fail(ASER_ERR_ALIGN, #p " is not 16-byte aligned"); \
+    } while (0)
+#define ASER_OPTIONAL_PTR(p)                                                  \
+    do {                                                                      \
+        if ((p) != nullptr && misaligned16(p))                                \
+            return fail(ASER_ERR_ALIGN, #p " is not 16-byte aligned");        \
+    } while (0)
+
+int linear_common(const int8_t* Xq, const float* a_scale, const void* Wk, const float* w_scale,
+                  const void* T_bf16, const void* LB_f16, int M, int N, int K, int r, void* Y_f16,
+                  int32_t* acc_debug, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!shape_ok(M, N, K, r)) return fail(ASER_ERR_SHAPE, "unsupported M, N, K or r");
+    if (M == 0 || N == 0) return ASER_OK;
+    ASER_REQUIRE_PTR(Xq);
+    ASER_REQUIRE_PTR(a_scale);
+    ASER_REQUIRE_PTR(Wk);
+    ASER_REQUIRE_PTR(w_scale);
+    ASER_REQUIRE_PTR(Y_f16);
+    ASER_OPTIONAL_PTR(acc_debug);
+    if (r > 0) {
+        ASER_REQUIRE_PTR(T_bf16);
+        ASER_REQUIRE_PTR(LB_f16);
+    }
+    if (workspace == nullptr || misaligned16(workspace) ||
+        workspace_bytes < aser_workspace_bytes(M, N, K, r))
+        return fail(ASER_ERR_WORKSPACE, "workspace missing, misaligned or too small");
+    int rc = check_device();
+    if (rc != ASER_OK) return rc;
+    return launch_linear_tc(Xq, a_scale, static_cast<const uint8_t*>(Wk), w_scale,
+                            static_cast<const __nv_bfloat16*>(T_bf16),
+                            static_cast<const __half*>(LB_f16), M, N, K, r,
+                            static_cast<__half*>(Y_f16), acc_debug, workspace, workspace_bytes,
+                            static_cast<cudaStream_t>(stream));
+}
+
+}  // namespace
+}  // namespace aser
+
+using namespace aser;
+
+extern "C" {
+
+int aser_version(void) { return 1000; }
+
+const char* aser_last_error(void) { return g_last_error; }
+
+int aser_pack_w4(const void* W_f16, const float* s, int N, int K, uint8_t* Wq, float* w_scale,
+                 void* stream) {
+    if (!shape_ok(0, N, K, 0)) return fail(ASER_ERR_SHAPE, "unsupported N or K");
+    if (N == 0) return ASER_OK;
+    ASER_REQUIRE_PTR(W_f16);
+    ASER_OPTIONAL_PTR(s);
+    ASER_REQUIRE_PTR(Wq);
+    ASER_REQUIRE_PTR(w_scale);
+    int rc = check_device();
+    if (rc != ASER_OK) return rc;
+    return launch_pack_w4(static_cast<const __half*>(W_f16), s, N, K, Wq, w_scale,
+                          static_cast<cudaStream_t>(stream));
+}
+
+size_t aser_repacked_bytes(int N, int K) {
+    if (N <= 0 || K <= 0) return 0;
+    size_t nb = ((size_t)N + kWkRows - 1) / kWkRows, kb = ((size_t)K + kWkCols - 1) / kWkCols;
+    return nb * kb * kWkBlockBytes;
+}
+
+int aser_repack_w4(const uint8_t* Wq, int N, int K, void* Wk, void* stream) {
+    if (!shape_ok(0, N, K, 0)) return fail(ASER_ERR_SHAPE, "unsupported N or K");
+    if (N == 0) return ASER_OK;
+    ASER_REQUIRE_PTR(Wq);
+    ASER_REQUIRE_PTR(Wk);
+    int rc = check_device();
+    if (rc != ASER_OK) return rc;
+    return launch_repack_w4(Wq, N, K, static_cast<uint8_t*>(Wk), false,
+                            static_cast<cudaStream_t>(stream));
+}
+
+int aser_unrepack_w4(const void* Wk, int N, int K, uint8_t* Wq, void* stream) {
+    if (!shape_ok(0, N, K, 0)) return fail(ASER_ERR_SHAPE, "unsupported N or K");
+    if (N == 0) return ASER_OK;
+    ASER_REQUIRE_PTR(Wq);
+    ASER_REQUIRE_PTR(Wk);
+    int rc = check_device();
+    if (rc != ASER_OK) return rc;
+    return launch_repack_w4(Wq, N, K, static_cast<uint8_t*>(const_cast<void*>(Wk)), true,
+                            static_cast<cudaStream_t>(stream));
+}
+
+int aser_quant_act(const void* X_f16, const float* s, const void* LA_f16, int M, int K, int r,
+                   int8_t* Xq, float* a_scale, void* T_bf16, void* stream) {
+    if (!shape_ok(M, 0, K, r)) return fail(ASER_ERR_SHAPE, "unsupported M, K or r");
+    if (M == 0) return ASER_OK;
+    ASER_REQUIRE_PTR(X_f16);
+    ASER_OPTIONAL_PTR(s);
+    ASER_REQUIRE_PTR(Xq);
+    ASER_REQUIRE_PTR(a_scale);
+    if (r > 0) {
+        ASER_REQUIRE_PTR(LA_f16);
+        ASER_REQUIRE_PTR(T_bf16);
+    }
+    int rc = check_device();
+    if (rc != ASER_OK) return rc;
+    return launch_quant_act(static_cast<const __half*>(X_f16), s, static_cast<const __half*>(LA_f16),
+                            M, K, r, Xq, a_scale, static_cast<__nv_bfloat16*>(T_bf16),
+                            static_cast<cudaStream_t>(stream));
+}
+
+int aser_linear_w4a8_lr(const int8_t* Xq, const float* a_scale, const void* Wk,
+                        const float* w_scale, const void* T_bf16, const void* LB_f16, int M, int N,
+                        int K, int r, void* Y_f16, int32_t* acc_debug, void* workspace,
+                        size_t workspace_bytes, void* stream) {
+    return linear_common(Xq, a_scale, Wk, w_scale, T_bf16, LB_f16, M, N, K, r, Y_f16, acc_debug,
+                         workspace, workspace_bytes, stream);
+}
+
+int aser_linear_w4a8(const int8_t* Xq, const float* a_scale, const void* Wk, const float* w_scale,
+                     int M, int N, int K, void* Y_f16, int32_t* acc_debug, void* workspace,
+                     size_t workspace_bytes, void* stream) {
+    return linear_common(Xq, a_scale, Wk, w_scale, nullptr, nullptr, M, N, K, 0, Y_f16, acc_debug,
+                         workspace, workspace_bytes, stream);
+}
+
+int aser_linear_w4a8_lr_simt(const int8_t* Xq, const float* a_scale, const uint8_t* Wq,
+                             const float* w_scale, const void* T_bf16, const void* LB_f16, int M,
+                             int N, int K, int r, void* Y_f16, int32_t* acc_debug, void* stream) {
+    if (!shape_ok(M, N, K, r)) return fail(ASER_ERR_SHAPE, "unsupported M, N, K or r");
+    if (M == 0 || N == 0) return ASER_OK;
+    ASER_REQUIRE_PTR(Xq);
+    ASER_REQUIRE_PTR(a_scale);
+    ASER_REQUIRE_PTR(Wq);
+    ASER_REQUIRE_PTR(w_scale);
+    ASER_REQUIRE_PTR(Y_f16);
+    ASER_OPTIONAL_PTR(acc_debug);
+    if (r > 0) {
+        ASER_REQUIRE_PTR(T_bf16);
+        ASER_REQUIRE_PTR(LB_f16);
+    }
+    int rc = check_device();
+    if (rc != ASER_OK) return rc;
+    return launch_linear_simt(Xq, a_scale, Wq, w_scale, static_cast<const __nv_bfloat16*>(T_bf16),
+                              static_cast<const __half*>(LB_f16), M, N, K, r,
+                              static_cast<__half*>(Y_f16), acc_debug,
+                              static_cast<cudaStream_t>(stream));
+}
+
+size_t aser_workspace_bytes(int M, int N, int K, int r) {
+    if (!shape_ok(M, N, K, r)) return 0;
+    return kWsHeaderBytes + linear_tc_workspace_bytes(M, N, K, r);
+}
+
+int aser_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
+    if (workspace == nullptr || misaligned16(workspace) || workspace_bytes < kWsHeaderBytes)
+        return fail(ASER_ERR_WORKSPACE, "workspace missing, misaligned or too small");
+    cudaError_t e = cudaMemsetAsync(workspace, 0, workspace_bytes, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return record_cuda_error(e, "cudaMemsetAsync(workspace)");
+    return ASER_OK;
+}
+
+int aser_check_status(void* workspace, void* stream) {
+    if (workspace == nullptr) return fail(ASER_ERR_WORKSPACE, "workspace is NULL");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint32_t word = 0;
+    cudaError_t e = cudaMemcpyAsync(&word, workspace, sizeof(word), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return record_cuda_error(e, "aser_check_status");
+    if (word == 0) return ASER_OK;
+    e = cudaMemsetAsync(workspace, 0, sizeof(word), st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return record_cuda_error(e, "aser_check_status clear");
+    snprintf(g_last_error, sizeof(g_last_error),
+             "a bounded device-side wait gave up (status word 0x%08x)", word);
+    return ASER_ERR_DEVICE_TIMEOUT;
+}
+
+int aser_forward_host(const void* X_host_f16, void* Y_host_f16, void* X_dev, int8_t* Xq_dev,
+                      float* a_scale_dev, void* T_dev, void* Y_dev, const float* s,
+                      const void* LA_f16, const void* Wk, const float* w_scale, const void* LB_f16,
+                      int M, int N, int K, int r, void* workspace, size_t workspace_bytes,
+                      void* stream) {
+    if (!shape_ok(M, N, K, r)) return fail(ASER_ERR_SHAPE, "unsupported M, N, K or r");
+    if (M == 0 || N == 0) return ASER_OK;
+    if (X_host_f16 == nullptr || Y_host_f16 == nullptr)
+        return fail(ASER_ERR_NULL, "host buffer is NULL");
+    ASER_REQUIRE_PTR(X_dev);
+    ASER_REQUIRE_PTR(Y_dev);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(X_dev, X_host_f16, (size_t)M * K * 2, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return record_cuda_error(e, "copy X to device");
+    int rc = aser_quant_act(X_dev, s, LA_f16, M, K, r, Xq_dev, a_scale_dev, T_dev, stream);
+    if (rc != ASER_OK) return rc;
+    rc = linear_common(Xq_dev, a_scale_dev, Wk, w_scale, r > 0 ? T_dev : nullptr,
+                       r > 0 ? LB_f16 : nullptr, M, N, K, r, Y_dev, nullptr, workspace,
+                       workspace_bytes, stream);
+    if (rc != ASER_OK) return rc;
+    e = cudaMemcpyAsync(Y_host_f16, Y_dev, (size_t)M * N * 2, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return record_cuda_error(e, "copy Y to host");
+    return ASER_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,70 @@
+// Shared host/device helpers of the ASER linear library (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "aser.h"
+
+namespace aser {
+
+// ---- host side -------------------------------------------------------------
+// Records the text of a CUDA error for aser_last_error() and returns ASER_ERR_LAUNCH.
+int record_cuda_error(cudaError_t e, const char* where);
+// cudaGetLastError() after a launch -> ASER_OK or ASER_ERR_LAUNCH.
+int check_launch(const char* where);
+
+inline bool misaligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+// Kernel launchers (one per .cu file); arguments are already validated.
+int launch_pack_w4(const __half* W, const float* s, int N, int K, uint8_t* Wq, float* w_scale,
+                   cudaStream_t st);
+int launch_repack_w4(const uint8_t* Wq, int N, int K, uint8_t* Wk, bool inverse, cudaStream_t st);
+int launch_quant_act(const __half* X, const float* s, const __half* LA, int M, int K, int r,
+                     int8_t* Xq, float* a_scale, __nv_bfloat16* T, cudaStream_t st);
+int launch_linear_simt(const int8_t* Xq, const float* a_scale, const uint8_t* Wq,
+                       const float* w_scale, const __nv_bfloat16* T, const __half* LB,
+                       int M, int N, int K, int r, __half* Y, int32_t* acc_debug, cudaStream_t st);
+int launch_linear_tc(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
+                     const float* w_scale, const __nv_bfloat16* T, const __half* LB,
+                     int M, int N, int K, int r, __half* Y, int32_t* acc_debug,
+                     void* workspace, size_t workspace_bytes, cudaStream_t st);
+size_t linear_tc_workspace_bytes(int M, int N, int K, int r);
+
+// Layout of the repacked weight: [N/128 row blocks][K/128 column blocks][8 KiB].
+// Inside a block: 4 sub-blocks of 32 columns; each holds 128 rows x 16 bytes.
+// The 16 bytes of a row are four 32-bit words; word w covers columns c0 = 32*sub + 8*w .. +7
+// with column c0+i   in nibble 2*i   (i = 0..3)  -> bytes of (word << 4) & 0xF0F0F0F0
+// and  column c0+4+i in nibble 2*i+1 (i = 0..3)  -> bytes of  word       & 0xF0F0F0F0,
+// so two ALU operations turn a word into eight int8 values equal to 16*q, already in
+// column order.
+constexpr int kWkRows = 128;
+constexpr int kWkCols = 128;
+constexpr int kWkBlockBytes = kWkRows * kWkCols / 2;  // 8192
+
+// Workspace header (first 256 bytes): word 0 = status, rest reserved.
+constexpr size_t kWsHeaderBytes = 256;
+
+#ifdef __CUDACC__
+// ---- device side -----------------------------------------------------------
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+// Round-half-to-even to an integer-valued float, then clamp; returns the int.
+__device__ __forceinline__ int rne_clamp(float v, float lo, float hi) {
+    float c = rintf(v);
+    c = fminf(fmaxf(c, lo), hi);
+    return (int)c;
+}
+#endif
+
+}  // namespace aser

@@ -1,0 +1,338 @@
+// Fused activation kernel: smoothing divide (Sec. 4.2, the M^-1 X factor of Eq. 9),
+// per-token int8 round-to-nearest (Sec. 5.1) and the down projection T = X~ L_A^T of the
+// error-reconstruction branch (Sec. 4.1).
+//
+// Two launch shapes:
+//   * few tokens (decode): one CTA per (token, group of L_A rows) so that the L_A stream is
+//     spread over many SMs; CUDA-core FMAs in fp32.
+//   * many tokens (prefill): one CTA per 16 tokens; x~ is rounded to fp16 and multiplied with
+//     L_A on the tensor cores (mma.sync m16n8k16, fp32 accumulation) while the row absmax is
+//     collected; a second sweep over the (L2-resident) rows writes the int8 codes.
+#include "aser_common.cuh"
+
+namespace aser {
+
+namespace {
+
+struct RawChunk {  // 8 activations and their 8 smoothing divisors
+    uint4 x;
+    float4 s0, s1;
+};
+
+__device__ __forceinline__ RawChunk load_raw(const __half* xrow, const float* s, int col, bool ok) {
+    RawChunk rc;
+    rc.x = ok ? *reinterpret_cast<const uint4*>(xrow + col) : make_uint4(0, 0, 0, 0);
+    if (s) {
+        rc.s0 = *reinterpret_cast<const float4*>(s + col);
+        rc.s1 = *reinterpret_cast<const float4*>(s + col + 4);
+    } else {
+        rc.s0 = make_float4(1.f, 1.f, 1.f, 1.f);
+        rc.s1 = rc.s0;
+    }
+    return rc;
+}
+
+// x~ = fp32(x) / s, one IEEE division each.
+__device__ __forceinline__ void smooth8(const RawChunk& rc, float (&v)[8]) {
+    const __half* h = reinterpret_cast<const __half*>(&rc.x);
+    v[0] = __fdiv_rn(__half2float(h[0]), rc.s0.x); v[1] = __fdiv_rn(__half2float(h[1]), rc.s0.y);
+    v[2] = __fdiv_rn(__half2float(h[2]), rc.s0.z); v[3] = __fdiv_rn(__half2float(h[3]), rc.s0.w);
+    v[4] = __fdiv_rn(__half2float(h[4]), rc.s1.x); v[5] = __fdiv_rn(__half2float(h[5]), rc.s1.y);
+    v[6] = __fdiv_rn(__half2float(h[6]), rc.s1.z); v[7] = __fdiv_rn(__half2float(h[7]), rc.s1.w);
+}
+
+// Eight int8 codes rne(x~ / scale) clamped to +-127, packed low column first.
+__device__ __forceinline__ uint2 quant8(const float (&v)[8], float sc, bool nonzero) {
+    uint32_t w[2] = {0, 0};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        int q = 0;
+        if (nonzero) q = rne_clamp(__fdiv_rn(v[i], sc), -127.f, 127.f);
+        w[i >> 2] |= (uint32_t)(q & 0xFF) << (8 * (i & 3));
+    }
+    return make_uint2(w[0], w[1]);
+}
+
+// ---------------------------------------------------------------------------
+// few tokens
+// ---------------------------------------------------------------------------
+constexpr int kSmallThreads = 256;
+constexpr int kRowsPerCta = 4;  // L_A rows handled by one projection CTA
+
+// grid = (1 + ceil(r / kRowsPerCta), M).  blockIdx.x == 0 quantizes token blockIdx.y,
+// the others compute kRowsPerCta entries of T for that token.
+// dynamic smem: K floats (the smoothed row).
+__global__ void __launch_bounds__(kSmallThreads)
+quant_act_small_kernel(const __half* __restrict__ X, const float* __restrict__ s,
+                       const __half* __restrict__ LA, int M, int K, int r,
+                       int8_t* __restrict__ Xq, float* __restrict__ a_scale,
+                       __nv_bfloat16* __restrict__ T) {
+    extern __shared__ __align__(16) float xs[];
+    __shared__ float red[kRowsPerCta][kSmallThreads / 32];
+    const int m = blockIdx.y;
+    const int chunks = K / 8;
+    const __half* row = X + (size_t)m * K;
+
+    float amax = 0.f;
+    for (int c = threadIdx.x; c < chunks; c += kSmallThreads) {
+        RawChunk rc = load_raw(row, s, c * 8, true);
+        float v[8];
+        smooth8(rc, v);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(v[i]));
+        *reinterpret_cast<float4*>(xs + c * 8) = make_float4(v[0], v[1], v[2], v[3]);
+        *reinterpret_cast<float4*>(xs + c * 8 + 4) = make_float4(v[4], v[5], v[6], v[7]);
+    }
+
+    if (blockIdx.x == 0) {
+        // ---- quantize this token ----
+        amax = warp_max(amax);
+        if ((threadIdx.x & 31) == 0) red[0][threadIdx.x >> 5] = amax;
+        __syncthreads();
+        amax = red[0][0];
+#pragma unroll
+        for (int i = 1; i < kSmallThreads / 32; ++i) amax = fmaxf(amax, red[0][i]);
+        const float sc = __fdiv_rn(amax, 127.0f);
+        if (threadIdx.x == 0) a_scale[m] = sc;
+        int8_t* out = Xq + (size_t)m * K;
+        for (int c = threadIdx.x; c < chunks; c += kSmallThreads) {
+            float v[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v[i] = xs[c * 8 + i];
+            *reinterpret_cast<uint2*>(out + c * 8) = quant8(v, sc, amax > 0.f);
+        }
+        return;
+    }
+
+    // ---- down projection: kRowsPerCta rows of L_A against the smoothed token ----
+    __syncthreads();
+    const int j0 = (blockIdx.x - 1) * kRowsPerCta;
+    float acc[kRowsPerCta];
+#pragma unroll
+    for (int jj = 0; jj < kRowsPerCta; ++jj) acc[jj] = 0.f;
+    for (int c = threadIdx.x; c < chunks; c += kSmallThreads) {
+        float4 x0 = *reinterpret_cast<const float4*>(xs + c * 8);
+        float4 x1 = *reinterpret_cast<const float4*>(xs + c * 8 + 4);
+#pragma unroll
+        for (int jj = 0; jj < kRowsPerCta; ++jj) {
+            if (j0 + jj < r) {
+                uint4 raw = *reinterpret_cast<const uint4*>(LA + (size_t)(j0 + jj) * K + c * 8);
+                const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
+                float2 a = __half22float2(h2[0]), b = __half22float2(h2[1]);
+                float2 cc = __half22float2(h2[2]), d = __half22float2(h2[3]);
+                float t = acc[jj];
+                t = fmaf(a.x, x0.x, t); t = fmaf(a.y, x0.y, t);
+                t = fmaf(b.x, x0.z, t); t = fmaf(b.y, x0.w, t);
+                t = fmaf(cc.x, x1.x, t); t = fmaf(cc.y, x1.y, t);
+                t = fmaf(d.x, x1.z, t); t = fmaf(d.y, x1.w, t);
+                acc[jj] = t;
+            }
+        }
+    }
+#pragma unroll
+    for (int jj = 0; jj < kRowsPerCta; ++jj) {
+        float t = warp_sum(acc[jj]);
+        if ((threadIdx.x & 31) == 0) red[jj][threadIdx.x >> 5] = t;
+    }
+    __syncthreads();
+    if (threadIdx.x < kRowsPerCta && j0 + threadIdx.x < r) {
+        float t = 0.f;
+#pragma unroll
+        for (int i = 0; i < kSmallThreads / 32; ++i) t += red[threadIdx.x][i];
+        T[(size_t)m * r + j0 + threadIdx.x] = __float2bfloat16_rn(t);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// many tokens
+// ---------------------------------------------------------------------------
+constexpr int kTileM = 16;          // tokens per CTA (one mma.sync M tile)
+constexpr int kChunkK = 128;        // columns staged per pipeline step
+constexpr int kLargeThreads = 256;  // 16 threads per token row
+constexpr int kRowBytes = kChunkK * 2 + 16;  // padded smem row (272 B): conflict-free ldmatrix
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(src));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& a, uint32_t& b, uint32_t& c,
+                                            uint32_t& d) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(a), "=r"(b), "=r"(c), "=r"(d)
+                 : "r"(addr)
+                 : "memory");
+}
+__device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                        uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, "
+        "{%8,%9}, {%0,%1,%2,%3};\n"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// grid = ceil(M / 16).  dynamic smem: 2 stages x (16 + r) rows x 272 B.
+// MAXT = tiles of 8 T-columns per warp = ceil(r / 64).
+template <int MAXT>
+__global__ void __launch_bounds__(kLargeThreads)
+quant_act_large_kernel(const __half* __restrict__ X, const float* __restrict__ s,
+                       const __half* __restrict__ LA, int M, int K, int r,
+                       int8_t* __restrict__ Xq, float* __restrict__ a_scale,
+                       __nv_bfloat16* __restrict__ T) {
+    extern __shared__ __align__(16) uint8_t smem[];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int m0 = blockIdx.x * kTileM;
+    const int trow = tid >> 4;  // token row of this thread (0..15)
+    const int tcol = tid & 15;  // 16-byte column chunk within the 128-column step
+    const int m = m0 + trow;
+    const bool row_ok = m < M;
+    const __half* xrow = X + (size_t)(row_ok ? m : 0) * K;
+    const int nch = K / kChunkK;
+    const int stage_bytes = (kTileM + r) * kRowBytes;
+    const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem);
+    const int ntiles = r / 8;
+
+    auto issue_la = [&](int c, int stage) {  // r rows x 16 chunks of 16 B
+        const uint32_t dst0 = smem_base + stage * stage_bytes + kTileM * kRowBytes;
+        for (int i = tid; i < r * 16; i += kLargeThreads) {
+            int j = i >> 4, cc = i & 15;
+            cp_async16(dst0 + j * kRowBytes + cc * 16, LA + (size_t)j * K + c * kChunkK + cc * 8);
+        }
+    };
+
+    float acc[MAXT][4];
+#pragma unroll
+    for (int t = 0; t < MAXT; ++t)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[t][i] = 0.f;
+
+    float amax = 0.f;
+    if (r > 0) issue_la(0, 0);
+    cp_async_commit();
+    RawChunk rc = load_raw(xrow, s, tcol * 8, row_ok);
+
+    for (int c = 0; c < nch; ++c) {
+        const int stage = c & 1;
+        if (r > 0 && c + 1 < nch) issue_la(c + 1, stage ^ 1);
+        cp_async_commit();
+        {
+            float v[8];
+            smooth8(rc, v);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(v[i]));
+            if (r > 0) {
+                __half2 p0 = __floats2half2_rn(v[0], v[1]), p1 = __floats2half2_rn(v[2], v[3]);
+                __half2 p2 = __floats2half2_rn(v[4], v[5]), p3 = __floats2half2_rn(v[6], v[7]);
+                uint4 pk;
+                pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
+                pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
+                *reinterpret_cast<uint4*>(smem + stage * stage_bytes + trow * kRowBytes + tcol * 16) = pk;
+            }
+        }
+        if (c + 1 < nch) rc = load_raw(xrow, s, (c + 1) * kChunkK + tcol * 8, row_ok);
+        if (r > 0) {
+            cp_async_wait<1>();
+            __syncthreads();
+            const uint32_t a_base = smem_base + stage * stage_bytes;
+            const uint32_t b_base = a_base + kTileM * kRowBytes;
+            // A fragment: lanes 0-15 give rows 0-15 at k, lanes 16-31 rows 0-15 at k+8
+            const uint32_t a_addr = a_base + (lane & 15) * kRowBytes + (lane >> 4) * 16;
+#pragma unroll
+            for (int kk = 0; kk < kChunkK / 32; ++kk) {
+                uint32_t a0, a1, a2, a3, a4, a5, a6, a7;
+                ldmatrix_x4(a_addr + kk * 64, a0, a1, a2, a3);
+                ldmatrix_x4(a_addr + kk * 64 + 32, a4, a5, a6, a7);
+#pragma unroll
+                for (int t = 0; t < MAXT; ++t) {
+                    int nt = warp + t * 8;
+                    if (nt < ntiles) {
+                        // B: 8 rows of L_A (T columns) x 32 k = four 8x8 matrices along k
+                        uint32_t b_addr = b_base + (nt * 8 + (lane & 7)) * kRowBytes + kk * 64 +
+                                          (lane >> 3) * 16;
+                        uint32_t b0, b1, b2, b3;
+                        ldmatrix_x4(b_addr, b0, b1, b2, b3);
+                        mma_f16(acc[t], a0, a1, a2, a3, b0, b1);
+                        mma_f16(acc[t], a4, a5, a6, a7, b2, b3);
+                    }
+                }
+            }
+            __syncthreads();
+        }
+    }
+    cp_async_wait<0>();
+
+    // ---- per-token scale: the 16 threads of a row are 16 consecutive lanes ----
+#pragma unroll
+    for (int o = 8; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    const float sc = __fdiv_rn(amax, 127.0f);
+    if (tcol == 0 && row_ok) a_scale[m] = sc;
+
+    // ---- T tile (fp32 accumulators -> bf16) ----
+    if (r > 0) {
+        const int g = lane >> 2, tq = lane & 3;
+#pragma unroll
+        for (int t = 0; t < MAXT; ++t) {
+            int nt = warp + t * 8;
+            if (nt < ntiles) {
+                int j = nt * 8 + tq * 2;
+                if (m0 + g < M)
+                    *reinterpret_cast<__nv_bfloat162*>(T + (size_t)(m0 + g) * r + j) =
+                        __floats2bfloat162_rn(acc[t][0], acc[t][1]);
+                if (m0 + g + 8 < M)
+                    *reinterpret_cast<__nv_bfloat162*>(T + (size_t)(m0 + g + 8) * r + j) =
+                        __floats2bfloat162_rn(acc[t][2], acc[t][3]);
+            }
+        }
+    }
+
+    // ---- second sweep: int8 codes ----
+    if (!row_ok) return;
+    int8_t* out = Xq + (size_t)m * K;
+    rc = load_raw(xrow, s, tcol * 8, true);
+    for (int c = 0; c < nch; ++c) {
+        RawChunk cur = rc;
+        if (c + 1 < nch) rc = load_raw(xrow, s, (c + 1) * kChunkK + tcol * 8, true);
+        float v[8];
+        smooth8(cur, v);
+        *reinterpret_cast<uint2*>(out + c * kChunkK + tcol * 8) = quant8(v, sc, amax > 0.f);
+    }
+}
+
+template <int MAXT>
+int launch_large(const __half* X, const float* s, const __half* LA, int M, int K, int r,
+                 int8_t* Xq, float* a_scale, __nv_bfloat16* T, cudaStream_t st) {
+    size_t smem = 2 * (size_t)(kTileM + r) * kRowBytes;
+    cudaError_t e = cudaFuncSetAttribute(quant_act_large_kernel<MAXT>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return record_cuda_error(e, "quant_act_large smem attribute");
+    int grid = (M + kTileM - 1) / kTileM;
+    quant_act_large_kernel<MAXT><<<grid, kLargeThreads, smem, st>>>(X, s, LA, M, K, r, Xq, a_scale, T);
+    return check_launch("quant_act_large_kernel");
+}
+
+}  // namespace
+
+int launch_quant_act(const __half* X, const float* s, const __half* LA, int M, int K, int r,
+                     int8_t* Xq, float* a_scale, __nv_bfloat16* T, cudaStream_t st) {
+    if (M == 0) return ASER_OK;
+    if (M <= 32) {
+        size_t smem = (size_t)K * sizeof(float);
+        if (smem > 48 * 1024) {
+            cudaError_t e = cudaFuncSetAttribute(quant_act_small_kernel,
+                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return record_cuda_error(e, "quant_act_small smem attribute");
+        }
+        dim3 grid(1 + (r + kRowsPerCta - 1) / kRowsPerCta, M);
+        quant_act_small_kernel<<<grid, kSmallThreads, smem, st>>>(X, s, LA, M, K, r, Xq, a_scale, T);
+        return check_launch("quant_act_small_kernel");
+    }
+    if (r <= 64) return launch_large<1>(X, s, LA, M, K, r, Xq, a_scale, T, st);
+    if (r <= 128) return launch_large<2>(X, s, LA, M, K, r, Xq, a_scale, T, st);
+    return launch_large<4>(X, s, LA, M, K, r, Xq, a_scale, T, st);
+}
+
+}  // namespace aser

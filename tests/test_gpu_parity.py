@@ -1,0 +1,181 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle on the same
+seeded inputs.  Integer stages bit-exact; fp16 outputs within 2e-3 * max|y_ref| per row."""
+import numpy as np
+import pytest
+import torch
+
+import aser_synth as synth
+from oracle import forward as F
+from gpu_util import to_dev, oracle_layer, assert_rows_close, assert_T_close
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def aser(cuda_device):
+    import paper_2411_07762_b200 as aser
+    return aser
+
+
+def bits(a):
+    return np.ascontiguousarray(a).view(np.uint32)
+
+
+# ---------------------------------------------------------------------------
+# aser_pack_w4 / repack
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("N,K,smooth", [(512, 512, True), (136, 1024, True), (8, 128, False),
+                                        (1024, 4096, True), (264, 14336, True)])
+def test_pack_w4_bit_exact(aser, N, K, smooth):
+    lay = synth.make_layer(1, N, K, seed=100 + N + K, n_cal=8)
+    s = synth.standin_smoothing_vector(K, lay.outlier_idx, 11.5) if smooth else None
+    W = lay.W.copy()
+    if N >= 136:
+        W[3] = 0                        # zero row: scale 0, codes 0
+        W[5, :] = 0
+        W[5, 7] = np.float16(3.5)       # single element: code 7 and exact ties elsewhere
+        W[6, :8] = np.array([7, .5, 1.5, 2.5, -2.5, 6.5, -6.5, -7], np.float16)
+        W[6, 8:] = 0
+    q, w_scale = F.quant_w4(W, s)
+    Wq, wsc = aser.pack_w4(to_dev(W), None if s is None else to_dev(s))
+    assert np.array_equal(Wq.cpu().numpy(), F.pack_w4(q))
+    assert np.array_equal(bits(wsc.cpu().numpy()), bits(w_scale))
+    Wk = aser.repack_w4(Wq)
+    assert Wk.numel() == aser.repacked_bytes(N, K)
+    back = aser.unrepack_w4(Wk, N, K)
+    assert torch.equal(back, Wq)
+
+
+def test_repack_layout_by_definition(aser):
+    """Word w of sub-block `sub`, row `row` covers columns 32*sub + 8*w .. +7 with column
+    c0+i in nibble 2i and column c0+4+i in nibble 2i+1."""
+    N, K = 256, 384
+    rng = np.random.default_rng(5)
+    q = rng.integers(-8, 8, (N, K)).astype(np.int8)
+    Wq = to_dev(F.pack_w4(q))
+    Wk = aser.repack_w4(Wq).cpu().numpy().view(np.uint32).reshape(N // 128, K // 128, 4, 128, 4)
+    for (nb, kb, sub, row, w) in [(0, 0, 0, 0, 0), (1, 2, 3, 127, 3), (0, 1, 2, 77, 1), (1, 0, 1, 5, 2)]:
+        word = int(Wk[nb, kb, sub, row, w])
+        c0 = kb * 128 + sub * 32 + w * 8
+        n = nb * 128 + row
+        for i in range(4):
+            assert (word >> (8 * i)) & 0xF == int(q[n, c0 + i]) & 0xF
+            assert (word >> (8 * i + 4)) & 0xF == int(q[n, c0 + 4 + i]) & 0xF
+
+
+# ---------------------------------------------------------------------------
+# aser_quant_act
+# ---------------------------------------------------------------------------
+ACT_CASES = [  # M, K, r
+    (1, 512, 16), (3, 4096, 64), (8, 4096, 64), (16, 512, 16), (17, 1024, 0), (32, 8192, 32),
+    (33, 512, 16), (127, 1024, 64), (129, 4096, 128), (300, 2048, 256), (64, 14336, 64),
+]
+
+
+@pytest.mark.parametrize("M,K,r", ACT_CASES)
+def test_quant_act_parity(aser, M, K, r):
+    lay = synth.make_layer(M, 8, K, seed=200 + M + K + r, n_cal=8)
+    s = synth.standin_smoothing_vector(K, lay.outlier_idx, 13.0)
+    X = lay.X.copy()
+    if M >= 3:
+        X[1] = 0                                   # zero token: scale 0, codes 0
+        X[2, :] = 0
+        X[2, :6] = np.array([127, .5, 1.5, 2.5, -2.5, -126.5], np.float16)   # exact ties
+    L_A = synth.standin_factors(8, K, r, seed=M, scale_a=0.05)[0] if r else None
+    xs = F.smooth_act(X, s)
+    Xq_ref, sc_ref = F.quant_act(xs)
+    Xq, sc, T = aser.quant_act(to_dev(X), to_dev(s), None if L_A is None else to_dev(L_A))
+    assert np.array_equal(Xq.cpu().numpy(), Xq_ref)
+    assert np.array_equal(bits(sc.cpu().numpy()), bits(sc_ref))
+    if r:
+        T_ref = F.down_proj(xs, L_A)
+        assert_T_close(T.float().cpu().numpy(), T_ref)
+
+
+def test_quant_act_without_smoothing_vector(aser):
+    lay = synth.make_layer(5, 8, 256, seed=9, n_cal=8)
+    Xq, sc, _ = aser.quant_act(to_dev(lay.X), None, None)
+    Xq_ref, sc_ref = F.quant_act(F.smooth_act(lay.X, None))
+    assert np.array_equal(Xq.cpu().numpy(), Xq_ref) and np.array_equal(bits(sc.cpu().numpy()), bits(sc_ref))
+
+
+# ---------------------------------------------------------------------------
+# whole path: quant_act -> linear
+# ---------------------------------------------------------------------------
+def run_path(aser, lay, s, Wq_ref, w_scale_ref, L_A, L_B, impl, rows=None, use_dgemm=False):
+    M, K = lay.X.shape
+    N = lay.W.shape[0]
+    r = 0 if L_A is None else L_A.shape[0]
+    dW, ds = to_dev(lay.W), to_dev(s)
+    Wq, wsc = aser.pack_w4(dW, ds)
+    assert np.array_equal(Wq.cpu().numpy(), Wq_ref)
+    assert np.array_equal(bits(wsc.cpu().numpy()), bits(w_scale_ref))
+    dLA = None if r == 0 else to_dev(L_A)
+    dLB = None if r == 0 else to_dev(L_B)
+    Xq, sc, T = aser.quant_act(to_dev(lay.X), ds, dLA)
+    acc = torch.full((M, N), -7, dtype=torch.int32, device="cuda")
+    if impl == "simt":
+        Y = aser.linear_w4a8_lr_simt(Xq, sc, Wq, wsc, T, dLB, acc_debug=acc)
+    else:
+        Wk = aser.repack_w4(Wq)
+        ws = aser.new_workspace(M, N, K, r)
+        if r:
+            Y = aser.linear_w4a8_lr(Xq, sc, Wk, wsc, T, dLB, N, ws, acc_debug=acc)
+        else:
+            Y = aser.linear_w4a8(Xq, sc, Wk, wsc, N, ws, acc_debug=acc)
+        aser.check_status(ws)
+    torch.cuda.synchronize()
+    ref = F.forward(lay.X, s, Wq_ref, w_scale_ref, L_A, L_B, rows=rows, use_dgemm=use_dgemm)
+    assert np.array_equal(Xq.cpu().numpy(), ref.Xq)
+    assert np.array_equal(bits(sc.cpu().numpy()), bits(ref.a_scale))
+    acc_h = acc.cpu().numpy()
+    assert np.array_equal(acc_h if rows is None else acc_h[rows], ref.acc)
+    assert_rows_close(Y.cpu().numpy(), ref.y, rows)
+    return Y
+
+
+PATH_CASES = [  # M, N, K, r
+    (16, 512, 512, 16), (1, 256, 512, 16), (7, 136, 1024, 32), (33, 264, 512, 0),
+    (130, 384, 1024, 64), (257, 520, 2048, 128), (40, 128, 384, 256),
+]
+
+
+@pytest.mark.parametrize("impl", ["simt", "tc"])
+@pytest.mark.parametrize("M,N,K,r", PATH_CASES)
+def test_path_parity_small(aser, impl, M, N, K, r):
+    lay = synth.make_layer(M, N, K, seed=300 + M + N + K + r, n_cal=64,
+                           n_out=max(1, K // 100))
+    s, Wq, w_scale, L_A, L_B = oracle_layer(lay, r, construct=(K <= 1024 and r > 0))
+    if r == 0:
+        L_A = L_B = None
+    run_path(aser, lay, s, Wq, w_scale, L_A, L_B, impl)
+
+
+@pytest.mark.parametrize("impl", ["simt", "tc"])
+def test_config1_tiny_with_constructed_factors(aser, impl):
+    lay, r = synth.config1_tiny()
+    s, Wq, w_scale, L_A, L_B = oracle_layer(lay, r, construct=True)
+    Y = run_path(aser, lay, s, Wq, w_scale, L_A, L_B, impl)
+    # the compensated output is closer to the fp product than the plain W4A8 one
+    plain = run_path(aser, lay, s, Wq, w_scale, None, None, impl)
+    ref = lay.X.astype(np.float64) @ lay.W.astype(np.float64).T
+    e_lr = np.linalg.norm(Y.cpu().numpy().astype(np.float64) - ref)
+    e_plain = np.linalg.norm(plain.cpu().numpy().astype(np.float64) - ref)
+    assert e_lr < e_plain
+
+
+@pytest.mark.parametrize("impl", ["tc"])
+@pytest.mark.parametrize("M", [1, 8])
+def test_config2_decode_full_size(aser, impl, M):
+    lay, r = synth.config2_decode(M)
+    s, Wq, w_scale, L_A, L_B = oracle_layer(lay, r, construct=(M == 8))
+    run_path(aser, lay, s, Wq, w_scale, L_A, L_B, impl, use_dgemm=True)
+
+
+@pytest.mark.parametrize("impl", ["tc"])
+@pytest.mark.parametrize("which", ["gate_up", "down"])
+def test_config3_prefill_full_size_sampled_rows(aser, impl, which):
+    lay, r = synth.config3_prefill(which)
+    s, Wq, w_scale, L_A, L_B = oracle_layer(lay, r, construct=False)
+    rows = np.array([0, 1, 127, 128, 1000, 1023, 1024, 2046, 2047])
+    run_path(aser, lay, s, Wq, w_scale, L_A, L_B, impl, rows=rows, use_dgemm=True)

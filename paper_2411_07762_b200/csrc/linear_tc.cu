@@ -1,9 +1,758 @@
-// placeholder: replaced by the tcgen05 kernel
+// Tensor-core kernel of the ASER linear (Sec. 4.2, "W_q X + L_A L_B X"):
+//   acc = Xq Wq^T (int8 x int4 -> int32),  Y = fp16(acc * a_scale[m] * w_scale[n] + T L_B^T).
+//
+// Orientation: the output tile is computed transposed, D[n, token], so that the WEIGHTS sit on
+// the MMA's M side.  Packed int4 weights are streamed from HBM with bulk copies into shared
+// memory, turned into int8 (value 16*q) by two ALU operations per eight codes, and written
+// straight into TENSOR MEMORY as the A operand of tcgen05.mma kind::i8; they never go back to
+// shared memory.  The int8 activations arrive by TMA (128-byte swizzle) as the B operand, so the
+// MMA N dimension is the token tile (16..128) and decode shapes use the same kernel.
+// The low-rank term is a second accumulator fed by kind::f16 MMAs on L_B (TMA) and T (TMA, then
+// bf16 -> fp16 in place).  Work is split stream-K style: the list of (tile, 128-column block)
+// units is cut into equal contiguous ranges, one per CTA; tiles shared by several CTAs are
+// summed through the workspace by whichever CTA arrives last.
+//
+// Warp roles (320 threads): 0 = copy producer, 1 = MMA issuer (+ TMEM owner),
+// 2..5 = int4 -> int8 unpack into TMEM (+ T conversion), 6..9 = epilogue.
+// Every wait is bounded: on expiry the CTA sets the status word and winds down.
+#include <cuda.h>
+
 #include "aser_common.cuh"
+
 namespace aser {
-size_t linear_tc_workspace_bytes(int, int, int, int) { return 0; }
-int launch_linear_tc(const int8_t*, const float*, const uint8_t*, const float*, const __nv_bfloat16*,
-                     const __half*, int, int, int, int, __half*, int32_t*, void*, size_t, cudaStream_t) {
-    return ASER_ERR_SHAPE;
+
+namespace {
+
+constexpr int kThreads = 320;
+constexpr int kASlots = 4;        // A-operand slots in tensor memory (32 columns each)
+constexpr int kLrSlots = 2;       // ring of low-rank chunks (64 columns of r each)
+constexpr int kMaxCtas = 160;     // upper bound on the persistent grid (workspace sizing)
+constexpr uint32_t kStatusTimeout = 1u;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
+
+template <int BT>
+struct Cfg {
+    static constexpr int NW = (BT == 128) ? 8 : 12;   // weight ring (8 KiB each)
+    static constexpr int NX = (BT == 128) ? 4 : 8;    // activation ring (BT x 128 B each)
+    static constexpr int XBytes = BT * 128;
+    static constexpr int LbBytes = 128 * 128;          // 128 rows x 64 fp16
+    static constexpr int TBytes = BT * 128;            // BT rows x 64 bf16/fp16
+    static constexpr int OffW = 0;
+    static constexpr int OffX = OffW + NW * kWkBlockBytes;
+    static constexpr int OffLb = OffX + NX * XBytes;
+    static constexpr int OffT = OffLb + kLrSlots * LbBytes;
+    static constexpr int OffBar = OffT + kLrSlots * TBytes;
+    static constexpr int NumBars = 2 * NW + 2 * NX + 2 * kASlots + 3 * kLrSlots + 2 + 2 + 1;
+    static constexpr int SmemBytes = OffBar + NumBars * 8 + 64 + 1024;  // + slack for 1 KiB alignment
+    static constexpr int TmemColsUsed = 3 * BT + kASlots * 32;
+    static constexpr int TmemCols = TmemColsUsed <= 256 ? 256 : 512;
+};
+
+// ---------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
 }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes,
+                                              uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y,
+                                            uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async_smem() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                 ::"r"(bar)
+                 : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem desc], int8 x int8 -> int32
+__device__ __forceinline__ void mma_i8_ts(uint32_t d, uint32_t a, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d), "r"(a), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// D[tmem] (+)= A[smem desc] * B[smem desc], fp16 x fp16 -> fp32
+__device__ __forceinline__ void mma_f16_ss(uint32_t d, uint64_t adesc, uint64_t bdesc,
+                                           uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+        "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]),
+        "r"(v[7]), "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]),
+        "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]),
+        "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]),
+        "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() {
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
+          "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]),
+          "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr)
+        : "memory");
+}
+// Waits for the tensor-memory loads; the registers are listed as in/out operands so that no
+// use of them can be scheduled ahead of the wait.
+__device__ __forceinline__ void tmem_wait_ld(uint32_t (&v)[16]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]),
+                   "+r"(v[7]), "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]),
+                   "+r"(v[13]), "+r"(v[14]), "+r"(v[15])
+                 :
+                 : "memory");
+}
+// Barrier over `count` threads that also ANDs a predicate across them.
+__device__ __forceinline__ bool named_bar_all(int id, int count, bool pred) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %3, 0;\n\t"
+        "barrier.cta.red.and.pred q, %1, %2, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(out)
+        : "r"(id), "r"(count), "r"((uint32_t)pred)
+        : "memory");
+    return out != 0;
+}
+__device__ __forceinline__ void named_bar_sync(int id, int count) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes,
+// groups of 8 rows 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);        // start address
+    d |= (uint64_t)(1024u >> 4) << 32;              // stride between 8-row groups
+    d |= 1ull << 46;                                // descriptor version of this architecture
+    d |= 2ull << 61;                                // 128-byte swizzle
+    return d;
+}
+
+// Instruction descriptor: dense, D format (1 = f32, 2 = s32), A/B format, K-major both, N, M.
+__host__ __device__ constexpr uint32_t make_idesc(uint32_t dfmt, uint32_t abfmt, uint32_t M,
+                                                  uint32_t N) {
+    return (dfmt << 4) | (abfmt << 7) | (abfmt << 10) | ((N >> 3) << 17) | ((M >> 4) << 24);
+}
+
+// ---------------------------------------------------------------------------
+// kernel parameters and work enumeration
+// ---------------------------------------------------------------------------
+struct Params {
+    const uint8_t* Wk;
+    const float* a_scale;
+    const float* w_scale;
+    __half* Y;
+    int32_t* acc_debug;
+    uint32_t* status;      // workspace word 0
+    int* counters;         // one per tile
+    int32_t* part_int;     // [grid][2][BT][128]
+    float* part_lr;        // [grid][BT][128]
+    int M, N, K, r;
+    int KB, TT, NT;        // 128-column blocks, token tiles, 128-row tiles
+    long long units;       // NT * TT * KB
+};
+
+struct Work {
+    int tile, nt, tt, kb0, kb1;
+    bool has_lr, whole;
+};
+
+__device__ __forceinline__ long long range_begin(long long units, int c, int G) {
+    return units * c / G;
+}
+// CTA that owns unit x.
+__device__ __forceinline__ int unit_owner(long long units, long long x, int G) {
+    return (int)(((x + 1) * G - 1) / units);
+}
+
+__device__ __forceinline__ bool next_work(long long& u, long long u1, const Params& p, Work& w) {
+    if (u >= u1) return false;
+    w.tile = (int)(u / p.KB);
+    w.kb0 = (int)(u % p.KB);
+    long long left = u1 - u;
+    w.kb1 = (int)((long long)(p.KB - w.kb0) < left ? p.KB : w.kb0 + left);
+    w.nt = w.tile / p.TT;
+    w.tt = w.tile % p.TT;
+    w.has_lr = (w.kb0 == 0) && p.r > 0;
+    w.whole = (w.kb0 == 0) && (w.kb1 == p.KB);
+    u += w.kb1 - w.kb0;
+    return true;
+}
+
+struct Abort {
+    volatile int* flag;   // shared
+    uint32_t* status;     // global
+};
+
+// Bounded wait on an mbarrier phase.  Returns false after the time limit or when another role
+// of this CTA has already given up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const Abort& ab) {
+    if (mbar_try_wait(bar, parity)) return true;
+    unsigned long long t0 = global_ns();
+    uint32_t spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 63u) == 0) {
+            if (*ab.flag) return false;
+            if (global_ns() - t0 > kWaitLimitNs) {
+                *ab.flag = 1;
+                atomicOr(ab.status, kStatusTimeout);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+// ---------------------------------------------------------------------------
+// the kernel
+// ---------------------------------------------------------------------------
+template <int BT>
+__global__ void __launch_bounds__(kThreads, 1)
+linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_lb,
+                 const __grid_constant__ CUtensorMap map_t, const Params p) {
+    using C = Cfg<BT>;
+    extern __shared__ uint8_t smem_raw[];
+    // 1 KiB alignment for the swizzled tiles
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bar0 = sbase + C::OffBar;
+    auto bar = [&](int i) { return bar0 + 8u * i; };
+    // barrier indices
+    constexpr int B_FULL_W = 0, B_EMPTY_W = B_FULL_W + C::NW, B_FULL_X = B_EMPTY_W + C::NW,
+                  B_EMPTY_X = B_FULL_X + C::NX, B_A_FULL = B_EMPTY_X + C::NX,
+                  B_A_EMPTY = B_A_FULL + kASlots, B_FULL_LR = B_A_EMPTY + kASlots,
+                  B_CONV_LR = B_FULL_LR + kLrSlots, B_EMPTY_LR = B_CONV_LR + kLrSlots,
+                  B_ACC_FULL = B_EMPTY_LR + kLrSlots, B_ACC_EMPTY = B_ACC_FULL + 2,
+                  B_DLR_EMPTY = B_ACC_EMPTY + 2;
+    static_assert(B_DLR_EMPTY + 1 == C::NumBars, "barrier count");
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + C::OffBar + C::NumBars * 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    int* last_flag = reinterpret_cast<int*>(tmem_slot + 2);
+    volatile int* never_flag = reinterpret_cast<volatile int*>(tmem_slot + 3);  // stays 0
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int G = gridDim.x, cta = blockIdx.x;
+    const long long u_begin = range_begin(p.units, cta, G), u_end = range_begin(p.units, cta + 1, G);
+    Abort ab{abort_flag, p.status};
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < C::NW; ++i) { mbar_init(bar(B_FULL_W + i), 1); mbar_init(bar(B_EMPTY_W + i), 128); }
+        for (int i = 0; i < C::NX; ++i) { mbar_init(bar(B_FULL_X + i), 1); mbar_init(bar(B_EMPTY_X + i), 1); }
+        for (int i = 0; i < kASlots; ++i) { mbar_init(bar(B_A_FULL + i), 128); mbar_init(bar(B_A_EMPTY + i), 1); }
+        for (int i = 0; i < kLrSlots; ++i) {
+            mbar_init(bar(B_FULL_LR + i), 1); mbar_init(bar(B_CONV_LR + i), 128); mbar_init(bar(B_EMPTY_LR + i), 1);
+        }
+        for (int i = 0; i < 2; ++i) { mbar_init(bar(B_ACC_FULL + i), 1); mbar_init(bar(B_ACC_EMPTY + i), 128); }
+        mbar_init(bar(B_DLR_EMPTY), 128);
+        *abort_flag = 0;
+        *last_flag = 0;
+        *never_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_proxy_async_smem();
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)C::TmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    const uint32_t tm_dint0 = tmem, tm_dlr = tmem + 2 * BT, tm_a0 = tmem + 3 * BT;
+    const int lr_chunks = (p.r + 63) / 64;
+
+    if (warp == 0) {
+        // =================== copy producer (one lane, three rings) ===================
+        if (lane == 0) {
+            long long uw = u_begin, ux = u_begin, ul = u_begin;   // cursors
+            uint32_t cw = 0, cx = 0, cl = 0;                     // items issued per ring
+            Work wl{};                                           // current low-rank work item
+            int lc = 0;                                          // next chunk of wl
+            bool have_wl = false;
+            auto advance_lr = [&]() {
+                have_wl = false;
+                while (p.r > 0 && next_work(ul, u_end, p, wl)) {
+                    if (wl.has_lr) { have_wl = true; lc = 0; break; }
+                }
+            };
+            advance_lr();
+            unsigned long long t0 = global_ns();
+            uint32_t idle = 0;
+            bool failed = false;
+            while (uw < u_end || ux < u_end || have_wl) {
+                bool progressed = false;
+                if (uw < u_end) {
+                    int s = cw % C::NW;
+                    if (mbar_try_wait(bar(B_EMPTY_W + s), ((cw / C::NW) & 1) ^ 1)) {
+                        // units are stored in the order they are consumed: block index == unit's
+                        // (row tile, column block) with tiles of one row tile adjacent in tt
+                        int tile = (int)(uw / p.KB), kb = (int)(uw % p.KB), nt = tile / p.TT;
+                        mbar_arrive_expect_tx(bar(B_FULL_W + s), kWkBlockBytes);
+                        bulk_copy_g2s(sbase + C::OffW + s * kWkBlockBytes,
+                                      p.Wk + ((size_t)nt * p.KB + kb) * kWkBlockBytes, kWkBlockBytes,
+                                      bar(B_FULL_W + s));
+                        ++cw; ++uw; progressed = true;
+                    }
+                }
+                if (ux < u_end) {
+                    int s = cx % C::NX;
+                    if (mbar_try_wait(bar(B_EMPTY_X + s), ((cx / C::NX) & 1) ^ 1)) {
+                        int tile = (int)(ux / p.KB), kb = (int)(ux % p.KB), tt = tile % p.TT;
+                        mbar_arrive_expect_tx(bar(B_FULL_X + s), C::XBytes);
+                        tma_load_2d(sbase + C::OffX + s * C::XBytes, &map_x, kb * 128, tt * BT,
+                                    bar(B_FULL_X + s));
+                        ++cx; ++ux; progressed = true;
+                    }
+                }
+                if (have_wl) {
+                    int s = cl % kLrSlots;
+                    if (mbar_try_wait(bar(B_EMPTY_LR + s), ((cl / kLrSlots) & 1) ^ 1)) {
+                        mbar_arrive_expect_tx(bar(B_FULL_LR + s), C::LbBytes + C::TBytes);
+                        tma_load_2d(sbase + C::OffLb + s * C::LbBytes, &map_lb, lc * 64, wl.nt * 128,
+                                    bar(B_FULL_LR + s));
+                        tma_load_2d(sbase + C::OffT + s * C::TBytes, &map_t, lc * 64, wl.tt * BT,
+                                    bar(B_FULL_LR + s));
+                        ++cl; ++lc; progressed = true;
+                        if (lc == lr_chunks) advance_lr();
+                    }
+                }
+                if (progressed) { idle = 0; continue; }
+                if (idle == 0) t0 = global_ns();
+                if ((++idle & 63u) == 0) {
+                    if (*abort_flag) { failed = true; break; }
+                    if (global_ns() - t0 > kWaitLimitNs) {
+                        *abort_flag = 1;
+                        atomicOr(p.status, kStatusTimeout);
+                        failed = true;
+                        break;
+                    }
+                }
+            }
+            if (failed || *abort_flag) {
+                // let copies already issued land before the CTA's shared memory goes away
+                for (uint32_t i = (cw > (uint32_t)C::NW ? cw - C::NW : 0); i < cw; ++i)
+                    mbar_wait(bar(B_FULL_W + i % C::NW), (i / C::NW) & 1, Abort{never_flag, p.status});
+                for (uint32_t i = (cx > (uint32_t)C::NX ? cx - C::NX : 0); i < cx; ++i)
+                    mbar_wait(bar(B_FULL_X + i % C::NX), (i / C::NX) & 1, Abort{never_flag, p.status});
+                for (uint32_t i = (cl > (uint32_t)kLrSlots ? cl - kLrSlots : 0); i < cl; ++i)
+                    mbar_wait(bar(B_FULL_LR + i % kLrSlots), (i / kLrSlots) & 1, Abort{never_flag, p.status});
+            }
+        }
+    } else if (warp == 1) {
+        // =================== MMA issuer (one lane) ===================
+        if (lane == 0) {
+            constexpr uint32_t idesc_i8 = make_idesc(2, 1, 128, BT);
+            constexpr uint32_t idesc_f16 = make_idesc(1, 0, 128, BT);
+            long long u = u_begin;
+            Work w;
+            uint32_t cx = 0, ca = 0, cl = 0, ci = 0, clr_items = 0;
+            bool ok = true;
+            while (ok && next_work(u, u_end, p, w)) {
+                const int buf = ci & 1;
+                const uint32_t d_int = tm_dint0 + buf * BT;
+                ok = mbar_wait(bar(B_ACC_EMPTY + buf), ((ci >> 1) & 1) ^ 1, ab);
+                if (!ok) break;
+                tc_fence_after();
+                for (int kb = w.kb0; kb < w.kb1 && ok; ++kb) {
+                    const int sx = cx % C::NX, sa = ca % kASlots;
+                    ok = mbar_wait(bar(B_FULL_X + sx), (cx / C::NX) & 1, ab) &&
+                         mbar_wait(bar(B_A_FULL + sa), (ca / kASlots) & 1, ab);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint64_t xdesc = smem_desc_sw128(sbase + C::OffX + sx * C::XBytes);
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        mma_i8_ts(d_int, tm_a0 + sa * 32 + kk * 8, xdesc + 2 * kk, idesc_i8,
+                                  (kb != w.kb0 || kk != 0) ? 1u : 0u);
+                    tc_commit(bar(B_EMPTY_X + sx));
+                    tc_commit(bar(B_A_EMPTY + sa));
+                    ++cx; ++ca;
+                }
+                if (ok && w.has_lr) {
+                    ok = mbar_wait(bar(B_DLR_EMPTY), (clr_items & 1) ^ 1, ab);
+                    for (int c = 0; c < lr_chunks && ok; ++c) {
+                        const int s = cl % kLrSlots;
+                        ok = mbar_wait(bar(B_CONV_LR + s), (cl / kLrSlots) & 1, ab);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint64_t adesc = smem_desc_sw128(sbase + C::OffLb + s * C::LbBytes);
+                        const uint64_t bdesc = smem_desc_sw128(sbase + C::OffT + s * C::TBytes);
+                        int steps = (p.r - c * 64) / 16;
+                        if (steps > 4) steps = 4;
+                        for (int kk = 0; kk < steps; ++kk)
+                            mma_f16_ss(tm_dlr, adesc + 2 * kk, bdesc + 2 * kk, idesc_f16,
+                                       (c != 0 || kk != 0) ? 1u : 0u);
+                        tc_commit(bar(B_EMPTY_LR + s));
+                        ++cl;
+                    }
+                    ++clr_items;
+                }
+                if (ok) tc_commit(bar(B_ACC_FULL + buf));
+                ++ci;
+            }
+        }
+    } else if (warp < 6) {
+        // =================== unpack warps: int4 -> int8 (x16) into tensor memory ===================
+        const int q = warp & 3;                    // TMEM lane quarter this warp may touch
+        const int row = q * 32 + lane;             // weight row inside the 128-row tile
+        const int t128 = (warp - 2) * 32 + lane;   // 0..127 among the unpack threads
+        long long u = u_begin;
+        Work w;
+        uint32_t cw = 0, ca = 0, cl = 0;
+        bool ok = true;
+        while (ok && next_work(u, u_end, p, w)) {
+            for (int kb = w.kb0; kb < w.kb1 && ok; ++kb) {
+                const int sw = cw % C::NW, sa = ca % kASlots;
+                ok = mbar_wait(bar(B_FULL_W + sw), (cw / C::NW) & 1, ab);
+                if (!ok) break;
+                const uint8_t* wsrc = smem + C::OffW + sw * kWkBlockBytes + row * 16;
+                uint32_t v[32];
+#pragma unroll
+                for (int sub = 0; sub < 4; ++sub) {
+                    uint4 x = *reinterpret_cast<const uint4*>(wsrc + sub * 2048);
+                    const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        v[sub * 8 + 2 * i] = (xs[i] << 4) & 0xF0F0F0F0u;   // columns c0 .. c0+3
+                        v[sub * 8 + 2 * i + 1] = xs[i] & 0xF0F0F0F0u;      // columns c0+4 .. c0+7
+                    }
+                }
+                mbar_arrive(bar(B_EMPTY_W + sw));   // values are in registers: slot may be refilled
+                ok = mbar_wait(bar(B_A_EMPTY + sa), ((ca / kASlots) & 1) ^ 1, ab);
+                if (!ok) break;
+                tc_fence_after();
+                tmem_st32(tm_a0 + sa * 32 + ((uint32_t)(q * 32) << 16), v);
+                tmem_wait_st();
+                tc_fence_before();
+                mbar_arrive(bar(B_A_FULL + sa));
+                ++cw; ++ca;
+            }
+            if (ok && w.has_lr) {
+                for (int c = 0; c < lr_chunks && ok; ++c) {
+                    const int s = cl % kLrSlots;
+                    ok = mbar_wait(bar(B_FULL_LR + s), (cl / kLrSlots) & 1, ab);
+                    if (!ok) break;
+                    // T chunk: bf16 -> fp16 in place (same element size, same swizzled position)
+                    uint8_t* tb = smem + C::OffT + s * C::TBytes;
+                    for (int i = t128; i < C::TBytes / 16; i += 128) {
+                        uint4 raw = *reinterpret_cast<uint4*>(tb + i * 16);
+                        uint32_t in[4] = {raw.x, raw.y, raw.z, raw.w}, out[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            float lo = __uint_as_float(in[e] << 16);
+                            float hi = __uint_as_float(in[e] & 0xFFFF0000u);
+                            __half2 h = __floats2half2_rn(lo, hi);
+                            out[e] = *reinterpret_cast<uint32_t*>(&h);
+                        }
+                        *reinterpret_cast<uint4*>(tb + i * 16) = make_uint4(out[0], out[1], out[2], out[3]);
+                    }
+                    fence_proxy_async_smem();
+                    mbar_arrive(bar(B_CONV_LR + s));
+                    ++cl;
+                }
+            }
+        }
+    } else {
+        // =================== epilogue warps ===================
+        const int q = warp & 3;
+        const int nl = q * 32 + lane;              // row of D = output channel inside the tile
+        const int et = (warp - 6) * 32 + lane;     // 0..127 among the epilogue threads
+        const uint32_t lane_sel = (uint32_t)(q * 32) << 16;
+        long long u = u_begin;
+        Work w;
+        uint32_t ci = 0;
+        int partial_idx = 0;                       // 0: first partial item of this CTA, 1: second
+        bool ok = true;
+        while (ok && next_work(u, u_end, p, w)) {
+            const int buf = ci & 1;
+            ok = mbar_wait(bar(B_ACC_FULL + buf), (ci >> 1) & 1, ab);
+            ok = named_bar_all(1, 128, ok);   // the 128 epilogue threads go on or give up together
+            if (!ok) break;
+            tc_fence_after();
+            const int n = w.nt * 128 + nl;
+            const bool n_ok = n < p.N;
+            const float ws = n_ok ? __ldg(p.w_scale + n) : 0.f;
+            const uint32_t d_int = tm_dint0 + buf * BT + lane_sel;
+            int32_t* pint = p.part_int + ((size_t)cta * 2 + partial_idx) * (BT * 128);
+            float* plr = p.part_lr + (size_t)cta * (BT * 128);
+#pragma unroll 1
+            for (int c0 = 0; c0 < BT; c0 += 16) {
+                uint32_t vi[16], vf[16];
+                tmem_ld16(d_int + c0, vi);
+                if (w.has_lr) tmem_ld16(tm_dlr + lane_sel + c0, vf);
+                tmem_wait_ld(vi);
+                if (w.has_lr) tmem_wait_ld(vf);
+                if (w.whole) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const int tok = w.tt * BT + c0 + j;
+                        if (tok < p.M && n_ok) {
+                            const int acc = ((int)vi[j]) >> 4;
+                            float y = (float)acc * __ldg(p.a_scale + tok) * ws;
+                            if (w.has_lr) y += __uint_as_float(vf[j]);
+                            p.Y[(size_t)tok * p.N + n] = __float2half_rn(y);
+                            if (p.acc_debug) p.acc_debug[(size_t)tok * p.N + n] = acc;
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        pint[(c0 + j) * 128 + nl] = (int)vi[j];
+                        if (w.has_lr) plr[(c0 + j) * 128 + nl] = __uint_as_float(vf[j]);
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(bar(B_ACC_EMPTY + buf));
+            if (w.has_lr) mbar_arrive(bar(B_DLR_EMPTY));
+            ++ci;
+            if (!w.whole) {
+                // ---- shared tile: publish the partial, the last CTA to arrive finishes it ----
+                ++partial_idx;
+                const long long first_unit = (long long)w.tile * p.KB;
+                const int c_first = unit_owner(p.units, first_unit, G);
+                const int c_last = unit_owner(p.units, first_unit + p.KB - 1, G);
+                __threadfence();
+                named_bar_sync(1, 128);
+                if (et == 0) {
+                    int old = atomicAdd(p.counters + w.tile, 1);
+                    *last_flag = (old == c_last - c_first) ? 1 : 0;
+                }
+                named_bar_sync(1, 128);
+                const bool last = *last_flag != 0;
+                named_bar_sync(1, 128);           // everyone has read the flag before it is reused
+                if (last) {
+                    __threadfence();
+                    if (et == 0) p.counters[w.tile] = 0;   // ready for the next launch
+#pragma unroll 1
+                    for (int col = 0; col < BT; ++col) {
+                        const int tok = w.tt * BT + col;
+                        if (tok >= p.M) break;
+                        int sum = 0;
+                        for (int c = c_first; c <= c_last; ++c) {
+                            // CTA c's items in order: a tile cut off at the start of its range
+                            // (slot 0), whole tiles, a tile cut off at the end of its range.
+                            const long long bc = range_begin(p.units, c, G);
+                            const int slot = (bc >= first_unit) ? 0 : ((bc % p.KB != 0) ? 1 : 0);
+                            const int32_t* src = p.part_int + ((size_t)c * 2 + slot) * (BT * 128);
+                            sum += __ldcg(src + col * 128 + nl);
+                        }
+                        if (n_ok) {
+                            const int acc = sum >> 4;
+                            float y = (float)acc * __ldg(p.a_scale + tok) * ws;
+                            if (p.r > 0) y += __ldcg(p.part_lr + (size_t)c_first * (BT * 128) + col * 128 + nl);
+                            p.Y[(size_t)tok * p.N + n] = __float2half_rn(y);
+                            if (p.acc_debug) p.acc_debug[(size_t)tok * p.N + n] = acc;
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    // =================== teardown ===================
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
+                     ::"r"(tmem), "r"((uint32_t)C::TmemCols)
+                     : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (fn) return fn;
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || ptr == nullptr) return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    return fn;
+}
+
+// 2-D row-major tensor [rows, cols] of `esize`-byte elements, box = [box_rows, box_cols],
+// 128-byte swizzle, out-of-range elements read as zero.
+int make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, int esize, const void* base,
+                uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t box_cols) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return record_cuda_error(cudaErrorUnknown, "cuTensorMapEncodeTiled unavailable");
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * (uint64_t)esize};
+    cuuint32_t box[2] = {box_cols, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return record_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+    return ASER_OK;
+}
+
+int pick_bt(int M) { return M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128; }
+
+struct Layout {
+    int BT, NT, TT, KB;
+    long long units;
+    size_t off_counters, off_part_int, off_part_lr, total;
+};
+
+Layout make_layout(int M, int N, int K, int r) {
+    Layout L;
+    L.BT = pick_bt(M);
+    L.NT = (N + 127) / 128;
+    L.TT = (M + L.BT - 1) / L.BT;
+    L.KB = K / 128;
+    L.units = (long long)L.NT * L.TT * L.KB;
+    size_t tiles = (size_t)L.NT * L.TT;
+    L.off_counters = kWsHeaderBytes;
+    L.off_part_int = L.off_counters + ((tiles * 4 + 255) / 256) * 256;
+    L.off_part_lr = L.off_part_int + (size_t)kMaxCtas * 2 * L.BT * 128 * 4;
+    L.total = L.off_part_lr + (r > 0 ? (size_t)kMaxCtas * L.BT * 128 * 4 : 0);
+    return L;
+}
+
+template <int BT>
+int launch_bt(const CUtensorMap& mx, const CUtensorMap& mlb, const CUtensorMap& mt, const Params& p,
+              int grid, cudaStream_t st) {
+    using C = Cfg<BT>;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(linear_tc_kernel<BT>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, C::SmemBytes);
+        if (e != cudaSuccess) return record_cuda_error(e, "linear_tc smem attribute");
+        configured = true;
+    }
+    linear_tc_kernel<BT><<<grid, kThreads, C::SmemBytes, st>>>(mx, mlb, mt, p);
+    return check_launch("linear_tc_kernel");
+}
+
+}  // namespace
+
+size_t linear_tc_workspace_bytes(int M, int N, int K, int r) {
+    if (M <= 0 || N <= 0) return 0;
+    return make_layout(M, N, K, r).total - kWsHeaderBytes;
+}
+
+int launch_linear_tc(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
+                     const float* w_scale, const __nv_bfloat16* T, const __half* LB,
+                     int M, int N, int K, int r, __half* Y, int32_t* acc_debug,
+                     void* workspace, size_t workspace_bytes, cudaStream_t st) {
+    Layout L = make_layout(M, N, K, r);
+    if (workspace_bytes < L.total) return ASER_ERR_WORKSPACE;
+
+    static int num_sms = 0;
+    if (num_sms == 0) {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) { num_sms = 0; return record_cuda_error(e, "query SM count"); }
+    }
+    int grid = num_sms < kMaxCtas ? num_sms : kMaxCtas;
+    long long want = (L.units + 1) / 2;   // at least two units per CTA on tiny problems
+    if (want < 1) want = 1;
+    if (grid > want) grid = (int)want;
+
+    CUtensorMap mx, mlb, mt;
+    int rc = make_map_2d(&mx, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Xq, M, K, L.BT, 128);
+    if (rc != ASER_OK) return rc;
+    if (r > 0) {
+        rc = make_map_2d(&mlb, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, LB, N, r, 128, 64);
+        if (rc != ASER_OK) return rc;
+        rc = make_map_2d(&mt, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, T, M, r, L.BT, 64);
+        if (rc != ASER_OK) return rc;
+    } else {
+        mlb = mx;
+        mt = mx;
+    }
+
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    Params p;
+    p.Wk = Wk; p.a_scale = a_scale; p.w_scale = w_scale; p.Y = Y; p.acc_debug = acc_debug;
+    p.status = reinterpret_cast<uint32_t*>(ws);
+    p.counters = reinterpret_cast<int*>(ws + L.off_counters);
+    p.part_int = reinterpret_cast<int32_t*>(ws + L.off_part_int);
+    p.part_lr = reinterpret_cast<float*>(ws + L.off_part_lr);
+    p.M = M; p.N = N; p.K = K; p.r = r;
+    p.KB = L.KB; p.TT = L.TT; p.NT = L.NT; p.units = L.units;
+
+    switch (L.BT) {
+        case 16: return launch_bt<16>(mx, mlb, mt, p, grid, st);
+        case 32: return launch_bt<32>(mx, mlb, mt, p, grid, st);
+        case 64: return launch_bt<64>(mx, mlb, mt, p, grid, st);
+        default: return launch_bt<128>(mx, mlb, mt, p, grid, st);
+    }
+}
+
+}  // namespace aser

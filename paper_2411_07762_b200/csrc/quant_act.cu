@@ -306,9 +306,13 @@ template <int MAXT>
 int launch_large(const __half* X, const float* s, const __half* LA, int M, int K, int r,
                  int8_t* Xq, float* a_scale, __nv_bfloat16* T, cudaStream_t st) {
     size_t smem = 2 * (size_t)(kTileM + r) * kRowBytes;
-    cudaError_t e = cudaFuncSetAttribute(quant_act_large_kernel<MAXT>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return record_cuda_error(e, "quant_act_large smem attribute");
+    static size_t configured = 0;   // largest dynamic shared memory size opted into so far
+    if (smem > configured) {
+        cudaError_t e = cudaFuncSetAttribute(quant_act_large_kernel<MAXT>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return record_cuda_error(e, "quant_act_large smem attribute");
+        configured = smem;
+    }
     int grid = (M + kTileM - 1) / kTileM;
     quant_act_large_kernel<MAXT><<<grid, kLargeThreads, smem, st>>>(X, s, LA, M, K, r, Xq, a_scale, T);
     return check_launch("quant_act_large_kernel");
@@ -321,10 +325,12 @@ int launch_quant_act(const __half* X, const float* s, const __half* LA, int M, i
     if (M == 0) return ASER_OK;
     if (M <= 32) {
         size_t smem = (size_t)K * sizeof(float);
-        if (smem > 48 * 1024) {
+        static size_t configured = 48 * 1024;
+        if (smem > configured) {
             cudaError_t e = cudaFuncSetAttribute(quant_act_small_kernel,
                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return record_cuda_error(e, "quant_act_small smem attribute");
+            configured = smem;
         }
         dim3 grid(1 + (r + kRowsPerCta - 1) / kRowsPerCta, M);
         quant_act_small_kernel<<<grid, kSmallThreads, smem, st>>>(X, s, LA, M, K, r, Xq, a_scale, T);

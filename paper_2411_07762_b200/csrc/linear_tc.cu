@@ -28,7 +28,7 @@ constexpr int kASlots = 4;        // A-operand slots in tensor memory (32 column
 constexpr int kLrSlots = 2;       // ring of low-rank chunks (64 columns of r each)
 constexpr int kMaxCtas = 160;     // upper bound on the persistent grid (workspace sizing)
 constexpr uint32_t kStatusTimeout = 1u;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
+constexpr long long kWaitLimitClocks = 4000000000ll;  // about 2 s of SM clocks per wait
 
 template <int BT>
 struct Cfg {
@@ -75,10 +75,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ unsigned long long global_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
+// Non-blocking probe of a barrier phase (used where one thread polls several barriers).
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
 }
 __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes,
                                               uint32_t bar) {
@@ -210,7 +217,7 @@ struct Params {
     float* part_lr;        // [grid][BT][128]
     int M, N, K, r;
     int KB, TT, NT;        // 128-column blocks, token tiles, 128-row tiles
-    long long units;       // NT * TT * KB
+    int units;             // NT * TT * KB
 };
 
 struct Work {
@@ -218,25 +225,44 @@ struct Work {
     bool has_lr, whole;
 };
 
-__device__ __forceinline__ long long range_begin(long long units, int c, int G) {
-    return units * c / G;
+// Units are numbered tile-major: unit = tile * KB + column block.  CTA c owns
+// [range_begin(c), range_begin(c + 1)).  The unit count fits 31 bits (checked on the host).
+__device__ __forceinline__ int range_begin(int units, int c, int G) {
+    return (int)((long long)units * c / G);
 }
 // CTA that owns unit x.
-__device__ __forceinline__ int unit_owner(long long units, long long x, int G) {
-    return (int)(((x + 1) * G - 1) / units);
+__device__ __forceinline__ int unit_owner(int units, int x, int G) {
+    return (int)((((long long)x + 1) * G - 1) / units);
 }
 
-__device__ __forceinline__ bool next_work(long long& u, long long u1, const Params& p, Work& w) {
-    if (u >= u1) return false;
-    w.tile = (int)(u / p.KB);
-    w.kb0 = (int)(u % p.KB);
-    long long left = u1 - u;
-    w.kb1 = (int)((long long)(p.KB - w.kb0) < left ? p.KB : w.kb0 + left);
-    w.nt = w.tile / p.TT;
-    w.tt = w.tile % p.TT;
+// Cursor over a CTA's unit range; one division when it is created, none afterwards.
+struct Cursor {
+    int u, u_end, tile, nt, tt, kb;
+    __device__ __forceinline__ void init(int begin, int end, const Params& p) {
+        u = begin; u_end = end;
+        tile = begin / p.KB; kb = begin - tile * p.KB;
+        nt = tile / p.TT; tt = tile - nt * p.TT;
+    }
+    __device__ __forceinline__ bool done() const { return u >= u_end; }
+    // advance by n column blocks that stay inside the current tile
+    __device__ __forceinline__ void advance(int n, const Params& p) {
+        u += n; kb += n;
+        if (kb >= p.KB) {
+            kb = 0; ++tile;
+            if (++tt == p.TT) { tt = 0; ++nt; }
+        }
+    }
+};
+
+// Next work item (the part of one tile inside this CTA's range).
+__device__ __forceinline__ bool next_work(Cursor& c, const Params& p, Work& w) {
+    if (c.done()) return false;
+    w.tile = c.tile; w.nt = c.nt; w.tt = c.tt; w.kb0 = c.kb;
+    const int left = c.u_end - c.u;
+    w.kb1 = (p.KB - c.kb <= left) ? p.KB : c.kb + left;
     w.has_lr = (w.kb0 == 0) && p.r > 0;
     w.whole = (w.kb0 == 0) && (w.kb1 == p.KB);
-    u += w.kb1 - w.kb0;
+    c.advance(w.kb1 - w.kb0, p);
     return true;
 }
 
@@ -248,13 +274,14 @@ struct Abort {
 // Bounded wait on an mbarrier phase.  Returns false after the time limit or when another role
 // of this CTA has already given up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const Abort& ab) {
-    if (mbar_try_wait(bar, parity)) return true;
-    unsigned long long t0 = global_ns();
     uint32_t spins = 0;
+    long long t0 = 0;
     while (!mbar_try_wait(bar, parity)) {
-        if ((++spins & 63u) == 0) {
+        if ((++spins & 255u) == 0) {
             if (*ab.flag) return false;
-            if (global_ns() - t0 > kWaitLimitNs) {
+            if (t0 == 0) {
+                t0 = clock64();
+            } else if (clock64() - t0 > kWaitLimitClocks) {
                 *ab.flag = 1;
                 atomicOr(ab.status, kStatusTimeout);
                 return false;
@@ -293,7 +320,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = gridDim.x, cta = blockIdx.x;
-    const long long u_begin = range_begin(p.units, cta, G), u_end = range_begin(p.units, cta + 1, G);
+    const int u_begin = range_begin(p.units, cta, G), u_end = range_begin(p.units, cta + 1, G);
     Abort ab{abort_flag, p.status};
 
     if (threadIdx.x == 0) {
@@ -327,49 +354,48 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     if (warp == 0) {
         // =================== copy producer (one lane, three rings) ===================
         if (lane == 0) {
-            long long uw = u_begin, ux = u_begin, ul = u_begin;   // cursors
+            Cursor cw_, cx_, cl_;                                // one cursor per ring
+            cw_.init(u_begin, u_end, p); cx_.init(u_begin, u_end, p); cl_.init(u_begin, u_end, p);
             uint32_t cw = 0, cx = 0, cl = 0;                     // items issued per ring
             Work wl{};                                           // current low-rank work item
             int lc = 0;                                          // next chunk of wl
             bool have_wl = false;
             auto advance_lr = [&]() {
                 have_wl = false;
-                while (p.r > 0 && next_work(ul, u_end, p, wl)) {
+                while (p.r > 0 && next_work(cl_, p, wl)) {
                     if (wl.has_lr) { have_wl = true; lc = 0; break; }
                 }
             };
             advance_lr();
-            unsigned long long t0 = global_ns();
+            long long t0 = 0;
             uint32_t idle = 0;
             bool failed = false;
-            while (uw < u_end || ux < u_end || have_wl) {
+            while (!cw_.done() || !cx_.done() || have_wl) {
                 bool progressed = false;
-                if (uw < u_end) {
+                if (!cw_.done()) {
                     int s = cw % C::NW;
-                    if (mbar_try_wait(bar(B_EMPTY_W + s), ((cw / C::NW) & 1) ^ 1)) {
+                    if (mbar_test_wait(bar(B_EMPTY_W + s), ((cw / C::NW) & 1) ^ 1)) {
                         // units are stored in the order they are consumed: block index == unit's
                         // (row tile, column block) with tiles of one row tile adjacent in tt
-                        int tile = (int)(uw / p.KB), kb = (int)(uw % p.KB), nt = tile / p.TT;
                         mbar_arrive_expect_tx(bar(B_FULL_W + s), kWkBlockBytes);
                         bulk_copy_g2s(sbase + C::OffW + s * kWkBlockBytes,
-                                      p.Wk + ((size_t)nt * p.KB + kb) * kWkBlockBytes, kWkBlockBytes,
+                                      p.Wk + ((size_t)cw_.nt * p.KB + cw_.kb) * kWkBlockBytes, kWkBlockBytes,
                                       bar(B_FULL_W + s));
-                        ++cw; ++uw; progressed = true;
+                        ++cw; cw_.advance(1, p); progressed = true;
                     }
                 }
-                if (ux < u_end) {
+                if (!cx_.done()) {
                     int s = cx % C::NX;
-                    if (mbar_try_wait(bar(B_EMPTY_X + s), ((cx / C::NX) & 1) ^ 1)) {
-                        int tile = (int)(ux / p.KB), kb = (int)(ux % p.KB), tt = tile % p.TT;
+                    if (mbar_test_wait(bar(B_EMPTY_X + s), ((cx / C::NX) & 1) ^ 1)) {
                         mbar_arrive_expect_tx(bar(B_FULL_X + s), C::XBytes);
-                        tma_load_2d(sbase + C::OffX + s * C::XBytes, &map_x, kb * 128, tt * BT,
+                        tma_load_2d(sbase + C::OffX + s * C::XBytes, &map_x, cx_.kb * 128, cx_.tt * BT,
                                     bar(B_FULL_X + s));
-                        ++cx; ++ux; progressed = true;
+                        ++cx; cx_.advance(1, p); progressed = true;
                     }
                 }
                 if (have_wl) {
                     int s = cl % kLrSlots;
-                    if (mbar_try_wait(bar(B_EMPTY_LR + s), ((cl / kLrSlots) & 1) ^ 1)) {
+                    if (mbar_test_wait(bar(B_EMPTY_LR + s), ((cl / kLrSlots) & 1) ^ 1)) {
                         mbar_arrive_expect_tx(bar(B_FULL_LR + s), C::LbBytes + C::TBytes);
                         tma_load_2d(sbase + C::OffLb + s * C::LbBytes, &map_lb, lc * 64, wl.nt * 128,
                                     bar(B_FULL_LR + s));
@@ -380,10 +406,10 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     }
                 }
                 if (progressed) { idle = 0; continue; }
-                if (idle == 0) t0 = global_ns();
-                if ((++idle & 63u) == 0) {
+                if (idle == 0) t0 = clock64();
+                if ((++idle & 1023u) == 0) {
                     if (*abort_flag) { failed = true; break; }
-                    if (global_ns() - t0 > kWaitLimitNs) {
+                    if (clock64() - t0 > kWaitLimitClocks) {
                         *abort_flag = 1;
                         atomicOr(p.status, kStatusTimeout);
                         failed = true;
@@ -406,11 +432,12 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         if (lane == 0) {
             constexpr uint32_t idesc_i8 = make_idesc(2, 1, 128, BT);
             constexpr uint32_t idesc_f16 = make_idesc(1, 0, 128, BT);
-            long long u = u_begin;
+            Cursor cur;
+            cur.init(u_begin, u_end, p);
             Work w;
             uint32_t cx = 0, ca = 0, cl = 0, ci = 0, clr_items = 0;
             bool ok = true;
-            while (ok && next_work(u, u_end, p, w)) {
+            while (ok && next_work(cur, p, w)) {
                 const int buf = ci & 1;
                 const uint32_t d_int = tm_dint0 + buf * BT;
                 ok = mbar_wait(bar(B_ACC_EMPTY + buf), ((ci >> 1) & 1) ^ 1, ab);
@@ -459,11 +486,12 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         const int q = warp & 3;                    // TMEM lane quarter this warp may touch
         const int row = q * 32 + lane;             // weight row inside the 128-row tile
         const int t128 = (warp - 2) * 32 + lane;   // 0..127 among the unpack threads
-        long long u = u_begin;
+        Cursor cur;
+        cur.init(u_begin, u_end, p);
         Work w;
         uint32_t cw = 0, ca = 0, cl = 0;
         bool ok = true;
-        while (ok && next_work(u, u_end, p, w)) {
+        while (ok && next_work(cur, p, w)) {
             for (int kb = w.kb0; kb < w.kb1 && ok; ++kb) {
                 const int sw = cw % C::NW, sa = ca % kASlots;
                 ok = mbar_wait(bar(B_FULL_W + sw), (cw / C::NW) & 1, ab);
@@ -521,12 +549,13 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         const int nl = q * 32 + lane;              // row of D = output channel inside the tile
         const int et = (warp - 6) * 32 + lane;     // 0..127 among the epilogue threads
         const uint32_t lane_sel = (uint32_t)(q * 32) << 16;
-        long long u = u_begin;
+        Cursor cur;
+        cur.init(u_begin, u_end, p);
         Work w;
         uint32_t ci = 0;
         int partial_idx = 0;                       // 0: first partial item of this CTA, 1: second
         bool ok = true;
-        while (ok && next_work(u, u_end, p, w)) {
+        while (ok && next_work(cur, p, w)) {
             const int buf = ci & 1;
             ok = mbar_wait(bar(B_ACC_FULL + buf), (ci >> 1) & 1, ab);
             ok = named_bar_all(1, 128, ok);   // the 128 epilogue threads go on or give up together
@@ -572,7 +601,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             if (!w.whole) {
                 // ---- shared tile: publish the partial, the last CTA to arrive finishes it ----
                 ++partial_idx;
-                const long long first_unit = (long long)w.tile * p.KB;
+                const int first_unit = w.tile * p.KB;
                 const int c_first = unit_owner(p.units, first_unit, G);
                 const int c_last = unit_owner(p.units, first_unit + p.KB - 1, G);
                 __threadfence();
@@ -588,24 +617,31 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     __threadfence();
                     if (et == 0) p.counters[w.tile] = 0;   // ready for the next launch
 #pragma unroll 1
-                    for (int col = 0; col < BT; ++col) {
-                        const int tok = w.tt * BT + col;
-                        if (tok >= p.M) break;
-                        int sum = 0;
+                    for (int c0 = 0; c0 < BT; c0 += 16) {
+                        if (w.tt * BT + c0 >= p.M) break;
+                        int sum[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) sum[j] = 0;
                         for (int c = c_first; c <= c_last; ++c) {
                             // CTA c's items in order: a tile cut off at the start of its range
                             // (slot 0), whole tiles, a tile cut off at the end of its range.
-                            const long long bc = range_begin(p.units, c, G);
+                            const int bc = range_begin(p.units, c, G);
                             const int slot = (bc >= first_unit) ? 0 : ((bc % p.KB != 0) ? 1 : 0);
-                            const int32_t* src = p.part_int + ((size_t)c * 2 + slot) * (BT * 128);
-                            sum += __ldcg(src + col * 128 + nl);
+                            const int32_t* src = p.part_int + ((size_t)c * 2 + slot) * (BT * 128) + c0 * 128 + nl;
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) sum[j] += __ldcg(src + j * 128);
                         }
-                        if (n_ok) {
-                            const int acc = sum >> 4;
-                            float y = (float)acc * __ldg(p.a_scale + tok) * ws;
-                            if (p.r > 0) y += __ldcg(p.part_lr + (size_t)c_first * (BT * 128) + col * 128 + nl);
-                            p.Y[(size_t)tok * p.N + n] = __float2half_rn(y);
-                            if (p.acc_debug) p.acc_debug[(size_t)tok * p.N + n] = acc;
+                        const float* lsrc = p.part_lr + (size_t)c_first * (BT * 128) + c0 * 128 + nl;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const int tok = w.tt * BT + c0 + j;
+                            if (tok < p.M && n_ok) {
+                                const int acc = sum[j] >> 4;
+                                float y = (float)acc * __ldg(p.a_scale + tok) * ws;
+                                if (p.r > 0) y += __ldcg(lsrc + j * 128);
+                                p.Y[(size_t)tok * p.N + n] = __float2half_rn(y);
+                                if (p.acc_debug) p.acc_debug[(size_t)tok * p.N + n] = acc;
+                            }
                         }
                     }
                 }
@@ -664,7 +700,7 @@ int pick_bt(int M) { return M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128; }
 
 struct Layout {
     int BT, NT, TT, KB;
-    long long units;
+    long long units;   // must stay below 2^31
     size_t off_counters, off_part_int, off_part_lr, total;
 };
 
@@ -711,6 +747,7 @@ int launch_linear_tc(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
                      void* workspace, size_t workspace_bytes, cudaStream_t st) {
     Layout L = make_layout(M, N, K, r);
     if (workspace_bytes < L.total) return ASER_ERR_WORKSPACE;
+    if (L.units >= (1ll << 31) / kMaxCtas * kMaxCtas) return ASER_ERR_SHAPE;
 
     static int num_sms = 0;
     if (num_sms == 0) {
@@ -745,7 +782,7 @@ int launch_linear_tc(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
     p.part_int = reinterpret_cast<int32_t*>(ws + L.off_part_int);
     p.part_lr = reinterpret_cast<float*>(ws + L.off_part_lr);
     p.M = M; p.N = N; p.K = K; p.r = r;
-    p.KB = L.KB; p.TT = L.TT; p.NT = L.NT; p.units = L.units;
+    p.KB = L.KB; p.TT = L.TT; p.NT = L.NT; p.units = (int)L.units;
 
     switch (L.BT) {
         case 16: return launch_bt<16>(mx, mlb, mt, p, grid, st);

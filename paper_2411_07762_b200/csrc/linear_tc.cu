@@ -24,7 +24,6 @@ namespace aser {
 namespace {
 
 constexpr int kThreads = 320;
-constexpr int kASlots = 4;        // A-operand slots in tensor memory (32 columns each)
 constexpr int kLrSlots = 2;       // ring of low-rank chunks (64 columns of r each)
 constexpr int kMaxCtas = 160;     // upper bound on the persistent grid (workspace sizing)
 constexpr uint32_t kStatusTimeout = 1u;
@@ -32,6 +31,8 @@ constexpr long long kWaitLimitClocks = 4000000000ll;  // about 2 s of SM clocks 
 
 template <int BT>
 struct Cfg {
+    // A-operand slots in tensor memory (32 columns each): whatever 512 columns leave free
+    static constexpr int NA = (BT == 128) ? 4 : (BT == 64 ? 8 : 12);
     static constexpr int NW = (BT == 128) ? 8 : 12;   // weight ring (8 KiB each)
     static constexpr int NX = (BT == 128) ? 4 : 8;    // activation ring (BT x 128 B each)
     static constexpr int XBytes = BT * 128;
@@ -42,9 +43,9 @@ struct Cfg {
     static constexpr int OffLb = OffX + NX * XBytes;
     static constexpr int OffT = OffLb + kLrSlots * LbBytes;
     static constexpr int OffBar = OffT + kLrSlots * TBytes;
-    static constexpr int NumBars = 2 * NW + 2 * NX + 2 * kASlots + 3 * kLrSlots + 2 + 2 + 1;
+    static constexpr int NumBars = 2 * NW + 2 * NX + 2 * NA + 3 * kLrSlots + 2 + 2 + 1;
     static constexpr int SmemBytes = OffBar + NumBars * 8 + 64 + 1024;  // + slack for 1 KiB alignment
-    static constexpr int TmemColsUsed = 3 * BT + kASlots * 32;
+    static constexpr int TmemColsUsed = 3 * BT + NA * 32;
     static constexpr int TmemCols = TmemColsUsed <= 256 ? 256 : 512;
 };
 
@@ -291,6 +292,14 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const A
     return true;
 }
 
+// Warp-collective form: lane 0 polls, the result is broadcast (which also re-converges the
+// warp).  Keeps 31 of 32 lanes off the barrier unit, which every other role's waits share.
+__device__ __forceinline__ bool warp_mbar_wait(uint32_t bar, uint32_t parity, const Abort& ab, int lane) {
+    int ok = 1;
+    if (lane == 0) ok = mbar_wait(bar, parity, ab) ? 1 : 0;
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+
 // ---------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------
@@ -308,7 +317,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     // barrier indices
     constexpr int B_FULL_W = 0, B_EMPTY_W = B_FULL_W + C::NW, B_FULL_X = B_EMPTY_W + C::NW,
                   B_EMPTY_X = B_FULL_X + C::NX, B_A_FULL = B_EMPTY_X + C::NX,
-                  B_A_EMPTY = B_A_FULL + kASlots, B_FULL_LR = B_A_EMPTY + kASlots,
+                  B_A_EMPTY = B_A_FULL + C::NA, B_FULL_LR = B_A_EMPTY + C::NA,
                   B_CONV_LR = B_FULL_LR + kLrSlots, B_EMPTY_LR = B_CONV_LR + kLrSlots,
                   B_ACC_FULL = B_EMPTY_LR + kLrSlots, B_ACC_EMPTY = B_ACC_FULL + 2,
                   B_DLR_EMPTY = B_ACC_EMPTY + 2;
@@ -324,14 +333,14 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     Abort ab{abort_flag, p.status};
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < C::NW; ++i) { mbar_init(bar(B_FULL_W + i), 1); mbar_init(bar(B_EMPTY_W + i), 128); }
+        for (int i = 0; i < C::NW; ++i) { mbar_init(bar(B_FULL_W + i), 1); mbar_init(bar(B_EMPTY_W + i), 4); }
         for (int i = 0; i < C::NX; ++i) { mbar_init(bar(B_FULL_X + i), 1); mbar_init(bar(B_EMPTY_X + i), 1); }
-        for (int i = 0; i < kASlots; ++i) { mbar_init(bar(B_A_FULL + i), 128); mbar_init(bar(B_A_EMPTY + i), 1); }
+        for (int i = 0; i < C::NA; ++i) { mbar_init(bar(B_A_FULL + i), 4); mbar_init(bar(B_A_EMPTY + i), 1); }
         for (int i = 0; i < kLrSlots; ++i) {
-            mbar_init(bar(B_FULL_LR + i), 1); mbar_init(bar(B_CONV_LR + i), 128); mbar_init(bar(B_EMPTY_LR + i), 1);
+            mbar_init(bar(B_FULL_LR + i), 1); mbar_init(bar(B_CONV_LR + i), 4); mbar_init(bar(B_EMPTY_LR + i), 1);
         }
-        for (int i = 0; i < 2; ++i) { mbar_init(bar(B_ACC_FULL + i), 1); mbar_init(bar(B_ACC_EMPTY + i), 128); }
-        mbar_init(bar(B_DLR_EMPTY), 128);
+        for (int i = 0; i < 2; ++i) { mbar_init(bar(B_ACC_FULL + i), 1); mbar_init(bar(B_ACC_EMPTY + i), 4); }
+        mbar_init(bar(B_DLR_EMPTY), 4);
         *abort_flag = 0;
         *last_flag = 0;
         *never_flag = 0;
@@ -444,9 +453,9 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 if (!ok) break;
                 tc_fence_after();
                 for (int kb = w.kb0; kb < w.kb1 && ok; ++kb) {
-                    const int sx = cx % C::NX, sa = ca % kASlots;
+                    const int sx = cx % C::NX, sa = ca % C::NA;
                     ok = mbar_wait(bar(B_FULL_X + sx), (cx / C::NX) & 1, ab) &&
-                         mbar_wait(bar(B_A_FULL + sa), (ca / kASlots) & 1, ab);
+                         mbar_wait(bar(B_A_FULL + sa), (ca / C::NA) & 1, ab);
                     if (!ok) break;
                     tc_fence_after();
                     const uint64_t xdesc = smem_desc_sw128(sbase + C::OffX + sx * C::XBytes);
@@ -493,8 +502,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         bool ok = true;
         while (ok && next_work(cur, p, w)) {
             for (int kb = w.kb0; kb < w.kb1 && ok; ++kb) {
-                const int sw = cw % C::NW, sa = ca % kASlots;
-                ok = mbar_wait(bar(B_FULL_W + sw), (cw / C::NW) & 1, ab);
+                const int sw = cw % C::NW, sa = ca % C::NA;
+                ok = warp_mbar_wait(bar(B_FULL_W + sw), (cw / C::NW) & 1, ab, lane);
                 if (!ok) break;
                 const uint8_t* wsrc = smem + C::OffW + sw * kWkBlockBytes + row * 16;
                 uint32_t v[32];
@@ -508,20 +517,22 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                         v[sub * 8 + 2 * i + 1] = xs[i] & 0xF0F0F0F0u;      // columns c0+4 .. c0+7
                     }
                 }
-                mbar_arrive(bar(B_EMPTY_W + sw));   // values are in registers: slot may be refilled
-                ok = mbar_wait(bar(B_A_EMPTY + sa), ((ca / kASlots) & 1) ^ 1, ab);
+                __syncwarp();                       // every lane holds its values in registers:
+                if (lane == 0) mbar_arrive(bar(B_EMPTY_W + sw));   // the slot may be refilled
+                ok = warp_mbar_wait(bar(B_A_EMPTY + sa), ((ca / C::NA) & 1) ^ 1, ab, lane);
                 if (!ok) break;
                 tc_fence_after();
                 tmem_st32(tm_a0 + sa * 32 + ((uint32_t)(q * 32) << 16), v);
                 tmem_wait_st();
                 tc_fence_before();
-                mbar_arrive(bar(B_A_FULL + sa));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(B_A_FULL + sa));
                 ++cw; ++ca;
             }
             if (ok && w.has_lr) {
                 for (int c = 0; c < lr_chunks && ok; ++c) {
                     const int s = cl % kLrSlots;
-                    ok = mbar_wait(bar(B_FULL_LR + s), (cl / kLrSlots) & 1, ab);
+                    ok = warp_mbar_wait(bar(B_FULL_LR + s), (cl / kLrSlots) & 1, ab, lane);
                     if (!ok) break;
                     // T chunk: bf16 -> fp16 in place (same element size, same swizzled position)
                     uint8_t* tb = smem + C::OffT + s * C::TBytes;
@@ -538,7 +549,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                         *reinterpret_cast<uint4*>(tb + i * 16) = make_uint4(out[0], out[1], out[2], out[3]);
                     }
                     fence_proxy_async_smem();
-                    mbar_arrive(bar(B_CONV_LR + s));
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(B_CONV_LR + s));
                     ++cl;
                 }
             }
@@ -557,7 +569,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         bool ok = true;
         while (ok && next_work(cur, p, w)) {
             const int buf = ci & 1;
-            ok = mbar_wait(bar(B_ACC_FULL + buf), (ci >> 1) & 1, ab);
+            ok = warp_mbar_wait(bar(B_ACC_FULL + buf), (ci >> 1) & 1, ab, lane);
             ok = named_bar_all(1, 128, ok);   // the 128 epilogue threads go on or give up together
             if (!ok) break;
             tc_fence_after();
@@ -595,8 +607,11 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 }
             }
             tc_fence_before();
-            mbar_arrive(bar(B_ACC_EMPTY + buf));
-            if (w.has_lr) mbar_arrive(bar(B_DLR_EMPTY));
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(bar(B_ACC_EMPTY + buf));
+                if (w.has_lr) mbar_arrive(bar(B_DLR_EMPTY));
+            }
             ++ci;
             if (!w.whole) {
                 // ---- shared tile: publish the partial, the last CTA to arrive finishes it ----

@@ -12,8 +12,9 @@
 // units is cut into equal contiguous ranges, one per CTA; tiles shared by several CTAs are
 // summed through the workspace by whichever CTA arrives last.
 //
-// Warp roles (320 threads): 0 = copy producer, 1 = MMA issuer (+ TMEM owner),
-// 2..5 = int4 -> int8 unpack into TMEM (+ T conversion), 6..9 = epilogue.
+// Warp roles (352 threads): 0 = weight producer, 1 = MMA issuer (+ TMEM owner),
+// 2..5 = int4 -> int8 unpack into TMEM (+ T conversion), 6..9 = epilogue,
+// 10 = activation and low-rank operand producer.
 // Every wait is bounded: on expiry the CTA sets the status word and winds down.
 #include <cuda.h>
 
@@ -23,30 +24,38 @@ namespace aser {
 
 namespace {
 
-constexpr int kThreads = 320;
+constexpr int kThreads = 352;
 constexpr int kLrSlots = 2;       // ring of low-rank chunks (64 columns of r each)
 constexpr int kMaxCtas = 160;     // upper bound on the persistent grid (workspace sizing)
 constexpr uint32_t kStatusTimeout = 1u;
 constexpr long long kWaitLimitClocks = 4000000000ll;  // about 2 s of SM clocks per wait
 
+// Per token-tile configuration.  A pipeline stage carries KS 128-column blocks: one bulk copy of
+// KS x 8 KiB of packed weights, one TMA box of KS activation tiles, KS x 32 tensor-memory columns
+// of unpacked A operand.  Large stages keep the per-byte count of copy issues, barrier waits and
+// commits low (each costs a single thread hundreds of cycles), which is what bounds decode shapes.
 template <int BT>
 struct Cfg {
-    // A-operand slots in tensor memory (32 columns each): whatever 512 columns leave free
-    static constexpr int NA = (BT == 128) ? 4 : (BT == 64 ? 8 : 12);
-    static constexpr int NW = (BT == 128) ? 8 : 12;   // weight ring (8 KiB each)
-    static constexpr int NX = (BT == 128) ? 4 : 8;    // activation ring (BT x 128 B each)
-    static constexpr int XBytes = BT * 128;
+    static constexpr int KS = (BT <= 32) ? 4 : (BT == 64 ? 2 : 1);
+    static constexpr int NW = (BT <= 32) ? 4 : (BT == 64 ? 5 : 8);     // weight ring depth
+    static constexpr int NA = (BT <= 32) ? 3 : 4;                       // activation / A-operand ring depth
+    static constexpr int WBytes = KS * kWkBlockBytes;
+    static constexpr int XTile = BT * 128;                              // one 128-column block of Xq
+    static constexpr int XBytes = KS * XTile;
     static constexpr int LbBytes = 128 * 128;          // 128 rows x 64 fp16
     static constexpr int TBytes = BT * 128;            // BT rows x 64 bf16/fp16
     static constexpr int OffW = 0;
-    static constexpr int OffX = OffW + NW * kWkBlockBytes;
-    static constexpr int OffLb = OffX + NX * XBytes;
+    static constexpr int OffX = OffW + NW * WBytes;
+    static constexpr int OffLb = OffX + NA * XBytes;
     static constexpr int OffT = OffLb + kLrSlots * LbBytes;
     static constexpr int OffBar = OffT + kLrSlots * TBytes;
-    static constexpr int NumBars = 2 * NW + 2 * NX + 2 * NA + 3 * kLrSlots + 2 + 2 + 1;
+    static constexpr int NumBars = 2 * NW + 2 * NA + 3 * kLrSlots + 2 + 2 + 1;
     static constexpr int SmemBytes = OffBar + NumBars * 8 + 64 + 1024;  // + slack for 1 KiB alignment
-    static constexpr int TmemColsUsed = 3 * BT + NA * 32;
+    static constexpr int ASlotCols = KS * 32;
+    static constexpr int TmemColsUsed = 3 * BT + NA * ASlotCols;
     static constexpr int TmemCols = TmemColsUsed <= 256 ? 256 : 512;
+    static_assert(TmemColsUsed <= 512, "tensor memory budget");
+    static_assert(SmemBytes <= 227 * 1024, "shared memory budget");
 };
 
 // ---------------------------------------------------------------------------
@@ -76,18 +85,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Non-blocking probe of a barrier phase (used where one thread polls several barriers).
-__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
 __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes,
                                               uint32_t bar) {
     asm volatile(
@@ -101,6 +98,14 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
         "[%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z,
+                                            uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
         : "memory");
 }
 __device__ __forceinline__ void fence_proxy_async_smem() {
@@ -308,6 +313,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_lb,
                  const __grid_constant__ CUtensorMap map_t, const Params p) {
     using C = Cfg<BT>;
+    constexpr int KS = C::KS;
     extern __shared__ uint8_t smem_raw[];
     // 1 KiB alignment for the swizzled tiles
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -315,9 +321,12 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     const uint32_t bar0 = sbase + C::OffBar;
     auto bar = [&](int i) { return bar0 + 8u * i; };
     // barrier indices
-    constexpr int B_FULL_W = 0, B_EMPTY_W = B_FULL_W + C::NW, B_FULL_X = B_EMPTY_W + C::NW,
-                  B_EMPTY_X = B_FULL_X + C::NX, B_A_FULL = B_EMPTY_X + C::NX,
-                  B_A_EMPTY = B_A_FULL + C::NA, B_FULL_LR = B_A_EMPTY + C::NA,
+    //   W_FULL[s]  weight bytes of stage landed (tx)          -> unpack warps
+    //   W_FREE[s]  unpack warps have the weights in registers -> weight producer
+    //   READY[a]   activation bytes landed (tx) AND A operand written to tensor memory -> MMA issuer
+    //   FREE[a]    MMAs of the stage retired (commit)         -> activation producer, unpack warps
+    constexpr int B_W_FULL = 0, B_W_FREE = B_W_FULL + C::NW, B_READY = B_W_FREE + C::NW,
+                  B_FREE = B_READY + C::NA, B_FULL_LR = B_FREE + C::NA,
                   B_CONV_LR = B_FULL_LR + kLrSlots, B_EMPTY_LR = B_CONV_LR + kLrSlots,
                   B_ACC_FULL = B_EMPTY_LR + kLrSlots, B_ACC_EMPTY = B_ACC_FULL + 2,
                   B_DLR_EMPTY = B_ACC_EMPTY + 2;
@@ -333,9 +342,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     Abort ab{abort_flag, p.status};
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < C::NW; ++i) { mbar_init(bar(B_FULL_W + i), 1); mbar_init(bar(B_EMPTY_W + i), 4); }
-        for (int i = 0; i < C::NX; ++i) { mbar_init(bar(B_FULL_X + i), 1); mbar_init(bar(B_EMPTY_X + i), 1); }
-        for (int i = 0; i < C::NA; ++i) { mbar_init(bar(B_A_FULL + i), 4); mbar_init(bar(B_A_EMPTY + i), 1); }
+        for (int i = 0; i < C::NW; ++i) { mbar_init(bar(B_W_FULL + i), 1); mbar_init(bar(B_W_FREE + i), 4); }
+        for (int i = 0; i < C::NA; ++i) { mbar_init(bar(B_READY + i), 5); mbar_init(bar(B_FREE + i), 1); }
         for (int i = 0; i < kLrSlots; ++i) {
             mbar_init(bar(B_FULL_LR + i), 1); mbar_init(bar(B_CONV_LR + i), 4); mbar_init(bar(B_EMPTY_LR + i), 1);
         }
@@ -361,79 +369,75 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     const int lr_chunks = (p.r + 63) / 64;
 
     if (warp == 0) {
-        // =================== copy producer (one lane, three rings) ===================
+        // =================== weight producer (one lane) ===================
         if (lane == 0) {
-            Cursor cw_, cx_, cl_;                                // one cursor per ring
-            cw_.init(u_begin, u_end, p); cx_.init(u_begin, u_end, p); cl_.init(u_begin, u_end, p);
-            uint32_t cw = 0, cx = 0, cl = 0;                     // items issued per ring
-            Work wl{};                                           // current low-rank work item
-            int lc = 0;                                          // next chunk of wl
-            bool have_wl = false;
-            auto advance_lr = [&]() {
-                have_wl = false;
-                while (p.r > 0 && next_work(cl_, p, wl)) {
-                    if (wl.has_lr) { have_wl = true; lc = 0; break; }
-                }
-            };
-            advance_lr();
-            long long t0 = 0;
-            uint32_t idle = 0;
-            bool failed = false;
-            while (!cw_.done() || !cx_.done() || have_wl) {
-                bool progressed = false;
-                if (!cw_.done()) {
-                    int s = cw % C::NW;
-                    if (mbar_test_wait(bar(B_EMPTY_W + s), ((cw / C::NW) & 1) ^ 1)) {
-                        // units are stored in the order they are consumed: block index == unit's
-                        // (row tile, column block) with tiles of one row tile adjacent in tt
-                        mbar_arrive_expect_tx(bar(B_FULL_W + s), kWkBlockBytes);
-                        bulk_copy_g2s(sbase + C::OffW + s * kWkBlockBytes,
-                                      p.Wk + ((size_t)cw_.nt * p.KB + cw_.kb) * kWkBlockBytes, kWkBlockBytes,
-                                      bar(B_FULL_W + s));
-                        ++cw; cw_.advance(1, p); progressed = true;
-                    }
-                }
-                if (!cx_.done()) {
-                    int s = cx % C::NX;
-                    if (mbar_test_wait(bar(B_EMPTY_X + s), ((cx / C::NX) & 1) ^ 1)) {
-                        mbar_arrive_expect_tx(bar(B_FULL_X + s), C::XBytes);
-                        tma_load_2d(sbase + C::OffX + s * C::XBytes, &map_x, cx_.kb * 128, cx_.tt * BT,
-                                    bar(B_FULL_X + s));
-                        ++cx; cx_.advance(1, p); progressed = true;
-                    }
-                }
-                if (have_wl) {
-                    int s = cl % kLrSlots;
-                    if (mbar_test_wait(bar(B_EMPTY_LR + s), ((cl / kLrSlots) & 1) ^ 1)) {
-                        mbar_arrive_expect_tx(bar(B_FULL_LR + s), C::LbBytes + C::TBytes);
-                        tma_load_2d(sbase + C::OffLb + s * C::LbBytes, &map_lb, lc * 64, wl.nt * 128,
-                                    bar(B_FULL_LR + s));
-                        tma_load_2d(sbase + C::OffT + s * C::TBytes, &map_t, lc * 64, wl.tt * BT,
-                                    bar(B_FULL_LR + s));
-                        ++cl; ++lc; progressed = true;
-                        if (lc == lr_chunks) advance_lr();
-                    }
-                }
-                if (progressed) { idle = 0; continue; }
-                if (idle == 0) t0 = clock64();
-                if ((++idle & 1023u) == 0) {
-                    if (*abort_flag) { failed = true; break; }
-                    if (clock64() - t0 > kWaitLimitClocks) {
-                        *abort_flag = 1;
-                        atomicOr(p.status, kStatusTimeout);
-                        failed = true;
-                        break;
-                    }
+            Cursor cur;
+            cur.init(u_begin, u_end, p);
+            Work w;
+            uint32_t cw = 0;
+            bool ok = true;
+            while (ok && next_work(cur, p, w)) {
+                for (int kb = w.kb0; kb < w.kb1; kb += KS) {
+                    const int nkb = (w.kb1 - kb < KS) ? (w.kb1 - kb) : KS;
+                    const int s = cw % C::NW;
+                    ok = mbar_wait(bar(B_W_FREE + s), ((cw / C::NW) & 1) ^ 1, ab);
+                    if (!ok) break;
+                    // the blocks of one row tile are adjacent in memory: one copy per stage
+                    mbar_arrive_expect_tx(bar(B_W_FULL + s), nkb * kWkBlockBytes);
+                    bulk_copy_g2s(sbase + C::OffW + s * C::WBytes,
+                                  p.Wk + ((size_t)w.nt * p.KB + kb) * kWkBlockBytes, nkb * kWkBlockBytes,
+                                  bar(B_W_FULL + s));
+                    ++cw;
                 }
             }
-            if (failed || *abort_flag) {
+            if (!ok || *abort_flag) {
                 // let copies already issued land before the CTA's shared memory goes away
                 for (uint32_t i = (cw > (uint32_t)C::NW ? cw - C::NW : 0); i < cw; ++i)
-                    mbar_wait(bar(B_FULL_W + i % C::NW), (i / C::NW) & 1, Abort{never_flag, p.status});
-                for (uint32_t i = (cx > (uint32_t)C::NX ? cx - C::NX : 0); i < cx; ++i)
-                    mbar_wait(bar(B_FULL_X + i % C::NX), (i / C::NX) & 1, Abort{never_flag, p.status});
+                    mbar_wait(bar(B_W_FULL + i % C::NW), (i / C::NW) & 1, Abort{never_flag, p.status});
+            }
+        }
+    } else if (warp == 10) {
+        // =================== activation + low-rank operand producer (one lane) ===================
+        if (lane == 0) {
+            Cursor cur;
+            cur.init(u_begin, u_end, p);
+            Work w{};
+            uint32_t ca = 0, cl = 0;
+            bool ok = true;
+            auto issue_lr = [&](int c) {
+                const int s = cl % kLrSlots;
+                if (!mbar_wait(bar(B_EMPTY_LR + s), ((cl / kLrSlots) & 1) ^ 1, ab)) return false;
+                mbar_arrive_expect_tx(bar(B_FULL_LR + s), C::LbBytes + C::TBytes);
+                tma_load_2d(sbase + C::OffLb + s * C::LbBytes, &map_lb, c * 64, w.nt * 128, bar(B_FULL_LR + s));
+                tma_load_2d(sbase + C::OffT + s * C::TBytes, &map_t, c * 64, w.tt * BT, bar(B_FULL_LR + s));
+                ++cl;
+                return true;
+            };
+            while (ok && next_work(cur, p, w)) {
+                // low-rank chunks that fit the ring go first (they are needed last, so this only
+                // prefetches); any further chunk follows the activation stages, which keeps every
+                // ring's producer and consumer in the same order
+                const int early = !w.has_lr ? 0 : (lr_chunks < kLrSlots ? lr_chunks : kLrSlots);
+                for (int c = 0; c < early && ok; ++c) ok = issue_lr(c);
+                for (int kb = w.kb0; kb < w.kb1 && ok; kb += KS) {
+                    const int s = ca % C::NA;
+                    ok = mbar_wait(bar(B_FREE + s), ((ca / C::NA) & 1) ^ 1, ab);
+                    if (!ok) break;
+                    // box = KS column blocks x BT tokens x 128 bytes (blocks past K read as zero)
+                    mbar_arrive_expect_tx(bar(B_READY + s), C::XBytes);
+                    tma_load_3d(sbase + C::OffX + s * C::XBytes, &map_x, 0, w.tt * BT, kb, bar(B_READY + s));
+                    ++ca;
+                }
+                if (w.has_lr)
+                    for (int c = early; c < lr_chunks && ok; ++c) ok = issue_lr(c);
+            }
+            if (!ok || *abort_flag) {
+                // Activation copies complete on READY barriers, which also count the unpack
+                // warps; after an abort they may never flip, so wait (bounded) on what can.
                 for (uint32_t i = (cl > (uint32_t)kLrSlots ? cl - kLrSlots : 0); i < cl; ++i)
                     mbar_wait(bar(B_FULL_LR + i % kLrSlots), (i / kLrSlots) & 1, Abort{never_flag, p.status});
+                for (uint32_t i = (ca > (uint32_t)C::NA ? ca - C::NA : 0); i < ca; ++i)
+                    mbar_wait(bar(B_READY + i % C::NA), (i / C::NA) & 1, Abort{never_flag, p.status});
             }
         }
     } else if (warp == 1) {
@@ -444,7 +448,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             Cursor cur;
             cur.init(u_begin, u_end, p);
             Work w;
-            uint32_t cx = 0, ca = 0, cl = 0, ci = 0, clr_items = 0;
+            uint32_t ca = 0, cl = 0, ci = 0, clr_items = 0;
             bool ok = true;
             while (ok && next_work(cur, p, w)) {
                 const int buf = ci & 1;
@@ -452,20 +456,26 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 ok = mbar_wait(bar(B_ACC_EMPTY + buf), ((ci >> 1) & 1) ^ 1, ab);
                 if (!ok) break;
                 tc_fence_after();
-                for (int kb = w.kb0; kb < w.kb1 && ok; ++kb) {
-                    const int sx = cx % C::NX, sa = ca % C::NA;
-                    ok = mbar_wait(bar(B_FULL_X + sx), (cx / C::NX) & 1, ab) &&
-                         mbar_wait(bar(B_A_FULL + sa), (ca / C::NA) & 1, ab);
+                for (int kb = w.kb0; kb < w.kb1 && ok; kb += KS) {
+                    const int nkb = (w.kb1 - kb < KS) ? (w.kb1 - kb) : KS;
+                    const int sa = ca % C::NA;
+                    ok = mbar_wait(bar(B_READY + sa), (ca / C::NA) & 1, ab);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint64_t xdesc = smem_desc_sw128(sbase + C::OffX + sx * C::XBytes);
+                    const uint64_t xdesc = smem_desc_sw128(sbase + C::OffX + sa * C::XBytes);
+                    const uint32_t a_tm = tm_a0 + sa * C::ASlotCols;
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)
-                        mma_i8_ts(d_int, tm_a0 + sa * 32 + kk * 8, xdesc + 2 * kk, idesc_i8,
-                                  (kb != w.kb0 || kk != 0) ? 1u : 0u);
-                    tc_commit(bar(B_EMPTY_X + sx));
-                    tc_commit(bar(B_A_EMPTY + sa));
-                    ++cx; ++ca;
+                    for (int j = 0; j < KS; ++j) {
+                        if (j < nkb) {
+#pragma unroll
+                            for (int kk = 0; kk < 4; ++kk)
+                                mma_i8_ts(d_int, a_tm + j * 32 + kk * 8,
+                                          xdesc + (uint64_t)(j * (C::XTile >> 4) + 2 * kk), idesc_i8,
+                                          (kb != w.kb0 || j != 0 || kk != 0) ? 1u : 0u);
+                        }
+                    }
+                    tc_commit(bar(B_FREE + sa));
+                    ++ca;
                 }
                 if (ok && w.has_lr) {
                     ok = mbar_wait(bar(B_DLR_EMPTY), (clr_items & 1) ^ 1, ab);
@@ -501,32 +511,38 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         uint32_t cw = 0, ca = 0, cl = 0;
         bool ok = true;
         while (ok && next_work(cur, p, w)) {
-            for (int kb = w.kb0; kb < w.kb1 && ok; ++kb) {
+            for (int kb = w.kb0; kb < w.kb1 && ok; kb += KS) {
+                const int nkb = (w.kb1 - kb < KS) ? (w.kb1 - kb) : KS;
                 const int sw = cw % C::NW, sa = ca % C::NA;
-                ok = warp_mbar_wait(bar(B_FULL_W + sw), (cw / C::NW) & 1, ab, lane);
-                if (!ok) break;
-                const uint8_t* wsrc = smem + C::OffW + sw * kWkBlockBytes + row * 16;
-                uint32_t v[32];
-#pragma unroll
-                for (int sub = 0; sub < 4; ++sub) {
-                    uint4 x = *reinterpret_cast<const uint4*>(wsrc + sub * 2048);
-                    const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        v[sub * 8 + 2 * i] = (xs[i] << 4) & 0xF0F0F0F0u;   // columns c0 .. c0+3
-                        v[sub * 8 + 2 * i + 1] = xs[i] & 0xF0F0F0F0u;      // columns c0+4 .. c0+7
-                    }
-                }
-                __syncwarp();                       // every lane holds its values in registers:
-                if (lane == 0) mbar_arrive(bar(B_EMPTY_W + sw));   // the slot may be refilled
-                ok = warp_mbar_wait(bar(B_A_EMPTY + sa), ((ca / C::NA) & 1) ^ 1, ab, lane);
+                ok = warp_mbar_wait(bar(B_W_FULL + sw), (cw / C::NW) & 1, ab, lane) &&
+                     warp_mbar_wait(bar(B_FREE + sa), ((ca / C::NA) & 1) ^ 1, ab, lane);
                 if (!ok) break;
                 tc_fence_after();
-                tmem_st32(tm_a0 + sa * 32 + ((uint32_t)(q * 32) << 16), v);
+                const uint8_t* wsrc = smem + C::OffW + sw * C::WBytes + row * 16;
+                const uint32_t a_tm = tm_a0 + sa * C::ASlotCols + ((uint32_t)(q * 32) << 16);
+#pragma unroll
+                for (int j = 0; j < KS; ++j) {
+                    if (j < nkb) {
+                        uint32_t v[32];
+#pragma unroll
+                        for (int sub = 0; sub < 4; ++sub) {
+                            uint4 x = *reinterpret_cast<const uint4*>(wsrc + j * kWkBlockBytes + sub * 2048);
+                            const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                v[sub * 8 + 2 * i] = (xs[i] << 4) & 0xF0F0F0F0u;   // columns c0 .. c0+3
+                                v[sub * 8 + 2 * i + 1] = xs[i] & 0xF0F0F0F0u;      // columns c0+4 .. c0+7
+                            }
+                        }
+                        tmem_st32(a_tm + j * 32, v);
+                    }
+                }
+                __syncwarp();                                        // all lanes have read the slot:
+                if (lane == 0) mbar_arrive(bar(B_W_FREE + sw));      // it may be refilled
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(B_A_FULL + sa));
+                if (lane == 0) mbar_arrive(bar(B_READY + sa));
                 ++cw; ++ca;
             }
             if (ok && w.has_lr) {
@@ -555,7 +571,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 }
             }
         }
-    } else {
+    } else if (warp < 10) {
         // =================== epilogue warps ===================
         const int q = warp & 3;
         const int nl = q * 32 + lane;              // row of D = output channel inside the tile
@@ -711,6 +727,23 @@ int make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, int esize, const void*
     return ASER_OK;
 }
 
+// Xq [M, K] int8 viewed as [K/128 column blocks][M tokens][128 bytes]; box = KS blocks x BT
+// tokens x 128 bytes, 128-byte swizzle.  In shared memory each block's BT x 128-byte tile is
+// contiguous, which is the K-major operand layout the MMA descriptor expects.
+int make_map_x(CUtensorMap* map, const void* base, uint64_t M, uint64_t K, uint32_t BT, uint32_t KS) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return record_cuda_error(cudaErrorUnknown, "cuTensorMapEncodeTiled unavailable");
+    cuuint64_t dims[3] = {128, M, K / 128};
+    cuuint64_t strides[2] = {K, 128};
+    cuuint32_t box[3] = {128, BT, KS};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(base), dims, strides, box,
+                    estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return record_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled (Xq)");
+    return ASER_OK;
+}
+
 int pick_bt(int M) { return M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128; }
 
 struct Layout {
@@ -777,7 +810,8 @@ int launch_linear_tc(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
     if (grid > want) grid = (int)want;
 
     CUtensorMap mx, mlb, mt;
-    int rc = make_map_2d(&mx, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Xq, M, K, L.BT, 128);
+    const int ks = L.BT <= 32 ? 4 : (L.BT == 64 ? 2 : 1);   // Cfg<BT>::KS
+    int rc = make_map_x(&mx, Xq, M, K, L.BT, ks);
     if (rc != ASER_OK) return rc;
     if (r > 0) {
         rc = make_map_2d(&mlb, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, LB, N, r, 128, 64);

@@ -37,6 +37,7 @@ WORKLOADS = {
     "c2_decode_m1": (2, 1, 4096, 4096, 64, False, 30.0, 0.02, "hbm"),
     "c3_prefill_gate_up": (3, 2048, 14336, 4096, 64, False, 30.0, 0.02, "tensor"),
     "c3_prefill_down": (3, 2048, 4096, 14336, 64, True, 30.0, 0.02, "tensor"),
+    "c3_small": (3, 2048, 4096, 4096, 64, False, 30.0, 0.02, "tensor"),
     "c5_decode_m16_8192": (5, 16, 8192, 8192, 64, False, 50.0, 0.015, "hbm"),
     "c5_decode_m16_28672": (5, 16, 28672, 8192, 64, False, 50.0, 0.015, "hbm"),
     "c5_prefill_m4096_8192": (5, 4096, 8192, 8192, 64, False, 50.0, 0.015, "tensor"),

@@ -12,9 +12,9 @@
 // units is cut into equal contiguous ranges, one per CTA; tiles shared by several CTAs are
 // summed through the workspace by whichever CTA arrives last.
 //
-// Warp roles (352 threads): 0 = weight producer, 1 = MMA issuer (+ TMEM owner),
-// 2..5 = int4 -> int8 unpack into TMEM (+ T conversion), 6..9 = epilogue,
-// 10 = activation and low-rank operand producer.
+// Warp roles (480 threads): 0 = weight producer, 1 = MMA issuer (+ TMEM owner),
+// 2..5 and 6..9 = two groups of int4 -> int8 unpack warps that take alternate stages
+// (group 0 also converts T), 10..13 = epilogue, 14 = activation and low-rank operand producer.
 // Every wait is bounded: on expiry the CTA sets the status word and winds down.
 #include <cuda.h>
 
@@ -24,7 +24,7 @@ namespace aser {
 
 namespace {
 
-constexpr int kThreads = 352;
+constexpr int kThreads = 480;
 constexpr int kLrSlots = 2;       // ring of low-rank chunks (64 columns of r each)
 constexpr int kMaxCtas = 160;     // upper bound on the persistent grid (workspace sizing)
 constexpr uint32_t kStatusTimeout = 1u;
@@ -32,13 +32,15 @@ constexpr long long kWaitLimitClocks = 4000000000ll;  // about 2 s of SM clocks 
 
 // Per token-tile configuration.  A pipeline stage carries KS 128-column blocks: one bulk copy of
 // KS x 8 KiB of packed weights, one TMA box of KS activation tiles, KS x 32 tensor-memory columns
-// of unpacked A operand.  Large stages keep the per-byte count of copy issues, barrier waits and
-// commits low (each costs a single thread hundreds of cycles), which is what bounds decode shapes.
+// of unpacked A operand.  Under copy traffic every mbarrier operation costs a thread a few
+// hundred cycles, so stages are made large (few waits, arrivals, copy issues and commits per
+// byte) and the unpack work alternates between two groups of four warps.
 template <int BT>
 struct Cfg {
-    static constexpr int KS = (BT <= 32) ? 4 : (BT == 64 ? 2 : 1);
-    static constexpr int NW = (BT <= 32) ? 4 : (BT == 64 ? 5 : 8);     // weight ring depth
-    static constexpr int NA = (BT <= 32) ? 3 : 4;                       // activation / A-operand ring depth
+    static constexpr int KS = (BT <= 32) ? 4 : 2;
+    static constexpr int NW = (BT == 128) ? 3 : 4;                      // weight ring depth
+    static constexpr int NX = (BT == 128) ? 3 : (BT == 64 ? 4 : 3);     // activation ring depth
+    static constexpr int NA = (BT == 128) ? 2 : (BT == 64 ? 4 : 3);     // A-operand ring (tensor memory)
     static constexpr int WBytes = KS * kWkBlockBytes;
     static constexpr int XTile = BT * 128;                              // one 128-column block of Xq
     static constexpr int XBytes = KS * XTile;
@@ -46,10 +48,10 @@ struct Cfg {
     static constexpr int TBytes = BT * 128;            // BT rows x 64 bf16/fp16
     static constexpr int OffW = 0;
     static constexpr int OffX = OffW + NW * WBytes;
-    static constexpr int OffLb = OffX + NA * XBytes;
+    static constexpr int OffLb = OffX + NX * XBytes;
     static constexpr int OffT = OffLb + kLrSlots * LbBytes;
     static constexpr int OffBar = OffT + kLrSlots * TBytes;
-    static constexpr int NumBars = 2 * NW + 2 * NA + 3 * kLrSlots + 2 + 2 + 1;
+    static constexpr int NumBars = 2 * NW + 2 * NX + 2 * NA + 3 * kLrSlots + 2 + 2 + 1;
     static constexpr int SmemBytes = OffBar + NumBars * 8 + 64 + 1024;  // + slack for 1 KiB alignment
     static constexpr int ASlotCols = KS * 32;
     static constexpr int TmemColsUsed = 3 * BT + NA * ASlotCols;
@@ -323,9 +325,12 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     // barrier indices
     //   W_FULL[s]  weight bytes of stage landed (tx)          -> unpack warps
     //   W_FREE[s]  unpack warps have the weights in registers -> weight producer
-    //   READY[a]   activation bytes landed (tx) AND A operand written to tensor memory -> MMA issuer
-    //   FREE[a]    MMAs of the stage retired (commit)         -> activation producer, unpack warps
-    constexpr int B_W_FULL = 0, B_W_FREE = B_W_FULL + C::NW, B_READY = B_W_FREE + C::NW,
+    //   X_FULL[x]  activation bytes of stage landed (tx)      -> first warp of the unpack group
+    //   X_FREE[x]  MMAs of the stage retired (commit)         -> activation producer
+    //   READY[a]   A operand in tensor memory, activations seen in shared memory -> MMA issuer
+    //   FREE[a]    MMAs of the stage retired (commit)         -> unpack warps
+    constexpr int B_W_FULL = 0, B_W_FREE = B_W_FULL + C::NW, B_X_FULL = B_W_FREE + C::NW,
+                  B_X_FREE = B_X_FULL + C::NX, B_READY = B_X_FREE + C::NX,
                   B_FREE = B_READY + C::NA, B_FULL_LR = B_FREE + C::NA,
                   B_CONV_LR = B_FULL_LR + kLrSlots, B_EMPTY_LR = B_CONV_LR + kLrSlots,
                   B_ACC_FULL = B_EMPTY_LR + kLrSlots, B_ACC_EMPTY = B_ACC_FULL + 2,
@@ -343,7 +348,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < C::NW; ++i) { mbar_init(bar(B_W_FULL + i), 1); mbar_init(bar(B_W_FREE + i), 4); }
-        for (int i = 0; i < C::NA; ++i) { mbar_init(bar(B_READY + i), 5); mbar_init(bar(B_FREE + i), 1); }
+        for (int i = 0; i < C::NX; ++i) { mbar_init(bar(B_X_FULL + i), 1); mbar_init(bar(B_X_FREE + i), 1); }
+        for (int i = 0; i < C::NA; ++i) { mbar_init(bar(B_READY + i), 4); mbar_init(bar(B_FREE + i), 1); }
         for (int i = 0; i < kLrSlots; ++i) {
             mbar_init(bar(B_FULL_LR + i), 1); mbar_init(bar(B_CONV_LR + i), 4); mbar_init(bar(B_EMPTY_LR + i), 1);
         }
@@ -396,13 +402,13 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     mbar_wait(bar(B_W_FULL + i % C::NW), (i / C::NW) & 1, Abort{never_flag, p.status});
             }
         }
-    } else if (warp == 10) {
+    } else if (warp == 14) {
         // =================== activation + low-rank operand producer (one lane) ===================
         if (lane == 0) {
             Cursor cur;
             cur.init(u_begin, u_end, p);
             Work w{};
-            uint32_t ca = 0, cl = 0;
+            uint32_t cx = 0, cl = 0;
             bool ok = true;
             auto issue_lr = [&](int c) {
                 const int s = cl % kLrSlots;
@@ -420,24 +426,23 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 const int early = !w.has_lr ? 0 : (lr_chunks < kLrSlots ? lr_chunks : kLrSlots);
                 for (int c = 0; c < early && ok; ++c) ok = issue_lr(c);
                 for (int kb = w.kb0; kb < w.kb1 && ok; kb += KS) {
-                    const int s = ca % C::NA;
-                    ok = mbar_wait(bar(B_FREE + s), ((ca / C::NA) & 1) ^ 1, ab);
+                    const int s = cx % C::NX;
+                    ok = mbar_wait(bar(B_X_FREE + s), ((cx / C::NX) & 1) ^ 1, ab);
                     if (!ok) break;
                     // box = KS column blocks x BT tokens x 128 bytes (blocks past K read as zero)
-                    mbar_arrive_expect_tx(bar(B_READY + s), C::XBytes);
-                    tma_load_3d(sbase + C::OffX + s * C::XBytes, &map_x, 0, w.tt * BT, kb, bar(B_READY + s));
-                    ++ca;
+                    mbar_arrive_expect_tx(bar(B_X_FULL + s), C::XBytes);
+                    tma_load_3d(sbase + C::OffX + s * C::XBytes, &map_x, 0, w.tt * BT, kb, bar(B_X_FULL + s));
+                    ++cx;
                 }
                 if (w.has_lr)
                     for (int c = early; c < lr_chunks && ok; ++c) ok = issue_lr(c);
             }
             if (!ok || *abort_flag) {
-                // Activation copies complete on READY barriers, which also count the unpack
-                // warps; after an abort they may never flip, so wait (bounded) on what can.
+                // let copies already issued land before the CTA's shared memory goes away
                 for (uint32_t i = (cl > (uint32_t)kLrSlots ? cl - kLrSlots : 0); i < cl; ++i)
                     mbar_wait(bar(B_FULL_LR + i % kLrSlots), (i / kLrSlots) & 1, Abort{never_flag, p.status});
-                for (uint32_t i = (ca > (uint32_t)C::NA ? ca - C::NA : 0); i < ca; ++i)
-                    mbar_wait(bar(B_READY + i % C::NA), (i / C::NA) & 1, Abort{never_flag, p.status});
+                for (uint32_t i = (cx > (uint32_t)C::NX ? cx - C::NX : 0); i < cx; ++i)
+                    mbar_wait(bar(B_X_FULL + i % C::NX), (i / C::NX) & 1, Abort{never_flag, p.status});
             }
         }
     } else if (warp == 1) {
@@ -458,11 +463,11 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 tc_fence_after();
                 for (int kb = w.kb0; kb < w.kb1 && ok; kb += KS) {
                     const int nkb = (w.kb1 - kb < KS) ? (w.kb1 - kb) : KS;
-                    const int sa = ca % C::NA;
+                    const int sa = ca % C::NA, sx = ca % C::NX;   // ca counts stages
                     ok = mbar_wait(bar(B_READY + sa), (ca / C::NA) & 1, ab);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint64_t xdesc = smem_desc_sw128(sbase + C::OffX + sa * C::XBytes);
+                    const uint64_t xdesc = smem_desc_sw128(sbase + C::OffX + sx * C::XBytes);
                     const uint32_t a_tm = tm_a0 + sa * C::ASlotCols;
 #pragma unroll
                     for (int j = 0; j < KS; ++j) {
@@ -475,6 +480,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                         }
                     }
                     tc_commit(bar(B_FREE + sa));
+                    tc_commit(bar(B_X_FREE + sx));
                     ++ca;
                 }
                 if (ok && w.has_lr) {
@@ -500,22 +506,25 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 ++ci;
             }
         }
-    } else if (warp < 6) {
+    } else if (warp < 10) {
         // =================== unpack warps: int4 -> int8 (x16) into tensor memory ===================
         const int q = warp & 3;                    // TMEM lane quarter this warp may touch
         const int row = q * 32 + lane;             // weight row inside the 128-row tile
-        const int t128 = (warp - 2) * 32 + lane;   // 0..127 among the unpack threads
+        const int group = (warp - 2) >> 2;         // stages alternate between the two groups
+        const int gwarp = (warp - 2) & 3;          // warp within its group
+        const int t128 = gwarp * 32 + lane;        // 0..127 within the group
         Cursor cur;
         cur.init(u_begin, u_end, p);
         Work w;
-        uint32_t cw = 0, ca = 0, cl = 0;
+        uint32_t cw = 0, cl = 0;
         bool ok = true;
         while (ok && next_work(cur, p, w)) {
             for (int kb = w.kb0; kb < w.kb1 && ok; kb += KS) {
                 const int nkb = (w.kb1 - kb < KS) ? (w.kb1 - kb) : KS;
-                const int sw = cw % C::NW, sa = ca % C::NA;
+                const int sw = cw % C::NW, sa = cw % C::NA, sx = cw % C::NX;   // cw counts stages
+                if ((int)(cw & 1u) != group) { ++cw; continue; }
                 ok = warp_mbar_wait(bar(B_W_FULL + sw), (cw / C::NW) & 1, ab, lane) &&
-                     warp_mbar_wait(bar(B_FREE + sa), ((ca / C::NA) & 1) ^ 1, ab, lane);
+                     warp_mbar_wait(bar(B_FREE + sa), ((cw / C::NA) & 1) ^ 1, ab, lane);
                 if (!ok) break;
                 tc_fence_after();
                 const uint8_t* wsrc = smem + C::OffW + sw * C::WBytes + row * 16;
@@ -541,11 +550,14 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 if (lane == 0) mbar_arrive(bar(B_W_FREE + sw));      // it may be refilled
                 tmem_wait_st();
                 tc_fence_before();
+                // one warp of the group also vouches for the activation tile of this stage
+                if (gwarp == 0) ok = warp_mbar_wait(bar(B_X_FULL + sx), (cw / C::NX) & 1, ab, lane);
+                if (!ok) break;
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(B_READY + sa));
-                ++cw; ++ca;
+                ++cw;
             }
-            if (ok && w.has_lr) {
+            if (ok && w.has_lr && group == 0) {
                 for (int c = 0; c < lr_chunks && ok; ++c) {
                     const int s = cl % kLrSlots;
                     ok = warp_mbar_wait(bar(B_FULL_LR + s), (cl / kLrSlots) & 1, ab, lane);
@@ -571,11 +583,11 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 }
             }
         }
-    } else if (warp < 10) {
+    } else if (warp < 14) {
         // =================== epilogue warps ===================
         const int q = warp & 3;
         const int nl = q * 32 + lane;              // row of D = output channel inside the tile
-        const int et = (warp - 6) * 32 + lane;     // 0..127 among the epilogue threads
+        const int et = (warp - 10) * 32 + lane;     // 0..127 among the epilogue threads
         const uint32_t lane_sel = (uint32_t)(q * 32) << 16;
         Cursor cur;
         cur.init(u_begin, u_end, p);
@@ -810,7 +822,7 @@ int launch_linear_tc(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
     if (grid > want) grid = (int)want;
 
     CUtensorMap mx, mlb, mt;
-    const int ks = L.BT <= 32 ? 4 : (L.BT == 64 ? 2 : 1);   // Cfg<BT>::KS
+    const int ks = L.BT == 16 ? Cfg<16>::KS : L.BT == 32 ? Cfg<32>::KS : L.BT == 64 ? Cfg<64>::KS : Cfg<128>::KS;
     int rc = make_map_x(&mx, Xq, M, K, L.BT, ks);
     if (rc != ASER_OK) return rc;
     if (r > 0) {

@@ -113,6 +113,34 @@ int aser_linear_w4a8_lr_simt(const int8_t* Xq, const float* a_scale, const uint8
                              int M, int N, int K, int r, void* Y_f16, int32_t* acc_debug,
                              void* stream);
 
+/*
+ * aser_linear_w4a8_lr_static -- aser_linear_w4a8_lr for callers that must not allocate device
+ * memory and therefore have no workspace to hand over: code running inside a memory budget
+ * that was fixed at start-up (a serving process that gave every free byte to its own pool, so
+ * cudaMalloc would fail), or at a point where allocating is not allowed because it would
+ * synchronise the device (inside a latency-critical loop, between the kernels of a step).  The
+ * paper has no counterpart; this is a deployment convenience of the library.
+ * The scratch is a fixed 8 MiB array inside the library image; every GPU that loads the library
+ * holds one copy until the process exits.  Limits and rules:
+ *   - only problems with aser_workspace_bytes(M,N,K,r) <= 8 MiB are accepted, i.e. at most 32
+ *     tokens per call (any N, K, r the library supports); larger ones return ASER_ERR_WORKSPACE
+ *     and launch nothing;
+ *   - the first call on each device looks the array's device address up (with that device
+ *     current); make that first call before starting any stream capture;
+ *   - no cudaMalloc/cudaFree or other allocating routine is called; each call enqueues a small
+ *     memset (status word and tile counters) and the kernel on `stream`;
+ *   - all calls on a device share the one array, so two calls that may overlap in time on the
+ *     GPU (different streams, no dependency) corrupt each other: order them;
+ *   - the status word is not readable by the caller: a timed-out wait (see aser_check_status)
+ *     cannot be detected through this entry point.
+ * Arguments and results are those of aser_linear_w4a8_lr; pass r = 0 with NULL T/LB for the
+ * plain product.
+ */
+int aser_linear_w4a8_lr_static(const int8_t* Xq, const float* a_scale, const void* Wk,
+                               const float* w_scale, const void* T_bf16, const void* LB_f16,
+                               int M, int N, int K, int r, void* Y_f16, int32_t* acc_debug,
+                               void* stream);
+
 /* Workspace: split-K partial sums, tile counters and a status word. */
 size_t aser_workspace_bytes(int M, int N, int K, int r);
 int aser_workspace_init(void* workspace, size_t workspace_bytes, void* stream);

@@ -11,7 +11,7 @@ lib_path = os.path.join(_HERE, "libaser.so")
 
 EXPORTED_SYMBOLS = (
     "aser_pack_w4", "aser_repacked_bytes", "aser_repack_w4", "aser_unrepack_w4",
-    "aser_quant_act", "aser_linear_w4a8_lr", "aser_linear_w4a8", "aser_linear_w4a8_lr_simt",
+    "aser_quant_act", "aser_linear_w4a8_lr", "aser_linear_w4a8", "aser_linear_w4a8_lr_simt", "aser_linear_w4a8_lr_static",
     "aser_workspace_bytes", "aser_workspace_init", "aser_check_status", "aser_forward_host",
     "aser_last_error", "aser_version",
 )
@@ -32,6 +32,7 @@ lib.aser_quant_act.argtypes = [_P, _P, _P, _I, _I, _I, _P, _P, _P, _P]
 lib.aser_linear_w4a8_lr.argtypes = [_P, _P, _P, _P, _P, _P, _I, _I, _I, _I, _P, _P, _P, _Z, _P]
 lib.aser_linear_w4a8.argtypes = [_P, _P, _P, _P, _I, _I, _I, _P, _P, _P, _Z, _P]
 lib.aser_linear_w4a8_lr_simt.argtypes = [_P, _P, _P, _P, _P, _P, _I, _I, _I, _I, _P, _P, _P]
+lib.aser_linear_w4a8_lr_static.argtypes = [_P, _P, _P, _P, _P, _P, _I, _I, _I, _I, _P, _P, _P]
 lib.aser_workspace_bytes.argtypes = [_I, _I, _I, _I]
 lib.aser_workspace_bytes.restype = _Z
 lib.aser_workspace_init.argtypes = [_P, _Z, _P]
@@ -169,6 +170,20 @@ def linear_w4a8_lr_simt(Xq, a_scale, Wq, w_scale, T, L_B, Y=None, acc_debug=None
                                       _ptr(T) if r else None, _ptr(L_B) if r else None, M, N, K, r,
                                       _ptr(Y), _ptr(acc_debug), _stream()),
          "aser_linear_w4a8_lr_simt")
+    return Y
+
+
+def linear_w4a8_lr_static(Xq, a_scale, Wk, w_scale, T, L_B, N: int, Y=None, acc_debug=None):
+    """aser_linear_w4a8_lr_static: same result as linear_w4a8_lr, no workspace argument (the
+    library's built-in scratch array is used; at most 32 tokens per call)."""
+    M, K = Xq.shape
+    r = 0 if L_B is None else L_B.shape[1]
+    if Y is None:
+        Y = torch.empty((M, N), dtype=torch.float16, device=Xq.device)
+    _chk(lib.aser_linear_w4a8_lr_static(_ptr(Xq), _ptr(a_scale), _ptr(Wk), _ptr(w_scale),
+                                        _ptr(T) if r else None, _ptr(L_B) if r else None, M, N, K,
+                                        r, _ptr(Y), _ptr(acc_debug), _stream()),
+         "aser_linear_w4a8_lr_static")
     return Y
 
 

@@ -15,6 +15,11 @@ int record_cuda_error(cudaError_t e, const char* where) {
     return ASER_ERR_LAUNCH;
 }
 
+int record_error(int code, const char* msg) {
+    snprintf(g_last_error, sizeof(g_last_error), "%s", msg);
+    return code;
+}
+
 int check_launch(const char* where) {
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return record_cuda_error(e, where);

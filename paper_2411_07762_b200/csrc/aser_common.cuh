@@ -13,6 +13,8 @@ namespace aser {
 // ---- host side -------------------------------------------------------------
 // Records the text of a CUDA error for aser_last_error() and returns ASER_ERR_LAUNCH.
 int record_cuda_error(cudaError_t e, const char* where);
+// Records a plain message for aser_last_error() and returns `code`.
+int record_error(int code, const char* msg);
 // cudaGetLastError() after a launch -> ASER_OK or ASER_ERR_LAUNCH.
 int check_launch(const char* where);
 
@@ -32,6 +34,8 @@ int launch_linear_tc(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
                      int M, int N, int K, int r, __half* Y, int32_t* acc_debug,
                      void* workspace, size_t workspace_bytes, cudaStream_t st);
 size_t linear_tc_workspace_bytes(int M, int N, int K, int r);
+// Leading bytes of the workspace (status word + tile counters) that must be zero at launch.
+size_t linear_tc_zeroed_prefix_bytes(int M, int N, int K, int r);
 
 // Layout of the repacked weight: [N/128 row blocks][K/128 column blocks][8 KiB].
 // Inside a block: 4 sub-blocks of 32 columns; each holds 128 rows x 16 bytes.

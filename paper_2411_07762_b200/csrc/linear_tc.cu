@@ -801,6 +801,11 @@ size_t linear_tc_workspace_bytes(int M, int N, int K, int r) {
     return make_layout(M, N, K, r).total - kWsHeaderBytes;
 }
 
+size_t linear_tc_zeroed_prefix_bytes(int M, int N, int K, int r) {
+    if (M <= 0 || N <= 0) return kWsHeaderBytes;
+    return make_layout(M, N, K, r).off_part_int;
+}
+
 int launch_linear_tc(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
                      const float* w_scale, const __nv_bfloat16* T, const __half* LB,
                      int M, int N, int K, int r, __half* Y, int32_t* acc_debug,

@@ -12,9 +12,14 @@
 // units is cut into equal contiguous ranges, one per CTA; tiles shared by several CTAs are
 // summed through the workspace by whichever CTA arrives last.
 //
-// Warp roles (480 threads): 0 = weight producer, 1 = MMA issuer (+ TMEM owner),
-// 2..5 and 6..9 = two groups of int4 -> int8 unpack warps that take alternate stages
-// (group 0 also converts T), 10..13 = epilogue, 14 = activation and low-rank operand producer.
+// Warp roles (512 threads): 0 = weight producer, 1 and 15 = MMA issuers for even / odd stages
+// (1 also owns the TMEM allocation and issues the low-rank MMAs), 2..5 and 6..9 = two groups of
+// int4 -> int8 unpack warps that take alternate stages (group 0 also converts T),
+// 10..13 = epilogue, 14 = activation and low-rank operand producer.
+// A single lane issues one tcgen05.mma per ~60-85 cycles, which bounds decode shapes (16 MMAs
+// per 32 KiB of weights); the integer accumulation is order-independent, so two lanes share the
+// issue work.  For that the accumulator is zeroed by the epilogue warps (tcgen05.st) when they
+// hand it back, and every integer MMA accumulates.
 // Every wait is bounded: on expiry the CTA sets the status word and winds down.
 #include <cuda.h>
 
@@ -24,7 +29,7 @@ namespace aser {
 
 namespace {
 
-constexpr int kThreads = 480;
+constexpr int kThreads = 512;
 constexpr int kLrSlots = 2;       // ring of low-rank chunks (64 columns of r each)
 constexpr int kMaxCtas = 160;     // upper bound on the persistent grid (workspace sizing)
 constexpr uint32_t kStatusTimeout = 1u;
@@ -110,6 +115,9 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
         : "memory");
 }
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
@@ -152,6 +160,15 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32
         "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]),
         "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]),
         "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
+        : "memory");
+}
+// Zero 16 consecutive columns of this warp's 32 lanes.
+__device__ __forceinline__ void tmem_zero16(uint32_t taddr) {
+    const uint32_t z = 0;
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1};"
+        ::"r"(taddr), "r"(z)
         : "memory");
 }
 __device__ __forceinline__ void tmem_wait_st() {
@@ -353,13 +370,49 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         for (int i = 0; i < kLrSlots; ++i) {
             mbar_init(bar(B_FULL_LR + i), 1); mbar_init(bar(B_CONV_LR + i), 4); mbar_init(bar(B_EMPTY_LR + i), 1);
         }
-        for (int i = 0; i < 2; ++i) { mbar_init(bar(B_ACC_FULL + i), 1); mbar_init(bar(B_ACC_EMPTY + i), 4); }
+        for (int i = 0; i < 2; ++i) { mbar_init(bar(B_ACC_FULL + i), 2); mbar_init(bar(B_ACC_EMPTY + i), 4); }
         mbar_init(bar(B_DLR_EMPTY), 4);
         *abort_flag = 0;
         *last_flag = 0;
         *never_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async_smem();
+    }
+    // Weight producer state (thread 0).  Its first copies go out before the CTA-wide
+    // synchronisation below: they need only the barriers this thread has just initialised.
+    Cursor wcur;
+    wcur.init(u_begin, u_end, p);
+    Work ww{};
+    int wkb = 0;
+    bool w_have = false, w_ok = true;
+    uint32_t wcw = 0;
+    auto w_issue_one = [&]() -> bool {   // false: nothing left, or a wait gave up (w_ok)
+        if (!w_have) {
+            if (!next_work(wcur, p, ww)) return false;
+            wkb = ww.kb0;
+            w_have = true;
+        }
+        const int nkb = (ww.kb1 - wkb < KS) ? (ww.kb1 - wkb) : KS;
+        const int s = wcw % C::NW;
+        w_ok = mbar_wait(bar(B_W_FREE + s), ((wcw / C::NW) & 1) ^ 1, ab);
+        if (!w_ok) return false;
+        // the blocks of one row tile are adjacent in memory: one copy per stage
+        mbar_arrive_expect_tx(bar(B_W_FULL + s), nkb * kWkBlockBytes);
+        bulk_copy_g2s(sbase + C::OffW + s * C::WBytes,
+                      p.Wk + ((size_t)ww.nt * p.KB + wkb) * kWkBlockBytes, nkb * kWkBlockBytes,
+                      bar(B_W_FULL + s));
+        ++wcw;
+        wkb += KS;
+        if (wkb >= ww.kb1) w_have = false;
+        return true;
+    };
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < C::NW; ++i)
+            if (!w_issue_one()) break;
+    }
+    if (warp == 14 && lane == 0) {
+        prefetch_tensormap(&map_x);
+        if (p.r > 0) { prefetch_tensormap(&map_lb); prefetch_tensormap(&map_t); }
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -377,25 +430,9 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     if (warp == 0) {
         // =================== weight producer (one lane) ===================
         if (lane == 0) {
-            Cursor cur;
-            cur.init(u_begin, u_end, p);
-            Work w;
-            uint32_t cw = 0;
-            bool ok = true;
-            while (ok && next_work(cur, p, w)) {
-                for (int kb = w.kb0; kb < w.kb1; kb += KS) {
-                    const int nkb = (w.kb1 - kb < KS) ? (w.kb1 - kb) : KS;
-                    const int s = cw % C::NW;
-                    ok = mbar_wait(bar(B_W_FREE + s), ((cw / C::NW) & 1) ^ 1, ab);
-                    if (!ok) break;
-                    // the blocks of one row tile are adjacent in memory: one copy per stage
-                    mbar_arrive_expect_tx(bar(B_W_FULL + s), nkb * kWkBlockBytes);
-                    bulk_copy_g2s(sbase + C::OffW + s * C::WBytes,
-                                  p.Wk + ((size_t)w.nt * p.KB + kb) * kWkBlockBytes, nkb * kWkBlockBytes,
-                                  bar(B_W_FULL + s));
-                    ++cw;
-                }
-            }
+            while (w_ok && w_issue_one()) {}
+            const uint32_t cw = wcw;
+            const bool ok = w_ok;
             if (!ok || *abort_flag) {
                 // let copies already issued land before the CTA's shared memory goes away
                 for (uint32_t i = (cw > (uint32_t)C::NW ? cw - C::NW : 0); i < cw; ++i)
@@ -424,8 +461,10 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 // prefetches); any further chunk follows the activation stages, which keeps every
                 // ring's producer and consumer in the same order
                 const int early = !w.has_lr ? 0 : (lr_chunks < kLrSlots ? lr_chunks : kLrSlots);
-                for (int c = 0; c < early && ok; ++c) ok = issue_lr(c);
                 for (int kb = w.kb0; kb < w.kb1 && ok; kb += KS) {
+                    if (kb == w.kb0 + KS)   // after the first activation stage of the item
+                        for (int c = 0; c < early && ok; ++c) ok = issue_lr(c);
+                    if (!ok) break;
                     const int s = cx % C::NX;
                     ok = mbar_wait(bar(B_X_FREE + s), ((cx / C::NX) & 1) ^ 1, ab);
                     if (!ok) break;
@@ -434,8 +473,11 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     tma_load_3d(sbase + C::OffX + s * C::XBytes, &map_x, 0, w.tt * BT, kb, bar(B_X_FULL + s));
                     ++cx;
                 }
-                if (w.has_lr)
+                if (w.has_lr) {
+                    if (w.kb1 - w.kb0 <= KS)   // single-stage item: the early chunks are still due
+                        for (int c = 0; c < early && ok; ++c) ok = issue_lr(c);
                     for (int c = early; c < lr_chunks && ok; ++c) ok = issue_lr(c);
+                }
             }
             if (!ok || *abort_flag) {
                 // let copies already issued land before the CTA's shared memory goes away
@@ -445,8 +487,9 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     mbar_wait(bar(B_X_FULL + i % C::NX), (i / C::NX) & 1, Abort{never_flag, p.status});
             }
         }
-    } else if (warp == 1) {
-        // =================== MMA issuer (one lane) ===================
+    } else if (warp == 1 || warp == 15) {
+        // =================== MMA issuers (one lane each; even / odd stages) ===================
+        const int issuer = (warp == 1) ? 0 : 1;
         if (lane == 0) {
             constexpr uint32_t idesc_i8 = make_idesc(2, 1, 128, BT);
             constexpr uint32_t idesc_f16 = make_idesc(1, 0, 128, BT);
@@ -458,12 +501,14 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             while (ok && next_work(cur, p, w)) {
                 const int buf = ci & 1;
                 const uint32_t d_int = tm_dint0 + buf * BT;
-                ok = mbar_wait(bar(B_ACC_EMPTY + buf), ((ci >> 1) & 1) ^ 1, ab);
+                // the epilogue warps hand the accumulator over zeroed (first time: initial zeroing)
+                ok = mbar_wait(bar(B_ACC_EMPTY + buf), (ci >> 1) & 1, ab);
                 if (!ok) break;
                 tc_fence_after();
                 for (int kb = w.kb0; kb < w.kb1 && ok; kb += KS) {
                     const int nkb = (w.kb1 - kb < KS) ? (w.kb1 - kb) : KS;
                     const int sa = ca % C::NA, sx = ca % C::NX;   // ca counts stages
+                    if ((int)(ca & 1u) != issuer) { ++ca; continue; }
                     ok = mbar_wait(bar(B_READY + sa), (ca / C::NA) & 1, ab);
                     if (!ok) break;
                     tc_fence_after();
@@ -476,14 +521,14 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                             for (int kk = 0; kk < 4; ++kk)
                                 mma_i8_ts(d_int, a_tm + j * 32 + kk * 8,
                                           xdesc + (uint64_t)(j * (C::XTile >> 4) + 2 * kk), idesc_i8,
-                                          (kb != w.kb0 || j != 0 || kk != 0) ? 1u : 0u);
+                                          1u);
                         }
                     }
                     tc_commit(bar(B_FREE + sa));
                     tc_commit(bar(B_X_FREE + sx));
                     ++ca;
                 }
-                if (ok && w.has_lr) {
+                if (ok && w.has_lr && issuer == 0) {
                     ok = mbar_wait(bar(B_DLR_EMPTY), (clr_items & 1) ^ 1, ab);
                     for (int c = 0; c < lr_chunks && ok; ++c) {
                         const int s = cl % kLrSlots;
@@ -595,6 +640,12 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         uint32_t ci = 0;
         int partial_idx = 0;                       // 0: first partial item of this CTA, 1: second
         bool ok = true;
+        // both integer accumulators start at zero: every integer MMA accumulates
+        for (int c0 = 0; c0 < 2 * BT; c0 += 16) tmem_zero16(tm_dint0 + lane_sel + c0);
+        tmem_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) { mbar_arrive(bar(B_ACC_EMPTY + 0)); mbar_arrive(bar(B_ACC_EMPTY + 1)); }
         while (ok && next_work(cur, p, w)) {
             const int buf = ci & 1;
             ok = warp_mbar_wait(bar(B_ACC_FULL + buf), (ci >> 1) & 1, ab, lane);
@@ -634,6 +685,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     }
                 }
             }
+            for (int c0 = 0; c0 < BT; c0 += 16) tmem_zero16(d_int + c0);   // hand it back zeroed
+            tmem_wait_st();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) {
@@ -647,17 +700,17 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 const int first_unit = w.tile * p.KB;
                 const int c_first = unit_owner(p.units, first_unit, G);
                 const int c_last = unit_owner(p.units, first_unit + p.KB - 1, G);
-                __threadfence();
-                named_bar_sync(1, 128);
-                if (et == 0) {
-                    int old = atomicAdd(p.counters + w.tile, 1);
+                named_bar_sync(1, 128);            // every partial store of this CTA precedes ...
+                if (et == 0) {                     // ... this release; the last arriver acquires all
+                    int old;
+                    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;"
+                                 : "=r"(old) : "l"(p.counters + w.tile) : "memory");
                     *last_flag = (old == c_last - c_first) ? 1 : 0;
                 }
                 named_bar_sync(1, 128);
                 const bool last = *last_flag != 0;
                 named_bar_sync(1, 128);           // everyone has read the flag before it is reused
                 if (last) {
-                    __threadfence();
                     if (et == 0) p.counters[w.tile] = 0;   // ready for the next launch
 #pragma unroll 1
                     for (int c0 = 0; c0 < BT; c0 += 16) {
@@ -665,14 +718,29 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                         int sum[16];
 #pragma unroll
                         for (int j = 0; j < 16; ++j) sum[j] = 0;
-                        for (int c = c_first; c <= c_last; ++c) {
-                            // CTA c's items in order: a tile cut off at the start of its range
-                            // (slot 0), whole tiles, a tile cut off at the end of its range.
-                            const int bc = range_begin(p.units, c, G);
-                            const int slot = (bc >= first_unit) ? 0 : ((bc % p.KB != 0) ? 1 : 0);
-                            const int32_t* src = p.part_int + ((size_t)c * 2 + slot) * (BT * 128) + c0 * 128 + nl;
+                        for (int cb = c_first; cb <= c_last; cb += 4) {
+                            // four contributors' loads in flight at a time
+                            int v[4][16];
 #pragma unroll
-                            for (int j = 0; j < 16; ++j) sum[j] += __ldcg(src + j * 128);
+                            for (int u = 0; u < 4; ++u) {
+                                const int c = cb + u;
+                                if (c <= c_last) {
+                                    // CTA c's items in order: a tile cut off at the start of its
+                                    // range (slot 0), whole tiles, a tile cut off at its end.
+                                    const int bc = range_begin(p.units, c, G);
+                                    const int slot = (bc >= first_unit) ? 0 : ((bc % p.KB != 0) ? 1 : 0);
+                                    const int32_t* src = p.part_int + ((size_t)c * 2 + slot) * (BT * 128) + c0 * 128 + nl;
+#pragma unroll
+                                    for (int j = 0; j < 16; ++j) v[u][j] = __ldcg(src + j * 128);
+                                } else {
+#pragma unroll
+                                    for (int j = 0; j < 16; ++j) v[u][j] = 0;
+                                }
+                            }
+#pragma unroll
+                            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) sum[j] += v[u][j];
                         }
                         const float* lsrc = p.part_lr + (size_t)c_first * (BT * 128) + c0 * 128 + nl;
 #pragma unroll

@@ -30,7 +30,6 @@ namespace aser {
 namespace {
 
 constexpr int kThreads = 512;
-constexpr int kLrSlots = 2;       // ring of low-rank chunks (64 columns of r each)
 constexpr int kMaxCtas = 160;     // upper bound on the persistent grid (workspace sizing)
 constexpr uint32_t kStatusTimeout = 1u;
 constexpr long long kWaitLimitClocks = 4000000000ll;  // about 2 s of SM clocks per wait
@@ -42,10 +41,16 @@ constexpr long long kWaitLimitClocks = 4000000000ll;  // about 2 s of SM clocks 
 // byte) and the unpack work alternates between two groups of four warps.
 template <int BT>
 struct Cfg {
-    static constexpr int KS = (BT <= 32) ? 4 : 2;
-    static constexpr int NW = (BT == 128) ? 3 : 4;                      // weight ring depth
-    static constexpr int NX = (BT == 128) ? 3 : (BT == 64 ? 4 : 3);     // activation ring depth
-    static constexpr int NA = (BT == 128) ? 2 : (BT == 64 ? 4 : 3);     // A-operand ring (tensor memory)
+    static constexpr int KS = 2;
+    static constexpr int NW = (BT == 128) ? 4 : (BT == 64 ? 6 : 8);     // weight ring depth (even)
+    static constexpr int NX = 4;                                        // activation ring depth
+    // A-operand ring (tensor memory).  All ring depths are even: stages alternate between two
+    // unpack groups and two MMA issuers, and a parity wait is only sound if the waiter sees every
+    // phase of the barrier, i.e. if a ring slot always belongs to the same group.
+    static constexpr int NA = (BT == 128) ? 2 : 4;
+    static_assert(NA % 2 == 0 && NW % 2 == 0 && NX % 2 == 0, "ring ownership");
+    // ring of low-rank chunks (64 columns of r each); one slot where shared memory is tight
+    static constexpr int NL = (BT == 128) ? 1 : 2;
     static constexpr int WBytes = KS * kWkBlockBytes;
     static constexpr int XTile = BT * 128;                              // one 128-column block of Xq
     static constexpr int XBytes = KS * XTile;
@@ -54,9 +59,9 @@ struct Cfg {
     static constexpr int OffW = 0;
     static constexpr int OffX = OffW + NW * WBytes;
     static constexpr int OffLb = OffX + NX * XBytes;
-    static constexpr int OffT = OffLb + kLrSlots * LbBytes;
-    static constexpr int OffBar = OffT + kLrSlots * TBytes;
-    static constexpr int NumBars = 2 * NW + 2 * NX + 2 * NA + 3 * kLrSlots + 2 + 2 + 1;
+    static constexpr int OffT = OffLb + NL * LbBytes;
+    static constexpr int OffBar = OffT + NL * TBytes;
+    static constexpr int NumBars = 2 * NW + 2 * NX + 2 * NA + 3 * NL + 2 + 2 + 1;
     static constexpr int SmemBytes = OffBar + NumBars * 8 + 64 + 1024;  // + slack for 1 KiB alignment
     static constexpr int ASlotCols = KS * 32;
     static constexpr int TmemColsUsed = 3 * BT + NA * ASlotCols;
@@ -349,8 +354,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     constexpr int B_W_FULL = 0, B_W_FREE = B_W_FULL + C::NW, B_X_FULL = B_W_FREE + C::NW,
                   B_X_FREE = B_X_FULL + C::NX, B_READY = B_X_FREE + C::NX,
                   B_FREE = B_READY + C::NA, B_FULL_LR = B_FREE + C::NA,
-                  B_CONV_LR = B_FULL_LR + kLrSlots, B_EMPTY_LR = B_CONV_LR + kLrSlots,
-                  B_ACC_FULL = B_EMPTY_LR + kLrSlots, B_ACC_EMPTY = B_ACC_FULL + 2,
+                  B_CONV_LR = B_FULL_LR + C::NL, B_EMPTY_LR = B_CONV_LR + C::NL,
+                  B_ACC_FULL = B_EMPTY_LR + C::NL, B_ACC_EMPTY = B_ACC_FULL + 2,
                   B_DLR_EMPTY = B_ACC_EMPTY + 2;
     static_assert(B_DLR_EMPTY + 1 == C::NumBars, "barrier count");
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + C::OffBar + C::NumBars * 8);
@@ -367,7 +372,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         for (int i = 0; i < C::NW; ++i) { mbar_init(bar(B_W_FULL + i), 1); mbar_init(bar(B_W_FREE + i), 4); }
         for (int i = 0; i < C::NX; ++i) { mbar_init(bar(B_X_FULL + i), 1); mbar_init(bar(B_X_FREE + i), 1); }
         for (int i = 0; i < C::NA; ++i) { mbar_init(bar(B_READY + i), 4); mbar_init(bar(B_FREE + i), 1); }
-        for (int i = 0; i < kLrSlots; ++i) {
+        for (int i = 0; i < C::NL; ++i) {
             mbar_init(bar(B_FULL_LR + i), 1); mbar_init(bar(B_CONV_LR + i), 4); mbar_init(bar(B_EMPTY_LR + i), 1);
         }
         for (int i = 0; i < 2; ++i) { mbar_init(bar(B_ACC_FULL + i), 2); mbar_init(bar(B_ACC_EMPTY + i), 4); }
@@ -448,8 +453,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             uint32_t cx = 0, cl = 0;
             bool ok = true;
             auto issue_lr = [&](int c) {
-                const int s = cl % kLrSlots;
-                if (!mbar_wait(bar(B_EMPTY_LR + s), ((cl / kLrSlots) & 1) ^ 1, ab)) return false;
+                const int s = cl % C::NL;
+                if (!mbar_wait(bar(B_EMPTY_LR + s), ((cl / C::NL) & 1) ^ 1, ab)) return false;
                 mbar_arrive_expect_tx(bar(B_FULL_LR + s), C::LbBytes + C::TBytes);
                 tma_load_2d(sbase + C::OffLb + s * C::LbBytes, &map_lb, c * 64, w.nt * 128, bar(B_FULL_LR + s));
                 tma_load_2d(sbase + C::OffT + s * C::TBytes, &map_t, c * 64, w.tt * BT, bar(B_FULL_LR + s));
@@ -460,9 +465,15 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 // low-rank chunks that fit the ring go first (they are needed last, so this only
                 // prefetches); any further chunk follows the activation stages, which keeps every
                 // ring's producer and consumer in the same order
-                const int early = !w.has_lr ? 0 : (lr_chunks < kLrSlots ? lr_chunks : kLrSlots);
-                for (int kb = w.kb0; kb < w.kb1 && ok; kb += KS) {
-                    if (kb == w.kb0 + KS)   // after the first activation stage of the item
+                const int early = !w.has_lr ? 0 : (lr_chunks < C::NL ? lr_chunks : C::NL);
+                // With a two-slot ring the chunks go out right after the first activation stage
+                // (pure prefetch).  With one slot the previous tile's low-rank MMA has to retire
+                // first, so they go out four stages before the end of the tile instead.
+                const int nst = (w.kb1 - w.kb0 + KS - 1) / KS;
+                const int lr_at = (C::NL == 1 && nst > 5) ? nst - 4 : 1;
+                int st_idx = 0;
+                for (int kb = w.kb0; kb < w.kb1 && ok; kb += KS, ++st_idx) {
+                    if (st_idx == lr_at)
                         for (int c = 0; c < early && ok; ++c) ok = issue_lr(c);
                     if (!ok) break;
                     const int s = cx % C::NX;
@@ -481,8 +492,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             }
             if (!ok || *abort_flag) {
                 // let copies already issued land before the CTA's shared memory goes away
-                for (uint32_t i = (cl > (uint32_t)kLrSlots ? cl - kLrSlots : 0); i < cl; ++i)
-                    mbar_wait(bar(B_FULL_LR + i % kLrSlots), (i / kLrSlots) & 1, Abort{never_flag, p.status});
+                for (uint32_t i = (cl > (uint32_t)C::NL ? cl - C::NL : 0); i < cl; ++i)
+                    mbar_wait(bar(B_FULL_LR + i % C::NL), (i / C::NL) & 1, Abort{never_flag, p.status});
                 for (uint32_t i = (cx > (uint32_t)C::NX ? cx - C::NX : 0); i < cx; ++i)
                     mbar_wait(bar(B_X_FULL + i % C::NX), (i / C::NX) & 1, Abort{never_flag, p.status});
             }
@@ -531,8 +542,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 if (ok && w.has_lr && issuer == 0) {
                     ok = mbar_wait(bar(B_DLR_EMPTY), (clr_items & 1) ^ 1, ab);
                     for (int c = 0; c < lr_chunks && ok; ++c) {
-                        const int s = cl % kLrSlots;
-                        ok = mbar_wait(bar(B_CONV_LR + s), (cl / kLrSlots) & 1, ab);
+                        const int s = cl % C::NL;
+                        ok = mbar_wait(bar(B_CONV_LR + s), (cl / C::NL) & 1, ab);
                         if (!ok) break;
                         tc_fence_after();
                         const uint64_t adesc = smem_desc_sw128(sbase + C::OffLb + s * C::LbBytes);
@@ -604,8 +615,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             }
             if (ok && w.has_lr && group == 0) {
                 for (int c = 0; c < lr_chunks && ok; ++c) {
-                    const int s = cl % kLrSlots;
-                    ok = warp_mbar_wait(bar(B_FULL_LR + s), (cl / kLrSlots) & 1, ab, lane);
+                    const int s = cl % C::NL;
+                    ok = warp_mbar_wait(bar(B_FULL_LR + s), (cl / C::NL) & 1, ab, lane);
                     if (!ok) break;
                     // T chunk: bf16 -> fp16 in place (same element size, same swizzled position)
                     uint8_t* tb = smem + C::OffT + s * C::TBytes;

@@ -347,9 +347,9 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     // barrier indices
     //   W_FULL[s]  weight bytes of stage landed (tx)          -> unpack warps
     //   W_FREE[s]  unpack warps have the weights in registers -> weight producer
-    //   X_FULL[x]  activation bytes of stage landed (tx)      -> first warp of the unpack group
+    //   X_FULL[x]  activation bytes of stage landed (tx)      -> MMA issuer of the stage
     //   X_FREE[x]  MMAs of the stage retired (commit)         -> activation producer
-    //   READY[a]   A operand in tensor memory, activations seen in shared memory -> MMA issuer
+    //   READY[a]   A operand of the stage written to tensor memory -> MMA issuer of the stage
     //   FREE[a]    MMAs of the stage retired (commit)         -> unpack warps
     constexpr int B_W_FULL = 0, B_W_FREE = B_W_FULL + C::NW, B_X_FULL = B_W_FREE + C::NW,
                   B_X_FREE = B_X_FULL + C::NX, B_READY = B_X_FREE + C::NX,
@@ -368,23 +368,28 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     const int u_begin = range_begin(p.units, cta, G), u_end = range_begin(p.units, cta + 1, G);
     Abort ab{abort_flag, p.status};
 
-    if (threadIdx.x == 0) {
-        for (int i = 0; i < C::NW; ++i) { mbar_init(bar(B_W_FULL + i), 1); mbar_init(bar(B_W_FREE + i), 4); }
-        for (int i = 0; i < C::NX; ++i) { mbar_init(bar(B_X_FULL + i), 1); mbar_init(bar(B_X_FREE + i), 1); }
-        for (int i = 0; i < C::NA; ++i) { mbar_init(bar(B_READY + i), 4); mbar_init(bar(B_FREE + i), 1); }
-        for (int i = 0; i < C::NL; ++i) {
-            mbar_init(bar(B_FULL_LR + i), 1); mbar_init(bar(B_CONV_LR + i), 4); mbar_init(bar(B_EMPTY_LR + i), 1);
+    // Warp 0 initialises the barriers (one per lane and pass) and then only ARRIVES on the
+    // start-up barrier, so that its lane 0 can begin streaming weights at once; every other warp
+    // waits there until the barriers (and the tensor-memory allocation) are in place.
+    if (warp == 0) {
+        for (int i = lane; i < C::NumBars; i += 32) {
+            const uint32_t count =
+                (i >= B_W_FREE && i < B_X_FULL) || (i >= B_READY && i < B_FREE) ||
+                (i >= B_CONV_LR && i < B_EMPTY_LR) || (i >= B_ACC_EMPTY) ? 4u
+                : (i >= B_ACC_FULL && i < B_ACC_EMPTY) ? 2u : 1u;
+            mbar_init(bar(i), count);
         }
-        for (int i = 0; i < 2; ++i) { mbar_init(bar(B_ACC_FULL + i), 2); mbar_init(bar(B_ACC_EMPTY + i), 4); }
-        mbar_init(bar(B_DLR_EMPTY), 4);
-        *abort_flag = 0;
-        *last_flag = 0;
-        *never_flag = 0;
+        if (lane == 0) {
+            *abort_flag = 0;
+            *last_flag = 0;
+            *never_flag = 0;
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async_smem();
+        __syncwarp();
+        asm volatile("barrier.cta.arrive 2, %0;" ::"r"(kThreads) : "memory");
     }
-    // Weight producer state (thread 0).  Its first copies go out before the CTA-wide
-    // synchronisation below: they need only the barriers this thread has just initialised.
+    // Weight producer state (thread 0).
     Cursor wcur;
     wcur.init(u_begin, u_end, p);
     Work ww{};
@@ -411,10 +416,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         if (wkb >= ww.kb1) w_have = false;
         return true;
     };
-    if (threadIdx.x == 0) {
-        for (int i = 0; i < C::NW; ++i)
-            if (!w_issue_one()) break;
-    }
     if (warp == 14 && lane == 0) {
         prefetch_tensormap(&map_x);
         if (p.r > 0) { prefetch_tensormap(&map_lb); prefetch_tensormap(&map_t); }
@@ -425,10 +426,13 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem = *tmem_slot;
+    uint32_t tmem = 0;
+    if (warp != 0) {
+        tc_fence_before();
+        asm volatile("barrier.cta.sync 2, %0;" ::"r"(kThreads) : "memory");
+        tc_fence_after();
+        tmem = *tmem_slot;
+    }
     const uint32_t tm_dint0 = tmem, tm_dlr = tmem + 2 * BT, tm_a0 = tmem + 3 * BT;
     const int lr_chunks = (p.r + 63) / 64;
 
@@ -520,7 +524,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     const int nkb = (w.kb1 - kb < KS) ? (w.kb1 - kb) : KS;
                     const int sa = ca % C::NA, sx = ca % C::NX;   // ca counts stages
                     if ((int)(ca & 1u) != issuer) { ++ca; continue; }
-                    ok = mbar_wait(bar(B_READY + sa), (ca / C::NA) & 1, ab);
+                    ok = mbar_wait(bar(B_READY + sa), (ca / C::NA) & 1, ab) &&
+                         mbar_wait(bar(B_X_FULL + sx), (ca / C::NX) & 1, ab);
                     if (!ok) break;
                     tc_fence_after();
                     const uint64_t xdesc = smem_desc_sw128(sbase + C::OffX + sx * C::XBytes);
@@ -577,7 +582,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         while (ok && next_work(cur, p, w)) {
             for (int kb = w.kb0; kb < w.kb1 && ok; kb += KS) {
                 const int nkb = (w.kb1 - kb < KS) ? (w.kb1 - kb) : KS;
-                const int sw = cw % C::NW, sa = cw % C::NA, sx = cw % C::NX;   // cw counts stages
+                const int sw = cw % C::NW, sa = cw % C::NA;   // cw counts stages
                 if ((int)(cw & 1u) != group) { ++cw; continue; }
                 ok = warp_mbar_wait(bar(B_W_FULL + sw), (cw / C::NW) & 1, ab, lane) &&
                      warp_mbar_wait(bar(B_FREE + sa), ((cw / C::NA) & 1) ^ 1, ab, lane);
@@ -606,9 +611,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 if (lane == 0) mbar_arrive(bar(B_W_FREE + sw));      // it may be refilled
                 tmem_wait_st();
                 tc_fence_before();
-                // one warp of the group also vouches for the activation tile of this stage
-                if (gwarp == 0) ok = warp_mbar_wait(bar(B_X_FULL + sx), (cw / C::NX) & 1, ab, lane);
-                if (!ok) break;
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(B_READY + sa));
                 ++cw;

@@ -668,6 +668,9 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             const int n = w.nt * 128 + nl;
             const bool n_ok = n < p.N;
             const float ws = n_ok ? __ldg(p.w_scale + n) : 0.f;
+            const float ws16 = ws * 0.0625f;
+            const int tok0 = w.tt * BT;
+            const int valid = (p.M - tok0 < BT) ? (p.M - tok0) : BT;   // tokens of this tile inside M
             const uint32_t d_int = tm_dint0 + buf * BT + lane_sel;
             int32_t* pint = p.part_int + ((size_t)cta * 2 + partial_idx) * (BT * 128);
             float* plr = p.part_lr + (size_t)cta * (BT * 128);
@@ -679,16 +682,33 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 tmem_wait_ld(vi);
                 if (w.has_lr) tmem_wait_ld(vf);
                 if (w.whole) {
+                    // The accumulator holds 16 * sum(q x); 1/16 is folded into the scale (exact).
+                    // Straight-line code: one vector load of the token scales, then per column
+                    // convert, fused multiply-add, round to fp16, predicated 2-byte store.
+                    float as[16];
+                    if (c0 + 16 <= valid) {
+                        const float4* ap = reinterpret_cast<const float4*>(p.a_scale + tok0 + c0);
+#pragma unroll
+                        for (int v4 = 0; v4 < 4; ++v4) {
+                            const float4 a4 = __ldg(ap + v4);
+                            as[4 * v4] = a4.x; as[4 * v4 + 1] = a4.y; as[4 * v4 + 2] = a4.z; as[4 * v4 + 3] = a4.w;
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) as[j] = (c0 + j < valid) ? __ldg(p.a_scale + tok0 + c0 + j) : 0.f;
+                    }
+                    const uint32_t row0 = (uint32_t)(tok0 + c0) * (uint32_t)p.N + (uint32_t)n;
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
-                        const int tok = w.tt * BT + c0 + j;
-                        if (tok < p.M && n_ok) {
-                            const int acc = ((int)vi[j]) >> 4;
-                            float y = (float)acc * __ldg(p.a_scale + tok) * ws;
-                            if (w.has_lr) y += __uint_as_float(vf[j]);
-                            p.Y[(size_t)tok * p.N + n] = __float2half_rn(y);
-                            if (p.acc_debug) p.acc_debug[(size_t)tok * p.N + n] = acc;
-                        }
+                        const float lr = w.has_lr ? __uint_as_float(vf[j]) : 0.f;
+                        const float y = fmaf((float)(int)vi[j], as[j] * ws16, lr);
+                        if (c0 + j < valid && n_ok) p.Y[row0 + (uint32_t)j * (uint32_t)p.N] = __float2half_rn(y);
+                    }
+                    if (p.acc_debug) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            if (c0 + j < valid && n_ok)
+                                p.acc_debug[row0 + (uint32_t)j * (uint32_t)p.N] = ((int)vi[j]) >> 4;
                     }
                 } else {
 #pragma unroll
@@ -894,6 +914,7 @@ int launch_linear_tc(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
     Layout L = make_layout(M, N, K, r);
     if (workspace_bytes < L.total) return ASER_ERR_WORKSPACE;
     if (L.units >= (1ll << 31) / kMaxCtas * kMaxCtas) return ASER_ERR_SHAPE;
+    if ((long long)(M + 128) * N >= (1ll << 32)) return ASER_ERR_SHAPE;   // 32-bit element indices in the epilogue
 
     static int num_sms = 0;
     if (num_sms == 0) {

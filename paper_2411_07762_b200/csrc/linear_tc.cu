@@ -47,8 +47,13 @@ struct Cfg {
     // A-operand ring (tensor memory).  All ring depths are even: stages alternate between two
     // unpack groups and two MMA issuers, and a parity wait is only sound if the waiter sees every
     // phase of the barrier, i.e. if a ring slot always belongs to the same group.
-    static constexpr int NA = (BT == 128) ? 2 : 4;
-    static_assert(NA % 2 == 0 && NW % 2 == 0 && NX % 2 == 0, "ring ownership");
+    // An A slot holds KA column blocks.  With 128 tokens only 128 tensor-memory columns are left
+    // for A, so a slot is one block there: each group then still owns two slots and can unpack
+    // one block while the MMAs of the other are in flight.
+    static constexpr int KA = (BT == 128) ? 1 : KS;
+    static constexpr int SPS = KS / KA;                                 // A slots per stage
+    static constexpr int NA = 4;
+    static_assert(NA % (2 * SPS) == 0 && NW % 2 == 0 && NX % 2 == 0, "ring ownership");
     // ring of low-rank chunks (64 columns of r each); one slot where shared memory is tight
     static constexpr int NL = (BT == 128) ? 1 : 2;
     static constexpr int WBytes = KS * kWkBlockBytes;
@@ -63,7 +68,7 @@ struct Cfg {
     static constexpr int OffBar = OffT + NL * TBytes;
     static constexpr int NumBars = 2 * NW + 2 * NX + 2 * NA + 3 * NL + 2 + 2 + 1;
     static constexpr int SmemBytes = OffBar + NumBars * 8 + 64 + 1024;  // + slack for 1 KiB alignment
-    static constexpr int ASlotCols = KS * 32;
+    static constexpr int ASlotCols = KA * 32;
     static constexpr int TmemColsUsed = 3 * BT + NA * ASlotCols;
     static constexpr int TmemCols = TmemColsUsed <= 256 ? 256 : 512;
     static_assert(TmemColsUsed <= 512, "tensor memory budget");
@@ -522,25 +527,32 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 tc_fence_after();
                 for (int kb = w.kb0; kb < w.kb1 && ok; kb += KS) {
                     const int nkb = (w.kb1 - kb < KS) ? (w.kb1 - kb) : KS;
-                    const int sa = ca % C::NA, sx = ca % C::NX;   // ca counts stages
+                    const int sx = ca % C::NX;   // ca counts stages
                     if ((int)(ca & 1u) != issuer) { ++ca; continue; }
-                    ok = mbar_wait(bar(B_READY + sa), (ca / C::NA) & 1, ab) &&
-                         mbar_wait(bar(B_X_FULL + sx), (ca / C::NX) & 1, ab);
+                    ok = mbar_wait(bar(B_X_FULL + sx), (ca / C::NX) & 1, ab);
                     if (!ok) break;
-                    tc_fence_after();
                     const uint64_t xdesc = smem_desc_sw128(sbase + C::OffX + sx * C::XBytes);
-                    const uint32_t a_tm = tm_a0 + sa * C::ASlotCols;
 #pragma unroll
-                    for (int j = 0; j < KS; ++j) {
-                        if (j < nkb) {
+                    for (int sub = 0; sub < C::SPS; ++sub) {
+                        const uint32_t cs = ca * C::SPS + sub;          // running A-slot counter
+                        const int sa = cs % C::NA;
+                        ok = ok && mbar_wait(bar(B_READY + sa), (cs / C::NA) & 1, ab);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint32_t a_tm = tm_a0 + sa * C::ASlotCols;
 #pragma unroll
-                            for (int kk = 0; kk < 4; ++kk)
-                                mma_i8_ts(d_int, a_tm + j * 32 + kk * 8,
-                                          xdesc + (uint64_t)(j * (C::XTile >> 4) + 2 * kk), idesc_i8,
-                                          1u);
+                        for (int jj = 0; jj < C::KA; ++jj) {
+                            const int j = sub * C::KA + jj;
+                            if (j < nkb) {
+#pragma unroll
+                                for (int kk = 0; kk < 4; ++kk)
+                                    mma_i8_ts(d_int, a_tm + jj * 32 + kk * 8,
+                                              xdesc + (uint64_t)(j * (C::XTile >> 4) + 2 * kk), idesc_i8, 1u);
+                            }
                         }
+                        tc_commit(bar(B_FREE + sa));   // an empty slot (ragged last stage) still hands over
                     }
-                    tc_commit(bar(B_FREE + sa));
+                    if (!ok) break;
                     tc_commit(bar(B_X_FREE + sx));
                     ++ca;
                 }
@@ -582,37 +594,47 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         while (ok && next_work(cur, p, w)) {
             for (int kb = w.kb0; kb < w.kb1 && ok; kb += KS) {
                 const int nkb = (w.kb1 - kb < KS) ? (w.kb1 - kb) : KS;
-                const int sw = cw % C::NW, sa = cw % C::NA;   // cw counts stages
+                const int sw = cw % C::NW;   // cw counts stages
                 if ((int)(cw & 1u) != group) { ++cw; continue; }
-                ok = warp_mbar_wait(bar(B_W_FULL + sw), (cw / C::NW) & 1, ab, lane) &&
-                     warp_mbar_wait(bar(B_FREE + sa), ((cw / C::NA) & 1) ^ 1, ab, lane);
+                ok = warp_mbar_wait(bar(B_W_FULL + sw), (cw / C::NW) & 1, ab, lane);
                 if (!ok) break;
-                tc_fence_after();
                 const uint8_t* wsrc = smem + C::OffW + sw * C::WBytes + row * 16;
-                const uint32_t a_tm = tm_a0 + sa * C::ASlotCols + ((uint32_t)(q * 32) << 16);
 #pragma unroll
-                for (int j = 0; j < KS; ++j) {
-                    if (j < nkb) {
-                        uint32_t v[32];
+                for (int sub = 0; sub < C::SPS; ++sub) {
+                    const uint32_t cs = cw * C::SPS + sub;              // running A-slot counter
+                    const int sa = cs % C::NA;
+                    ok = ok && warp_mbar_wait(bar(B_FREE + sa), ((cs / C::NA) & 1) ^ 1, ab, lane);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t a_tm = tm_a0 + sa * C::ASlotCols + ((uint32_t)(q * 32) << 16);
 #pragma unroll
-                        for (int sub = 0; sub < 4; ++sub) {
-                            uint4 x = *reinterpret_cast<const uint4*>(wsrc + j * kWkBlockBytes + sub * 2048);
-                            const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
+                    for (int jj = 0; jj < C::KA; ++jj) {
+                        const int j = sub * C::KA + jj;
+                        if (j < nkb) {
+                            uint32_t v[32];
 #pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                v[sub * 8 + 2 * i] = (xs[i] << 4) & 0xF0F0F0F0u;   // columns c0 .. c0+3
-                                v[sub * 8 + 2 * i + 1] = xs[i] & 0xF0F0F0F0u;      // columns c0+4 .. c0+7
+                            for (int s4 = 0; s4 < 4; ++s4) {
+                                uint4 x = *reinterpret_cast<const uint4*>(wsrc + j * kWkBlockBytes + s4 * 2048);
+                                const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) {
+                                    v[s4 * 8 + 2 * i] = (xs[i] << 4) & 0xF0F0F0F0u;   // columns c0 .. c0+3
+                                    v[s4 * 8 + 2 * i + 1] = xs[i] & 0xF0F0F0F0u;      // columns c0+4 .. c0+7
+                                }
                             }
+                            tmem_st32(a_tm + jj * 32, v);
                         }
-                        tmem_st32(a_tm + j * 32, v);
                     }
+                    if (sub == C::SPS - 1) {
+                        __syncwarp();                                    // all lanes have read the
+                        if (lane == 0) mbar_arrive(bar(B_W_FREE + sw));  // weight slot: refill it
+                    }
+                    tmem_wait_st();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(B_READY + sa));
                 }
-                __syncwarp();                                        // all lanes have read the slot:
-                if (lane == 0) mbar_arrive(bar(B_W_FREE + sw));      // it may be refilled
-                tmem_wait_st();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(B_READY + sa));
+                if (!ok) break;
                 ++cw;
             }
             if (ok && w.has_lr && group == 0) {

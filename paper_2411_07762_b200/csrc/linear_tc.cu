@@ -12,10 +12,11 @@
 // units is cut into equal contiguous ranges, one per CTA; tiles shared by several CTAs are
 // summed through the workspace by whichever CTA arrives last.
 //
-// Warp roles (512 threads): 0 = weight producer, 1 and 15 = MMA issuers for even / odd stages
+// Warp roles (640 threads): 0 = weight producer, 1 and 19 = MMA issuers for even / odd stages
 // (1 also owns the TMEM allocation and issues the low-rank MMAs), 2..5 and 6..9 = two groups of
 // int4 -> int8 unpack warps that take alternate stages (group 0 also converts T),
-// 10..13 = epilogue, 14 = activation and low-rank operand producer.
+// 10..17 = epilogue (two warps per lane quarter, alternate 16-column chunks),
+// 18 = activation and low-rank operand producer.
 // A single lane issues one tcgen05.mma per ~60-85 cycles, which bounds decode shapes (16 MMAs
 // per 32 KiB of weights); the integer accumulation is order-independent, so two lanes share the
 // issue work.  For that the accumulator is zeroed by the epilogue warps (tcgen05.st) when they
@@ -29,7 +30,10 @@ namespace aser {
 
 namespace {
 
-constexpr int kThreads = 512;
+constexpr int kEpiWarps = 8;       // two epilogue warps per tensor-memory lane quarter
+constexpr int kEpiThreads = kEpiWarps * 32;
+constexpr int kWarpXProd = 10 + kEpiWarps, kWarpIssuer1 = 11 + kEpiWarps;
+constexpr int kThreads = (12 + kEpiWarps) * 32;
 constexpr int kMaxCtas = 160;     // upper bound on the persistent grid (workspace sizing)
 constexpr uint32_t kStatusTimeout = 1u;
 constexpr long long kWaitLimitClocks = 4000000000ll;  // about 2 s of SM clocks per wait
@@ -262,11 +266,11 @@ struct Work {
 
 // Units are numbered tile-major: unit = tile * KB + column block.  CTA c owns
 // [range_begin(c), range_begin(c + 1)).  The unit count fits 31 bits (checked on the host).
-__device__ __forceinline__ int range_begin(int units, int c, int G) {
+__device__ __noinline__ int range_begin(int units, int c, int G) {
     return (int)((long long)units * c / G);
 }
 // CTA that owns unit x.
-__device__ __forceinline__ int unit_owner(int units, int x, int G) {
+__device__ __noinline__ int unit_owner(int units, int x, int G) {
     return (int)((((long long)x + 1) * G - 1) / units);
 }
 
@@ -306,24 +310,32 @@ struct Abort {
     uint32_t* status;     // global
 };
 
-// Bounded wait on an mbarrier phase.  Returns false after the time limit or when another role
-// of this CTA has already given up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const Abort& ab) {
+// Slow path of a bounded wait, kept out of line so that the role loops stay small (the kernel
+// runs six different instruction streams per SM and lives or dies by its instruction cache).
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* flag,
+                                            uint32_t* status) {
     uint32_t spins = 0;
     long long t0 = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 255u) == 0) {
-            if (*ab.flag) return false;
+            if (*flag) return false;
             if (t0 == 0) {
                 t0 = clock64();
             } else if (clock64() - t0 > kWaitLimitClocks) {
-                *ab.flag = 1;
-                atomicOr(ab.status, kStatusTimeout);
+                *flag = 1;
+                atomicOr(status, kStatusTimeout);
                 return false;
             }
         }
     }
     return true;
+}
+
+// Bounded wait on an mbarrier phase.  Returns false after the time limit or when another role
+// of this CTA has already given up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const Abort& ab) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, ab.flag, ab.status);
 }
 
 // Warp-collective form: lane 0 polls, the result is broadcast (which also re-converges the
@@ -380,7 +392,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         for (int i = lane; i < C::NumBars; i += 32) {
             const uint32_t count =
                 (i >= B_W_FREE && i < B_X_FULL) || (i >= B_READY && i < B_FREE) ||
-                (i >= B_CONV_LR && i < B_EMPTY_LR) || (i >= B_ACC_EMPTY) ? 4u
+                (i >= B_CONV_LR && i < B_EMPTY_LR) ? 4u
+                : (i >= B_ACC_EMPTY) ? (uint32_t)kEpiWarps
                 : (i >= B_ACC_FULL && i < B_ACC_EMPTY) ? 2u : 1u;
             mbar_init(bar(i), count);
         }
@@ -421,7 +434,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         if (wkb >= ww.kb1) w_have = false;
         return true;
     };
-    if (warp == 14 && lane == 0) {
+    if (warp == kWarpXProd && lane == 0) {
         prefetch_tensormap(&map_x);
         if (p.r > 0) { prefetch_tensormap(&map_lb); prefetch_tensormap(&map_t); }
     }
@@ -453,7 +466,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     mbar_wait(bar(B_W_FULL + i % C::NW), (i / C::NW) & 1, Abort{never_flag, p.status});
             }
         }
-    } else if (warp == 14) {
+    } else if (warp == kWarpXProd) {
         // =================== activation + low-rank operand producer (one lane) ===================
         if (lane == 0) {
             Cursor cur;
@@ -507,7 +520,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     mbar_wait(bar(B_X_FULL + i % C::NX), (i / C::NX) & 1, Abort{never_flag, p.status});
             }
         }
-    } else if (warp == 1 || warp == 15) {
+    } else if (warp == 1 || warp == kWarpIssuer1) {
         // =================== MMA issuers (one lane each; even / odd stages) ===================
         const int issuer = (warp == 1) ? 0 : 1;
         if (lane == 0) {
@@ -663,11 +676,13 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 }
             }
         }
-    } else if (warp < 14) {
+    } else if (warp < 10 + kEpiWarps) {
         // =================== epilogue warps ===================
         const int q = warp & 3;
         const int nl = q * 32 + lane;              // row of D = output channel inside the tile
-        const int et = (warp - 10) * 32 + lane;     // 0..127 among the epilogue threads
+        const int et = (warp - 10) * 32 + lane;     // index among the epilogue threads
+        const int half = (warp - 10) >> 2;          // which of the quarter's two warps: it takes
+        constexpr int kChunkStep = 16 * (kEpiWarps / 4);   // every other 16-column chunk
         const uint32_t lane_sel = (uint32_t)(q * 32) << 16;
         Cursor cur;
         cur.init(u_begin, u_end, p);
@@ -676,7 +691,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         int partial_idx = 0;                       // 0: first partial item of this CTA, 1: second
         bool ok = true;
         // both integer accumulators start at zero: every integer MMA accumulates
-        for (int c0 = 0; c0 < 2 * BT; c0 += 16) tmem_zero16(tm_dint0 + lane_sel + c0);
+        for (int c0 = 16 * half; c0 < 2 * BT; c0 += kChunkStep) tmem_zero16(tm_dint0 + lane_sel + c0);
         tmem_wait_st();
         tc_fence_before();
         __syncwarp();
@@ -684,7 +699,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         while (ok && next_work(cur, p, w)) {
             const int buf = ci & 1;
             ok = warp_mbar_wait(bar(B_ACC_FULL + buf), (ci >> 1) & 1, ab, lane);
-            ok = named_bar_all(1, 128, ok);   // the 128 epilogue threads go on or give up together
+            ok = named_bar_all(1, kEpiThreads, ok);   // the 128 epilogue threads go on or give up together
             if (!ok) break;
             tc_fence_after();
             const int n = w.nt * 128 + nl;
@@ -697,7 +712,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             int32_t* pint = p.part_int + ((size_t)cta * 2 + partial_idx) * (BT * 128);
             float* plr = p.part_lr + (size_t)cta * (BT * 128);
 #pragma unroll 1
-            for (int c0 = 0; c0 < BT; c0 += 16) {
+            for (int c0 = 16 * half; c0 < BT; c0 += kChunkStep) {
                 uint32_t vi[16], vf[16];
                 tmem_ld16(d_int + c0, vi);
                 if (w.has_lr) tmem_ld16(tm_dlr + lane_sel + c0, vf);
@@ -740,7 +755,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     }
                 }
             }
-            for (int c0 = 0; c0 < BT; c0 += 16) tmem_zero16(d_int + c0);   // hand it back zeroed
+            for (int c0 = 16 * half; c0 < BT; c0 += kChunkStep) tmem_zero16(d_int + c0);   // hand it back zeroed
             tmem_wait_st();
             tc_fence_before();
             __syncwarp();
@@ -755,29 +770,29 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 const int first_unit = w.tile * p.KB;
                 const int c_first = unit_owner(p.units, first_unit, G);
                 const int c_last = unit_owner(p.units, first_unit + p.KB - 1, G);
-                named_bar_sync(1, 128);            // every partial store of this CTA precedes ...
+                named_bar_sync(1, kEpiThreads);            // every partial store of this CTA precedes ...
                 if (et == 0) {                     // ... this release; the last arriver acquires all
                     int old;
                     asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;"
                                  : "=r"(old) : "l"(p.counters + w.tile) : "memory");
                     *last_flag = (old == c_last - c_first) ? 1 : 0;
                 }
-                named_bar_sync(1, 128);
+                named_bar_sync(1, kEpiThreads);
                 const bool last = *last_flag != 0;
-                named_bar_sync(1, 128);           // everyone has read the flag before it is reused
+                named_bar_sync(1, kEpiThreads);           // everyone has read the flag before it is reused
                 if (last) {
                     if (et == 0) p.counters[w.tile] = 0;   // ready for the next launch
 #pragma unroll 1
-                    for (int c0 = 0; c0 < BT; c0 += 16) {
+                    for (int c0 = 16 * half; c0 < BT; c0 += kChunkStep) {
                         if (w.tt * BT + c0 >= p.M) break;
                         int sum[16];
 #pragma unroll
                         for (int j = 0; j < 16; ++j) sum[j] = 0;
-                        for (int cb = c_first; cb <= c_last; cb += 4) {
-                            // four contributors' loads in flight at a time
-                            int v[4][16];
+                        for (int cb = c_first; cb <= c_last; cb += 2) {
+                            // two contributors' loads in flight at a time
+                            int v[2][16];
 #pragma unroll
-                            for (int u = 0; u < 4; ++u) {
+                            for (int u = 0; u < 2; ++u) {
                                 const int c = cb + u;
                                 if (c <= c_last) {
                                     // CTA c's items in order: a tile cut off at the start of its
@@ -793,7 +808,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                                 }
                             }
 #pragma unroll
-                            for (int u = 0; u < 4; ++u)
+                            for (int u = 0; u < 2; ++u)
 #pragma unroll
                                 for (int j = 0; j < 16; ++j) sum[j] += v[u][j];
                         }

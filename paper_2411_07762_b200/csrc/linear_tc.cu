@@ -30,10 +30,6 @@ namespace aser {
 
 namespace {
 
-constexpr int kEpiWarps = 8;       // two epilogue warps per tensor-memory lane quarter
-constexpr int kEpiThreads = kEpiWarps * 32;
-constexpr int kWarpXProd = 10 + kEpiWarps, kWarpIssuer1 = 11 + kEpiWarps;
-constexpr int kThreads = (12 + kEpiWarps) * 32;
 constexpr int kMaxCtas = 160;     // upper bound on the persistent grid (workspace sizing)
 constexpr uint32_t kStatusTimeout = 1u;
 constexpr long long kWaitLimitClocks = 4000000000ll;  // about 2 s of SM clocks per wait
@@ -45,6 +41,11 @@ constexpr long long kWaitLimitClocks = 4000000000ll;  // about 2 s of SM clocks 
 // byte) and the unpack work alternates between two groups of four warps.
 template <int BT>
 struct Cfg {
+    // Epilogue warps: one per tensor-memory lane quarter, two where a tile has many columns.
+    static constexpr int EW = (BT >= 64) ? 8 : 4;
+    static constexpr int EpiThreads = EW * 32;
+    static constexpr int WarpXProd = 10 + EW, WarpIssuer1 = 11 + EW;
+    static constexpr int Threads = (12 + EW) * 32;
     static constexpr int KS = 2;
     static constexpr int NW = (BT == 128) ? 4 : (BT == 64 ? 6 : 8);     // weight ring depth (even)
     static constexpr int NX = 4;                                        // activation ring depth
@@ -346,11 +347,21 @@ __device__ __forceinline__ bool warp_mbar_wait(uint32_t bar, uint32_t parity, co
     return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 
+// Group-collective form for a 128-thread unpack group: a single lane polls the mbarrier and the
+// outcome is spread by a hardware named barrier.  Keeps the mbarrier traffic of a group at one
+// wait per event instead of four.
+__device__ __forceinline__ bool group_mbar_wait(uint32_t bar, uint32_t parity, const Abort& ab,
+                                                bool leader, int bar_id) {
+    bool ok = true;
+    if (leader) ok = mbar_wait(bar, parity, ab);
+    return named_bar_all(bar_id, 128, ok);
+}
+
 // ---------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------
 template <int BT>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(Cfg<BT>::Threads, 1)
 linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_lb,
                  const __grid_constant__ CUtensorMap map_t, const Params p) {
     using C = Cfg<BT>;
@@ -391,9 +402,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     if (warp == 0) {
         for (int i = lane; i < C::NumBars; i += 32) {
             const uint32_t count =
-                (i >= B_W_FREE && i < B_X_FULL) || (i >= B_READY && i < B_FREE) ||
-                (i >= B_CONV_LR && i < B_EMPTY_LR) ? 4u
-                : (i >= B_ACC_EMPTY) ? (uint32_t)kEpiWarps
+                (i >= B_ACC_EMPTY) ? (uint32_t)C::EW
                 : (i >= B_ACC_FULL && i < B_ACC_EMPTY) ? 2u : 1u;
             mbar_init(bar(i), count);
         }
@@ -405,7 +414,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async_smem();
         __syncwarp();
-        asm volatile("barrier.cta.arrive 2, %0;" ::"r"(kThreads) : "memory");
+        asm volatile("barrier.cta.arrive 2, %0;" ::"r"(C::Threads) : "memory");
     }
     // Weight producer state (thread 0).
     Cursor wcur;
@@ -434,7 +443,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         if (wkb >= ww.kb1) w_have = false;
         return true;
     };
-    if (warp == kWarpXProd && lane == 0) {
+    if (warp == C::WarpXProd && lane == 0) {
         prefetch_tensormap(&map_x);
         if (p.r > 0) { prefetch_tensormap(&map_lb); prefetch_tensormap(&map_t); }
     }
@@ -447,7 +456,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     uint32_t tmem = 0;
     if (warp != 0) {
         tc_fence_before();
-        asm volatile("barrier.cta.sync 2, %0;" ::"r"(kThreads) : "memory");
+        asm volatile("barrier.cta.sync 2, %0;" ::"r"(C::Threads) : "memory");
         tc_fence_after();
         tmem = *tmem_slot;
     }
@@ -466,7 +475,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     mbar_wait(bar(B_W_FULL + i % C::NW), (i / C::NW) & 1, Abort{never_flag, p.status});
             }
         }
-    } else if (warp == kWarpXProd) {
+    } else if (warp == C::WarpXProd) {
         // =================== activation + low-rank operand producer (one lane) ===================
         if (lane == 0) {
             Cursor cur;
@@ -520,7 +529,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     mbar_wait(bar(B_X_FULL + i % C::NX), (i / C::NX) & 1, Abort{never_flag, p.status});
             }
         }
-    } else if (warp == 1 || warp == kWarpIssuer1) {
+    } else if (warp == 1 || warp == C::WarpIssuer1) {
         // =================== MMA issuers (one lane each; even / odd stages) ===================
         const int issuer = (warp == 1) ? 0 : 1;
         if (lane == 0) {
@@ -599,6 +608,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         const int group = (warp - 2) >> 2;         // stages alternate between the two groups
         const int gwarp = (warp - 2) & 3;          // warp within its group
         const int t128 = gwarp * 32 + lane;        // 0..127 within the group
+        const bool leader = (t128 == 0);           // polls and signals the mbarriers for the group
+        const int gbar = 3 + group;                // hardware named barrier of the group
         Cursor cur;
         cur.init(u_begin, u_end, p);
         Work w;
@@ -609,14 +620,14 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 const int nkb = (w.kb1 - kb < KS) ? (w.kb1 - kb) : KS;
                 const int sw = cw % C::NW;   // cw counts stages
                 if ((int)(cw & 1u) != group) { ++cw; continue; }
-                ok = warp_mbar_wait(bar(B_W_FULL + sw), (cw / C::NW) & 1, ab, lane);
+                ok = group_mbar_wait(bar(B_W_FULL + sw), (cw / C::NW) & 1, ab, leader, gbar);
                 if (!ok) break;
                 const uint8_t* wsrc = smem + C::OffW + sw * C::WBytes + row * 16;
 #pragma unroll
                 for (int sub = 0; sub < C::SPS; ++sub) {
                     const uint32_t cs = cw * C::SPS + sub;              // running A-slot counter
                     const int sa = cs % C::NA;
-                    ok = ok && warp_mbar_wait(bar(B_FREE + sa), ((cs / C::NA) & 1) ^ 1, ab, lane);
+                    ok = ok && group_mbar_wait(bar(B_FREE + sa), ((cs / C::NA) & 1) ^ 1, ab, leader, gbar);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t a_tm = tm_a0 + sa * C::ASlotCols + ((uint32_t)(q * 32) << 16);
@@ -638,14 +649,14 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                             tmem_st32(a_tm + jj * 32, v);
                         }
                     }
-                    if (sub == C::SPS - 1) {
-                        __syncwarp();                                    // all lanes have read the
-                        if (lane == 0) mbar_arrive(bar(B_W_FREE + sw));  // weight slot: refill it
-                    }
                     tmem_wait_st();
                     tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar(B_READY + sa));
+                    named_bar_sync(gbar, 128);          // the whole group has written its rows
+                    if (leader) {
+                        mbar_arrive(bar(B_READY + sa));
+                        // ... and, after the last block, has the weight slot in registers: refill it
+                        if (sub == C::SPS - 1) mbar_arrive(bar(B_W_FREE + sw));
+                    }
                 }
                 if (!ok) break;
                 ++cw;
@@ -653,7 +664,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             if (ok && w.has_lr && group == 0) {
                 for (int c = 0; c < lr_chunks && ok; ++c) {
                     const int s = cl % C::NL;
-                    ok = warp_mbar_wait(bar(B_FULL_LR + s), (cl / C::NL) & 1, ab, lane);
+                    ok = group_mbar_wait(bar(B_FULL_LR + s), (cl / C::NL) & 1, ab, leader, gbar);
                     if (!ok) break;
                     // T chunk: bf16 -> fp16 in place (same element size, same swizzled position)
                     uint8_t* tb = smem + C::OffT + s * C::TBytes;
@@ -670,19 +681,19 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                         *reinterpret_cast<uint4*>(tb + i * 16) = make_uint4(out[0], out[1], out[2], out[3]);
                     }
                     fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar(B_CONV_LR + s));
+                    named_bar_sync(gbar, 128);
+                    if (leader) mbar_arrive(bar(B_CONV_LR + s));
                     ++cl;
                 }
             }
         }
-    } else if (warp < 10 + kEpiWarps) {
+    } else if (warp < 10 + C::EW) {
         // =================== epilogue warps ===================
         const int q = warp & 3;
         const int nl = q * 32 + lane;              // row of D = output channel inside the tile
         const int et = (warp - 10) * 32 + lane;     // index among the epilogue threads
         const int half = (warp - 10) >> 2;          // which of the quarter's two warps: it takes
-        constexpr int kChunkStep = 16 * (kEpiWarps / 4);   // every other 16-column chunk
+        constexpr int kChunkStep = 16 * (C::EW / 4);   // every other 16-column chunk
         const uint32_t lane_sel = (uint32_t)(q * 32) << 16;
         Cursor cur;
         cur.init(u_begin, u_end, p);
@@ -699,7 +710,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         while (ok && next_work(cur, p, w)) {
             const int buf = ci & 1;
             ok = warp_mbar_wait(bar(B_ACC_FULL + buf), (ci >> 1) & 1, ab, lane);
-            ok = named_bar_all(1, kEpiThreads, ok);   // the 128 epilogue threads go on or give up together
+            ok = named_bar_all(1, C::EpiThreads, ok);   // the 128 epilogue threads go on or give up together
             if (!ok) break;
             tc_fence_after();
             const int n = w.nt * 128 + nl;
@@ -770,16 +781,16 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 const int first_unit = w.tile * p.KB;
                 const int c_first = unit_owner(p.units, first_unit, G);
                 const int c_last = unit_owner(p.units, first_unit + p.KB - 1, G);
-                named_bar_sync(1, kEpiThreads);            // every partial store of this CTA precedes ...
+                named_bar_sync(1, C::EpiThreads);            // every partial store of this CTA precedes ...
                 if (et == 0) {                     // ... this release; the last arriver acquires all
                     int old;
                     asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;"
                                  : "=r"(old) : "l"(p.counters + w.tile) : "memory");
                     *last_flag = (old == c_last - c_first) ? 1 : 0;
                 }
-                named_bar_sync(1, kEpiThreads);
+                named_bar_sync(1, C::EpiThreads);
                 const bool last = *last_flag != 0;
-                named_bar_sync(1, kEpiThreads);           // everyone has read the flag before it is reused
+                named_bar_sync(1, C::EpiThreads);           // everyone has read the flag before it is reused
                 if (last) {
                     if (et == 0) p.counters[w.tile] = 0;   // ready for the next launch
 #pragma unroll 1
@@ -928,7 +939,7 @@ int launch_bt(const CUtensorMap& mx, const CUtensorMap& mlb, const CUtensorMap& 
         if (e != cudaSuccess) return record_cuda_error(e, "linear_tc smem attribute");
         configured = true;
     }
-    linear_tc_kernel<BT><<<grid, kThreads, C::SmemBytes, st>>>(mx, mlb, mt, p);
+    linear_tc_kernel<BT><<<grid, C::Threads, C::SmemBytes, st>>>(mx, mlb, mt, p);
     return check_launch("linear_tc_kernel");
 }
 

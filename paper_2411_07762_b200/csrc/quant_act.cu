@@ -32,9 +32,17 @@ __device__ __forceinline__ RawChunk load_raw(const __half* xrow, const float* s,
     return rc;
 }
 
-// x~ = fp32(x) / s, one IEEE division each.
+// x~ = fp32(x) / s, one IEEE division each.  Dividing by 1 is the identity, and s is 1 on all
+// but the few outlier channels, so the (long) division sequence is skipped for such groups.
 __device__ __forceinline__ void smooth8(const RawChunk& rc, float (&v)[8]) {
     const __half* h = reinterpret_cast<const __half*>(&rc.x);
+    const bool ones = rc.s0.x == 1.f && rc.s0.y == 1.f && rc.s0.z == 1.f && rc.s0.w == 1.f &&
+                      rc.s1.x == 1.f && rc.s1.y == 1.f && rc.s1.z == 1.f && rc.s1.w == 1.f;
+    if (ones) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = __half2float(h[i]);
+        return;
+    }
     v[0] = __fdiv_rn(__half2float(h[0]), rc.s0.x); v[1] = __fdiv_rn(__half2float(h[1]), rc.s0.y);
     v[2] = __fdiv_rn(__half2float(h[2]), rc.s0.z); v[3] = __fdiv_rn(__half2float(h[3]), rc.s0.w);
     v[4] = __fdiv_rn(__half2float(h[4]), rc.s1.x); v[5] = __fdiv_rn(__half2float(h[5]), rc.s1.y);
@@ -42,12 +50,22 @@ __device__ __forceinline__ void smooth8(const RawChunk& rc, float (&v)[8]) {
 }
 
 // Eight int8 codes rne(x~ / scale) clamped to +-127, packed low column first.
+// The definition uses the IEEE quotient.  |x~ / scale| <= 127 (1 + 2^-23), so x~ * (1/scale)
+// differs from the rounded quotient by less than 4 * 2^-24 * 127 < 3.1e-5: whenever that product
+// is at least 1e-4 away from every half-integer, both round to the same integer and the
+// multiplication stands in for the division.  Only the rare near-ties take the real division.
 __device__ __forceinline__ uint2 quant8(const float (&v)[8], float sc, bool nonzero) {
     uint32_t w[2] = {0, 0};
+    const float rcp = nonzero ? __frcp_rn(sc) : 0.f;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         int q = 0;
-        if (nonzero) q = rne_clamp(__fdiv_rn(v[i], sc), -127.f, 127.f);
+        if (nonzero) {
+            const float t = v[i] * rcp;
+            const float fr = fabsf(t) - floorf(fabsf(t));          // fractional part in [0, 1)
+            if (fabsf(fr - 0.5f) >= 1e-4f && fabsf(t) < 1e6f) q = rne_clamp(t, -127.f, 127.f);
+            else q = rne_clamp(__fdiv_rn(v[i], sc), -127.f, 127.f);
+        }
         w[i >> 2] |= (uint32_t)(q & 0xFF) << (8 * (i & 3));
     }
     return make_uint2(w[0], w[1]);
@@ -302,6 +320,263 @@ quant_act_large_kernel(const __half* __restrict__ X, const float* __restrict__ s
     }
 }
 
+// ---------------------------------------------------------------------------
+// many tokens, single pass over X: thread-block cluster split along K
+// ---------------------------------------------------------------------------
+// A cluster of CK CTAs owns 32 tokens; CTA `rank` owns the K-slice [rank*Kc, (rank+1)*Kc) with
+// Kc <= 2048, small enough to keep the raw fp16 activations of the slice in shared memory.
+// Sweep 1 (per 64-column chunk): x~ = x / s, row absmax, x~ rounded to fp16 and multiplied with
+// the L_A chunk on the tensor cores.  Then the CTAs exchange row maxima and partial T through
+// distributed shared memory, and sweep 2 quantizes the resident slice, so X is read from HBM
+// exactly once and L_A is re-read once per 32 tokens.
+constexpr int kCTok = 32;                   // tokens per cluster
+constexpr int kCThreads = 512;              // 16 threads per token row; 16 warps hide latencies
+constexpr int kCChunk = 128;                // columns per pipeline step
+constexpr int kCRow = kCChunk * 2 + 16;     // padded row of a staged fp16 chunk (272 B)
+// L_A chunks in flight: as many as shared memory allows beside the resident activations
+__host__ __device__ constexpr int cluster_stages(int r) { return r <= 64 ? 3 : 2; }
+
+struct ClusterSmem {
+    int x_raw, s_vec, a_stage, la_stage, t_part, amax_part, scale, total;
+};
+__host__ __device__ inline ClusterSmem cluster_smem(int Kc, int r) {
+    ClusterSmem L;
+    int off = 0;
+    L.x_raw = off;      off += kCTok * (Kc * 2 + 16);          // raw fp16 activations (padded rows)
+    L.s_vec = off;      off += Kc * 4;                         // smoothing divisors of the slice
+    L.a_stage = off;    off += 2 * kCTok * kCRow;              // x~ as fp16, double buffered
+    L.la_stage = off;                                          // L_A chunks; afterwards this CTA's
+    L.t_part = off;                                            // partial T (fp32) reuses the space
+    {
+        const int la = cluster_stages(r) * r * kCRow, tp = kCTok * r * 4;
+        off += (la > tp ? la : tp) + 16;
+    }
+    L.amax_part = off;  off += kCTok * 4;
+    L.scale = off;      off += kCTok * 4;
+    L.total = off;
+    return L;
+}
+
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Read a float from the same shared-memory offset in CTA `rank` of the cluster.
+__device__ __forceinline__ float dsmem_ld_f32(uint32_t local_addr, uint32_t rank) {
+    uint32_t remote;
+    float v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
+    return v;
+}
+
+// grid = (CK, ceil(M / 32)), cluster = (CK, 1, 1).  NTW = 8-column tiles of T per warp,
+// STG = L_A pipeline depth (cluster_stages(r)).
+template <int NTW, int STG>
+__global__ void __launch_bounds__(kCThreads)
+quant_act_cluster_kernel(const __half* __restrict__ X, const float* __restrict__ s,
+                         const __half* __restrict__ LA, int M, int K, int Kc, int r, int CK,
+                         int8_t* __restrict__ Xq, float* __restrict__ a_scale,
+                         __nv_bfloat16* __restrict__ T) {
+    extern __shared__ __align__(16) uint8_t smem[];
+    const ClusterSmem L = cluster_smem(Kc, r);
+    const int xrow_bytes = Kc * 2 + 16;            // padded: rows of a warp fall in different banks
+    const uint32_t sb = (uint32_t)__cvta_generic_to_shared(smem);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t rank = cluster_rank();
+    const int m0 = blockIdx.y * kCTok;
+    const int k0 = (int)rank * Kc;
+    const int nch = Kc / kCChunk;
+    const int trow = tid >> 4, tcg = tid & 15;     // this thread's token row and 8-column group
+    const bool row_ok = m0 + trow < M;
+    float* s_sm = reinterpret_cast<float*>(smem + L.s_vec);
+    float* t_part = reinterpret_cast<float*>(smem + L.t_part);
+    float* amax_part = reinterpret_cast<float*>(smem + L.amax_part);
+    float* scale_sm = reinterpret_cast<float*>(smem + L.scale);
+
+    // smoothing divisors of the slice (plain loads; ones when s is absent)
+    for (int i = tid; i < Kc; i += kCThreads) s_sm[i] = s ? s[k0 + i] : 1.f;
+
+    // Activations go to their final place, so they can be requested far ahead of use (the L_A
+    // ring cannot): kXAhead chunks = 64 KiB in flight per SM, what an HBM-bound stream needs.
+    constexpr int kXAhead = 8;
+    auto issue_x = [&](int c) {
+        // 32 rows x 256 B, one 16-byte copy per thread (zero rows past M)
+        const uint32_t xdst = sb + L.x_raw + trow * xrow_bytes + c * (kCChunk * 2) + tcg * 16;
+        if (row_ok) cp_async16(xdst, X + (size_t)(m0 + trow) * K + k0 + c * kCChunk + tcg * 8);
+        else *reinterpret_cast<uint4*>(smem + L.x_raw + trow * xrow_bytes + c * (kCChunk * 2) + tcg * 16) = make_uint4(0, 0, 0, 0);
+    };
+    auto issue_chunk = [&](int c) {
+        if (c + kXAhead < nch) issue_x(c + kXAhead);
+        // L_A chunk: r rows x 256 B
+        const uint32_t ldst = sb + L.la_stage + (c % STG) * r * kCRow;
+        for (int i = tid; i < r * 16; i += kCThreads) {
+            const int j = i >> 4, cc = i & 15;
+            cp_async16(ldst + j * kCRow + cc * 16, LA + (size_t)j * K + k0 + c * kCChunk + cc * 8);
+        }
+    };
+
+    float acc[NTW][4];
+#pragma unroll
+    for (int i = 0; i < NTW; ++i)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[i][e] = 0.f;
+    const int mt = warp & 1, nq = warp >> 1;
+    const int ntiles = r / 8;
+
+    for (int c = 0; c < kXAhead && c < nch; ++c) issue_x(c);   // joins the first commit group
+    for (int c = 0; c < STG - 1; ++c) {
+        if (c < nch) issue_chunk(c);
+        cp_async_commit();
+    }
+    float amax = 0.f;
+    for (int c = 0; c < nch; ++c) {
+        cp_async_wait<STG - 2>();      // chunk c has landed (for this thread's copies)
+        __syncthreads();                    // ... and for everyone's; chunk c-1 is fully consumed
+        if (c + STG - 1 < nch) issue_chunk(c + STG - 1);   // refills the stage of chunk c-1
+        cp_async_commit();
+        // x~ for this thread's 8 columns
+        {
+            const uint4 raw = *reinterpret_cast<const uint4*>(smem + L.x_raw + trow * xrow_bytes + c * (kCChunk * 2) + tcg * 16);
+            const float4 s0 = *reinterpret_cast<const float4*>(s_sm + c * kCChunk + tcg * 8);
+            const float4 s1 = *reinterpret_cast<const float4*>(s_sm + c * kCChunk + tcg * 8 + 4);
+            RawChunk rc{raw, s0, s1};
+            float v[8];
+            smooth8(rc, v);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(v[i]));
+            if (r > 0) {
+                __half2 p0 = __floats2half2_rn(v[0], v[1]), p1 = __floats2half2_rn(v[2], v[3]);
+                __half2 p2 = __floats2half2_rn(v[4], v[5]), p3 = __floats2half2_rn(v[6], v[7]);
+                uint4 pk;
+                pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
+                pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
+                *reinterpret_cast<uint4*>(smem + L.a_stage + (c & 1) * kCTok * kCRow + trow * kCRow + tcg * 16) = pk;
+            }
+        }
+        if (r > 0) {
+            __syncthreads();
+            const uint32_t a_base = sb + L.a_stage + (c & 1) * kCTok * kCRow + (mt * 16 + (lane & 15)) * kCRow + (lane >> 4) * 16;
+            const uint32_t b_base = sb + L.la_stage + (c % STG) * r * kCRow + (lane & 7) * kCRow + (lane >> 3) * 16;
+#pragma unroll
+            for (int kk = 0; kk < kCChunk / 32; ++kk) {
+                uint32_t a0, a1, a2, a3, a4, a5, a6, a7;
+                ldmatrix_x4(a_base + kk * 64, a0, a1, a2, a3);
+                ldmatrix_x4(a_base + kk * 64 + 32, a4, a5, a6, a7);
+#pragma unroll
+                for (int i = 0; i < NTW; ++i) {
+                    const int nt = nq + 8 * i;
+                    if (nt < ntiles) {
+                        uint32_t b0, b1, b2, b3;
+                        ldmatrix_x4(b_base + nt * 8 * kCRow + kk * 64, b0, b1, b2, b3);
+                        mma_f16(acc[i], a0, a1, a2, a3, b0, b1);
+                        mma_f16(acc[i], a4, a5, a6, a7, b2, b3);
+                    }
+                }
+            }
+        }
+    }
+    cp_async_wait<0>();
+    __syncthreads();        // every warp is done with the L_A stages: their space now holds T
+
+    // ---- publish this CTA's partial results for the cluster ----
+    // row maximum over this thread's 8-column groups: the 16 threads of a row are adjacent lanes
+#pragma unroll
+    for (int o = 8; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    if (tcg == 0) amax_part[trow] = amax;
+    if (r > 0) {
+        const int g = lane >> 2, tq = lane & 3;
+#pragma unroll
+        for (int i = 0; i < NTW; ++i) {
+            const int nt = nq + 8 * i;
+            if (nt < ntiles) {
+                const int j = nt * 8 + tq * 2;
+                *reinterpret_cast<float2*>(t_part + (mt * 16 + g) * r + j) = make_float2(acc[i][0], acc[i][1]);
+                *reinterpret_cast<float2*>(t_part + (mt * 16 + g + 8) * r + j) = make_float2(acc[i][2], acc[i][3]);
+            }
+        }
+    }
+    cluster_sync_all();
+
+    // ---- row scales: maximum over the K-slices (every CTA needs them for its own slice) ----
+    if (tid < kCTok) {
+        float a = 0.f;
+        for (int q = 0; q < CK; ++q) a = fmaxf(a, dsmem_ld_f32(sb + L.amax_part + tid * 4, q));
+        const float sc = __fdiv_rn(a, 127.0f);
+        scale_sm[tid] = sc;
+        if (rank == 0 && m0 + tid < M) a_scale[m0 + tid] = sc;
+    }
+    // ---- T: sum of the partial products; the cluster's CTAs share the elements ----
+    if (r > 0) {
+        for (int e = (int)rank * kCThreads + tid; e < kCTok * r; e += CK * kCThreads) {
+            float sum = 0.f;
+            for (int q = 0; q < CK; ++q) sum += dsmem_ld_f32(sb + L.t_part + e * 4, q);
+            const int row = e / r, j = e - row * r;
+            if (m0 + row < M) T[(size_t)(m0 + row) * r + j] = __float2bfloat16_rn(sum);
+        }
+    }
+    cluster_sync_all();      // nobody leaves (or reuses shared memory) while peers still read it
+
+    // ---- sweep 2: int8 codes of the resident slice ----
+    if (!row_ok) return;
+    const float sc = scale_sm[trow];
+    int8_t* out = Xq + (size_t)(m0 + trow) * K + k0;
+    for (int c = 0; c < nch; ++c) {
+        const uint4 raw = *reinterpret_cast<const uint4*>(smem + L.x_raw + trow * xrow_bytes + c * (kCChunk * 2) + tcg * 16);
+        const float4 s0 = *reinterpret_cast<const float4*>(s_sm + c * kCChunk + tcg * 8);
+        const float4 s1 = *reinterpret_cast<const float4*>(s_sm + c * kCChunk + tcg * 8 + 4);
+        RawChunk rc{raw, s0, s1};
+        float v[8];
+        smooth8(rc, v);
+        *reinterpret_cast<uint2*>(out + c * kCChunk + tcg * 8) = quant8(v, sc, sc > 0.f);
+    }
+}
+
+// Smallest cluster size (<= 8) whose K-slice fits shared memory and is a whole number of chunks.
+int pick_cluster(int K, int r) {
+    for (int ck = 1; ck <= 8; ++ck) {
+        if (K % ck) continue;
+        const int kc = K / ck;
+        if (kc % kCChunk) continue;
+        if (cluster_smem(kc, r).total <= 226 * 1024 && kc <= 2048) return ck;
+    }
+    return 0;
+}
+
+template <int NTW, int STG>
+int launch_cluster(const __half* X, const float* s, const __half* LA, int M, int K, int r, int ck,
+                   int8_t* Xq, float* a_scale, __nv_bfloat16* T, cudaStream_t st) {
+    const int kc = K / ck;
+    const size_t smem = (size_t)cluster_smem(kc, r).total;
+    static size_t configured = 0;
+    if (smem > configured) {
+        cudaError_t e = cudaFuncSetAttribute(quant_act_cluster_kernel<NTW, STG>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return record_cuda_error(e, "quant_act_cluster smem attribute");
+        configured = smem;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(ck, (M + kCTok - 1) / kCTok, 1);
+    cfg.blockDim = dim3(kCThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = ck;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, quant_act_cluster_kernel<NTW, STG>, X, s, LA, M, K, kc, r, ck,
+                                       Xq, a_scale, T);
+    if (e != cudaSuccess) return record_cuda_error(e, "quant_act_cluster_kernel");
+    return check_launch("quant_act_cluster_kernel");
+}
+
 template <int MAXT>
 int launch_large(const __half* X, const float* s, const __half* LA, int M, int K, int r,
                  int8_t* Xq, float* a_scale, __nv_bfloat16* T, cudaStream_t st) {
@@ -335,6 +610,12 @@ int launch_quant_act(const __half* X, const float* s, const __half* LA, int M, i
         dim3 grid(1 + (r + kRowsPerCta - 1) / kRowsPerCta, M);
         quant_act_small_kernel<<<grid, kSmallThreads, smem, st>>>(X, s, LA, M, K, r, Xq, a_scale, T);
         return check_launch("quant_act_small_kernel");
+    }
+    const int ck = pick_cluster(K, r);
+    if (ck > 0 && (long long)((M + kCTok - 1) / kCTok) <= 65535) {
+        if (r <= 64) return launch_cluster<1, 3>(X, s, LA, M, K, r, ck, Xq, a_scale, T, st);
+        if (r <= 128) return launch_cluster<2, 2>(X, s, LA, M, K, r, ck, Xq, a_scale, T, st);
+        return launch_cluster<4, 2>(X, s, LA, M, K, r, ck, Xq, a_scale, T, st);
     }
     if (r <= 64) return launch_large<1>(X, s, LA, M, K, r, Xq, a_scale, T, st);
     if (r <= 128) return launch_large<2>(X, s, LA, M, K, r, Xq, a_scale, T, st);

@@ -71,6 +71,28 @@ __device__ __forceinline__ uint2 quant8(const float (&v)[8], float sc, bool nonz
     return make_uint2(w[0], w[1]);
 }
 
+// d = bytes [lo0, lo1, hi0, hi1] as saturated int8 (two pack instructions per four codes).
+__device__ __forceinline__ uint32_t pack4_s8(int q0, int q1, int q2, int q3) {
+    uint32_t hi, out;
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(q3), "r"(q2), "r"(0));
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(out) : "r"(q1), "r"(q0), "r"(hi));
+    return out;
+}
+
+// Same codes as quant8 with fewer instructions: convert-to-nearest-even straight to an integer
+// and test the distance to that integer (more than 0.4999 = within 1e-4 of a tie -> real
+// division).  |x~ / scale| <= 127.00002, so no clamp is needed on the fast path.
+__device__ __forceinline__ uint2 quant8_fast(const float (&v)[8], float sc, float rcp) {
+    int q[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float t = v[i] * rcp;
+        q[i] = __float2int_rn(t);
+        if (fabsf(t - __int2float_rn(q[i])) > 0.4999f) q[i] = rne_clamp(__fdiv_rn(v[i], sc), -127.f, 127.f);
+    }
+    return make_uint2(pack4_s8(q[0], q[1], q[2], q[3]), pack4_s8(q[4], q[5], q[6], q[7]));
+}
+
 // ---------------------------------------------------------------------------
 // few tokens
 // ---------------------------------------------------------------------------
@@ -337,13 +359,14 @@ constexpr int kCRow = kCChunk * 2 + 16;     // padded row of a staged fp16 chunk
 __host__ __device__ constexpr int cluster_stages(int r) { return r <= 64 ? 3 : 2; }
 
 struct ClusterSmem {
-    int x_raw, s_vec, a_stage, la_stage, t_part, amax_part, scale, total;
+    int x_raw, s_vec, ones, a_stage, la_stage, t_part, amax_part, scale, total;
 };
 __host__ __device__ inline ClusterSmem cluster_smem(int Kc, int r) {
     ClusterSmem L;
     int off = 0;
     L.x_raw = off;      off += kCTok * (Kc * 2 + 16);          // raw fp16 activations (padded rows)
     L.s_vec = off;      off += Kc * 4;                         // smoothing divisors of the slice
+    L.ones = off;       off += ((Kc / 8 + 15) / 16) * 16;      // per 8 columns: all divisors are 1
     L.a_stage = off;    off += 2 * kCTok * kCRow;              // x~ as fp16, double buffered
     L.la_stage = off;                                          // L_A chunks; afterwards this CTA's
     L.t_part = off;                                            // partial T (fp32) reuses the space
@@ -398,8 +421,16 @@ quant_act_cluster_kernel(const __half* __restrict__ X, const float* __restrict__
     float* amax_part = reinterpret_cast<float*>(smem + L.amax_part);
     float* scale_sm = reinterpret_cast<float*>(smem + L.scale);
 
-    // smoothing divisors of the slice (plain loads; ones when s is absent)
+    // smoothing divisors of the slice (plain loads; ones when s is absent) and, per group of 8
+    // columns, whether all of them are 1: there x~ is the fp16 input itself
+    uint8_t* ones_sm = smem + L.ones;
     for (int i = tid; i < Kc; i += kCThreads) s_sm[i] = s ? s[k0 + i] : 1.f;
+    for (int g8 = tid; g8 < Kc / 8; g8 += kCThreads) {
+        bool one = true;
+        if (s)
+            for (int i = 0; i < 8; ++i) one = one && (s[k0 + g8 * 8 + i] == 1.f);
+        ones_sm[g8] = one ? 1 : 0;
+    }
 
     // Activations go to their final place, so they can be requested far ahead of use (the L_A
     // ring cannot): kXAhead chunks = 64 KiB in flight per SM, what an HBM-bound stream needs.
@@ -434,6 +465,7 @@ quant_act_cluster_kernel(const __half* __restrict__ X, const float* __restrict__
         cp_async_commit();
     }
     float amax = 0.f;
+    __half2 hamax = __float2half2_rn(0.f);
     for (int c = 0; c < nch; ++c) {
         cp_async_wait<STG - 2>();      // chunk c has landed (for this thread's copies)
         __syncthreads();                    // ... and for everyone's; chunk c-1 is fully consumed
@@ -442,21 +474,28 @@ quant_act_cluster_kernel(const __half* __restrict__ X, const float* __restrict__
         // x~ for this thread's 8 columns
         {
             const uint4 raw = *reinterpret_cast<const uint4*>(smem + L.x_raw + trow * xrow_bytes + c * (kCChunk * 2) + tcg * 16);
-            const float4 s0 = *reinterpret_cast<const float4*>(s_sm + c * kCChunk + tcg * 8);
-            const float4 s1 = *reinterpret_cast<const float4*>(s_sm + c * kCChunk + tcg * 8 + 4);
-            RawChunk rc{raw, s0, s1};
-            float v[8];
-            smooth8(rc, v);
+            uint4 pk;
+            if (ones_sm[c * (kCChunk / 8) + tcg]) {
+                // x~ == x: maximum of |x| in fp16 arithmetic is exact, the MMA operand is the input
+                const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(v[i]));
-            if (r > 0) {
+                for (int i = 0; i < 4; ++i) hamax = __hmax2(hamax, __habs2(h2[i]));
+                pk = raw;
+            } else {
+                const float4 s0 = *reinterpret_cast<const float4*>(s_sm + c * kCChunk + tcg * 8);
+                const float4 s1 = *reinterpret_cast<const float4*>(s_sm + c * kCChunk + tcg * 8 + 4);
+                RawChunk rc{raw, s0, s1};
+                float v[8];
+                smooth8(rc, v);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(v[i]));
                 __half2 p0 = __floats2half2_rn(v[0], v[1]), p1 = __floats2half2_rn(v[2], v[3]);
                 __half2 p2 = __floats2half2_rn(v[4], v[5]), p3 = __floats2half2_rn(v[6], v[7]);
-                uint4 pk;
                 pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
                 pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
-                *reinterpret_cast<uint4*>(smem + L.a_stage + (c & 1) * kCTok * kCRow + trow * kCRow + tcg * 16) = pk;
             }
+            if (r > 0)
+                *reinterpret_cast<uint4*>(smem + L.a_stage + (c & 1) * kCTok * kCRow + trow * kCRow + tcg * 16) = pk;
         }
         if (r > 0) {
             __syncthreads();
@@ -484,6 +523,7 @@ quant_act_cluster_kernel(const __half* __restrict__ X, const float* __restrict__
     __syncthreads();        // every warp is done with the L_A stages: their space now holds T
 
     // ---- publish this CTA's partial results for the cluster ----
+    amax = fmaxf(amax, fmaxf(__low2float(hamax), __high2float(hamax)));
     // row maximum over this thread's 8-column groups: the 16 threads of a row are adjacent lanes
 #pragma unroll
     for (int o = 8; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
@@ -525,14 +565,28 @@ quant_act_cluster_kernel(const __half* __restrict__ X, const float* __restrict__
     if (!row_ok) return;
     const float sc = scale_sm[trow];
     int8_t* out = Xq + (size_t)(m0 + trow) * K + k0;
+    if (!(sc > 0.f)) {   // all-zero token: codes 0
+        for (int c = 0; c < nch; ++c) *reinterpret_cast<uint2*>(out + c * kCChunk + tcg * 8) = make_uint2(0, 0);
+        return;
+    }
+    const float rcp = __frcp_rn(sc);
     for (int c = 0; c < nch; ++c) {
         const uint4 raw = *reinterpret_cast<const uint4*>(smem + L.x_raw + trow * xrow_bytes + c * (kCChunk * 2) + tcg * 16);
-        const float4 s0 = *reinterpret_cast<const float4*>(s_sm + c * kCChunk + tcg * 8);
-        const float4 s1 = *reinterpret_cast<const float4*>(s_sm + c * kCChunk + tcg * 8 + 4);
-        RawChunk rc{raw, s0, s1};
         float v[8];
-        smooth8(rc, v);
-        *reinterpret_cast<uint2*>(out + c * kCChunk + tcg * 8) = quant8(v, sc, sc > 0.f);
+        if (ones_sm[c * (kCChunk / 8) + tcg]) {
+            const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float2 f = __half22float2(h2[i]);
+                v[2 * i] = f.x; v[2 * i + 1] = f.y;
+            }
+        } else {
+            const float4 s0 = *reinterpret_cast<const float4*>(s_sm + c * kCChunk + tcg * 8);
+            const float4 s1 = *reinterpret_cast<const float4*>(s_sm + c * kCChunk + tcg * 8 + 4);
+            RawChunk rc{raw, s0, s1};
+            smooth8(rc, v);
+        }
+        *reinterpret_cast<uint2*>(out + c * kCChunk + tcg * 8) = quant8_fast(v, sc, rcp);
     }
 }
 

@@ -71,26 +71,27 @@ __device__ __forceinline__ uint2 quant8(const float (&v)[8], float sc, bool nonz
     return make_uint2(w[0], w[1]);
 }
 
-// d = bytes [lo0, lo1, hi0, hi1] as saturated int8 (two pack instructions per four codes).
-__device__ __forceinline__ uint32_t pack4_s8(int q0, int q1, int q2, int q3) {
-    uint32_t hi, out;
-    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(q3), "r"(q2), "r"(0));
-    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(out) : "r"(q1), "r"(q0), "r"(hi));
-    return out;
-}
-
-// Same codes as quant8 with fewer instructions: convert-to-nearest-even straight to an integer
-// and test the distance to that integer (more than 0.4999 = within 1e-4 of a tie -> real
-// division).  |x~ / scale| <= 127.00002, so no clamp is needed on the fast path.
+// Same codes as quant8 with fewer, cheaper instructions.  Conversions between float and int
+// run on a narrow pipe, so rounding uses the 1.5 * 2^23 constant instead: for |t| < 2^22,
+// t + 12582912.0f is rounded to the nearest-even integer and its low bits hold that integer in
+// two's complement.  The distance of t to that integer tells near-ties (within 1e-4 of a
+// half-integer), which alone take the real division.  |x~ / scale| <= 127.00002, so the fast
+// path needs no clamp.
 __device__ __forceinline__ uint2 quant8_fast(const float (&v)[8], float sc, float rcp) {
-    int q[8];
+    const float kMagic = 12582912.0f;   // 1.5 * 2^23
+    uint32_t q[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         const float t = v[i] * rcp;
-        q[i] = __float2int_rn(t);
-        if (fabsf(t - __int2float_rn(q[i])) > 0.4999f) q[i] = rne_clamp(__fdiv_rn(v[i], sc), -127.f, 127.f);
+        const float u = __fadd_rn(t, kMagic);
+        q[i] = __float_as_uint(u);      // low byte = code
+        if (fabsf(t - __fadd_rn(u, -kMagic)) > 0.4999f)
+            q[i] = (uint32_t)rne_clamp(__fdiv_rn(v[i], sc), -127.f, 127.f);
     }
-    return make_uint2(pack4_s8(q[0], q[1], q[2], q[3]), pack4_s8(q[4], q[5], q[6], q[7]));
+    // gather the low bytes of eight words
+    const uint32_t a01 = __byte_perm(q[0], q[1], 0x0040), a23 = __byte_perm(q[2], q[3], 0x0040);
+    const uint32_t a45 = __byte_perm(q[4], q[5], 0x0040), a67 = __byte_perm(q[6], q[7], 0x0040);
+    return make_uint2(__byte_perm(a01, a23, 0x5410), __byte_perm(a45, a67, 0x5410));
 }
 
 // ---------------------------------------------------------------------------

@@ -194,6 +194,25 @@ def run_reference(args, rank, world):
 
 
 # ---------------------------------------------------------------------------
+# multi-rank aggregation (replicas: no collective on the data path)
+# ---------------------------------------------------------------------------
+def max_over_ranks_ms(ms: float, world: int, device=None) -> float:
+    """Slowest rank's device time: the job is as fast as its slowest replica."""
+    if world == 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tops(ops_per_rank_step: float, ms_per_step: float, world: int) -> float:
+    """Aggregate throughput of `world` independent replicas that each finish a step in ms_per_step."""
+    return world * ops_per_rank_step / (ms_per_step * 1e-3) / 1e12
+
+
+# ---------------------------------------------------------------------------
 # GPU arm
 # ---------------------------------------------------------------------------
 class Bench:
@@ -291,11 +310,7 @@ def run_ours(args, rank, world, local_rank):
         torch.cuda.synchronize()
 
     def max_over_ranks(ms):
-        if world == 1:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return max_over_ranks_ms(ms, world, dev)
 
     W = max(args.warmup, 3)
     for i in range(W):
@@ -336,7 +351,7 @@ def run_ours(args, rank, world, local_rank):
         b.aser.check_status(L.ws)
 
     ms_step = ms_total / args.steps
-    tops = world * ops / (ms_step * 1e-3) / 1e12
+    tops = whole_job_tops(ops, ms_step, world)
     bytes_lin = algorithmic_bytes_linear(M, N, K, r)
     if b.bound == "hbm":
         achieved = bytes_lin / (ms_lin * 1e-3) / 1e9

@@ -12,11 +12,11 @@
 // units is cut into equal contiguous ranges, one per CTA; tiles shared by several CTAs are
 // summed through the workspace by whichever CTA arrives last.
 //
-// Warp roles (640 threads): 0 = weight producer, 1 and 19 = MMA issuers for even / odd stages
-// (1 also owns the TMEM allocation and issues the low-rank MMAs), 2..5 and 6..9 = two groups of
-// int4 -> int8 unpack warps that take alternate stages (group 0 also converts T),
-// 10..17 = epilogue (two warps per lane quarter, alternate 16-column chunks),
-// 18 = activation and low-rank operand producer.
+// Warp roles (512 threads for token tiles of 16/32, 640 above): 0 = weight producer, 1 and the
+// last warp = MMA issuers for even / odd stages (1 also owns the TMEM allocation and issues the
+// low-rank MMAs), 2..5 and 6..9 = two groups of int4 -> int8 unpack warps that take alternate
+// stages (group 0 also converts T), then 4 or 8 epilogue warps (two per tensor-memory lane
+// quarter take alternate 16-column chunks), then the activation / low-rank operand producer.
 // A single lane issues one tcgen05.mma per ~60-85 cycles, which bounds decode shapes (16 MMAs
 // per 32 KiB of weights); the integer accumulation is order-independent, so two lanes share the
 // issue work.  For that the accumulator is zeroed by the epilogue warps (tcgen05.st) when they

@@ -72,7 +72,7 @@ struct Cfg {
     static constexpr int OffT = OffLb + NL * LbBytes;
     static constexpr int OffBar = OffT + NL * TBytes;
     static constexpr int NumBars = 2 * NW + 2 * NX + 2 * NA + 3 * NL + 2 + 2 + 1;
-    static constexpr int SmemBytes = OffBar + NumBars * 8 + 64 + 1024;  // + slack for 1 KiB alignment
+    static constexpr int SmemBytes = OffBar + NumBars * 8 + 128 + 1024;  // + slack for 1 KiB alignment
     static constexpr int ASlotCols = KA * 32;
     static constexpr int TmemColsUsed = 3 * BT + NA * ASlotCols;
     static constexpr int TmemCols = TmemColsUsed <= 256 ? 256 : 512;
@@ -390,6 +390,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     int* last_flag = reinterpret_cast<int*>(tmem_slot + 2);
     volatile int* never_flag = reinterpret_cast<volatile int*>(tmem_slot + 3);  // stays 0
+    constexpr int kMaxContrib = 12;
+    int* contrib_slot = reinterpret_cast<int*>(tmem_slot + 4);                 // finalizer scratch
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = gridDim.x, cta = blockIdx.x;
@@ -759,10 +761,14 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                                 p.acc_debug[row0 + (uint32_t)j * (uint32_t)p.N] = ((int)vi[j]) >> 4;
                     }
                 } else {
+                    // partial tiles are stored [token / 4][row][4 tokens]: every thread moves 16
+                    // bytes and a warp 512 contiguous bytes per instruction
+                    uint4* pi = reinterpret_cast<uint4*>(pint + (c0 / 4) * 512 + nl * 4);
+                    uint4* pf = reinterpret_cast<uint4*>(plr + (c0 / 4) * 512 + nl * 4);
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        pint[(c0 + j) * 128 + nl] = (int)vi[j];
-                        if (w.has_lr) plr[(c0 + j) * 128 + nl] = __uint_as_float(vf[j]);
+                    for (int v4 = 0; v4 < 4; ++v4) {
+                        pi[v4 * 128] = make_uint4(vi[4 * v4], vi[4 * v4 + 1], vi[4 * v4 + 2], vi[4 * v4 + 3]);
+                        if (w.has_lr) pf[v4 * 128] = make_uint4(vf[4 * v4], vf[4 * v4 + 1], vf[4 * v4 + 2], vf[4 * v4 + 3]);
                     }
                 }
             }
@@ -793,46 +799,64 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 named_bar_sync(1, C::EpiThreads);           // everyone has read the flag before it is reused
                 if (last) {
                     if (et == 0) p.counters[w.tile] = 0;   // ready for the next launch
+                    // Slot of every contributor, computed once (by one thread each) instead of
+                    // per chunk: CTA c's items in order are a tile cut off at the start of its
+                    // range (slot 0), whole tiles, a tile cut off at the end of its range.
+                    const int ncontrib = c_last - c_first + 1;
+                    if (et < ncontrib && et < kMaxContrib) {
+                        const int c = c_first + et;
+                        const int bc = range_begin(p.units, c, G);
+                        contrib_slot[et] = c * 2 + ((bc >= first_unit) ? 0 : ((bc % p.KB != 0) ? 1 : 0));
+                    }
+                    named_bar_sync(1, C::EpiThreads);
 #pragma unroll 1
                     for (int c0 = 16 * half; c0 < BT; c0 += kChunkStep) {
-                        if (w.tt * BT + c0 >= p.M) break;
+                        if (tok0 + c0 >= p.M) break;
                         int sum[16];
 #pragma unroll
                         for (int j = 0; j < 16; ++j) sum[j] = 0;
-                        for (int cb = c_first; cb <= c_last; cb += 2) {
-                            // two contributors' loads in flight at a time
-                            int v[2][16];
+                        uint4 lr4[4];
+                        if (p.r > 0) {
+                            const uint4* lsrc = reinterpret_cast<const uint4*>(
+                                p.part_lr + (size_t)c_first * (BT * 128) + (c0 / 4) * 512 + nl * 4);
+#pragma unroll
+                            for (int v4 = 0; v4 < 4; ++v4) lr4[v4] = __ldcg(lsrc + v4 * 128);
+                        }
+                        for (int cb = 0; cb < ncontrib; cb += 2) {
+                            // two contributors' loads (eight 16-byte loads) in flight at a time
+                            uint4 v[2][4];
 #pragma unroll
                             for (int u = 0; u < 2; ++u) {
-                                const int c = cb + u;
-                                if (c <= c_last) {
-                                    // CTA c's items in order: a tile cut off at the start of its
-                                    // range (slot 0), whole tiles, a tile cut off at its end.
-                                    const int bc = range_begin(p.units, c, G);
-                                    const int slot = (bc >= first_unit) ? 0 : ((bc % p.KB != 0) ? 1 : 0);
-                                    const int32_t* src = p.part_int + ((size_t)c * 2 + slot) * (BT * 128) + c0 * 128 + nl;
+                                if (cb + u < ncontrib) {
+                                    // contributors past the table lie strictly inside the tile: slot 0
+                                    const int slot = (cb + u < kMaxContrib) ? contrib_slot[cb + u]
+                                                                            : (c_first + cb + u) * 2;
+                                    const uint4* src = reinterpret_cast<const uint4*>(
+                                        p.part_int + (size_t)slot * (BT * 128) + (c0 / 4) * 512 + nl * 4);
 #pragma unroll
-                                    for (int j = 0; j < 16; ++j) v[u][j] = __ldcg(src + j * 128);
+                                    for (int v4 = 0; v4 < 4; ++v4) v[u][v4] = __ldcg(src + v4 * 128);
                                 } else {
 #pragma unroll
-                                    for (int j = 0; j < 16; ++j) v[u][j] = 0;
+                                    for (int v4 = 0; v4 < 4; ++v4) v[u][v4] = make_uint4(0, 0, 0, 0);
                                 }
                             }
 #pragma unroll
                             for (int u = 0; u < 2; ++u)
 #pragma unroll
-                                for (int j = 0; j < 16; ++j) sum[j] += v[u][j];
+                                for (int v4 = 0; v4 < 4; ++v4) {
+                                    sum[4 * v4] += (int)v[u][v4].x; sum[4 * v4 + 1] += (int)v[u][v4].y;
+                                    sum[4 * v4 + 2] += (int)v[u][v4].z; sum[4 * v4 + 3] += (int)v[u][v4].w;
+                                }
                         }
-                        const float* lsrc = p.part_lr + (size_t)c_first * (BT * 128) + c0 * 128 + nl;
+                        const uint32_t row0 = (uint32_t)(tok0 + c0) * (uint32_t)p.N + (uint32_t)n;
+                        const uint32_t* lrw = reinterpret_cast<const uint32_t*>(lr4);
 #pragma unroll
                         for (int j = 0; j < 16; ++j) {
-                            const int tok = w.tt * BT + c0 + j;
-                            if (tok < p.M && n_ok) {
-                                const int acc = sum[j] >> 4;
-                                float y = (float)acc * __ldg(p.a_scale + tok) * ws;
-                                if (p.r > 0) y += __ldcg(lsrc + j * 128);
-                                p.Y[(size_t)tok * p.N + n] = __float2half_rn(y);
-                                if (p.acc_debug) p.acc_debug[(size_t)tok * p.N + n] = acc;
+                            if (c0 + j < valid && n_ok) {
+                                const float lr = (p.r > 0) ? __uint_as_float(lrw[j]) : 0.f;
+                                const float y = fmaf((float)sum[j], __ldg(p.a_scale + tok0 + c0 + j) * ws16, lr);
+                                p.Y[row0 + (uint32_t)j * (uint32_t)p.N] = __float2half_rn(y);
+                                if (p.acc_debug) p.acc_debug[row0 + (uint32_t)j * (uint32_t)p.N] = sum[j] >> 4;
                             }
                         }
                     }

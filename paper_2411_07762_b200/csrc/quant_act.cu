@@ -2,13 +2,16 @@
 // per-token int8 round-to-nearest (Sec. 5.1) and the down projection T = X~ L_A^T of the
 // error-reconstruction branch (Sec. 4.1).
 //
-// Two launch shapes:
+// Launch shapes:
 //   * few tokens (decode): one CTA per (token, group of L_A rows) so that the L_A stream is
 //     spread over many SMs; CUDA-core FMAs in fp32.
-//   * many tokens (prefill): one CTA per 16 tokens; x~ is rounded to fp16 and multiplied with
-//     L_A on the tensor cores (mma.sync m16n8k16, fp32 accumulation) while the row absmax is
-//     collected; a second sweep over the (L2-resident) rows writes the int8 codes.
+//   * many tokens (prefill): clusters of CTAs own 128 tokens each and split K; TMA streams the
+//     activations through shared memory twice (row maxima + tcgen05 down projection, then the
+//     int8 codes, written back by TMA stores).  See the section below.
+//   * a plain mma.sync kernel (16 tokens per CTA) remains for shapes the cluster kernel
+//     cannot take.
 #include "aser_common.cuh"
+#include "sm100_ptx.cuh"
 
 namespace aser {
 
@@ -69,29 +72,6 @@ __device__ __forceinline__ uint2 quant8(const float (&v)[8], float sc, bool nonz
         w[i >> 2] |= (uint32_t)(q & 0xFF) << (8 * (i & 3));
     }
     return make_uint2(w[0], w[1]);
-}
-
-// Same codes as quant8 with fewer, cheaper instructions.  Conversions between float and int
-// run on a narrow pipe, so rounding uses the 1.5 * 2^23 constant instead: for |t| < 2^22,
-// t + 12582912.0f is rounded to the nearest-even integer and its low bits hold that integer in
-// two's complement.  The distance of t to that integer tells near-ties (within 1e-4 of a
-// half-integer), which alone take the real division.  |x~ / scale| <= 127.00002, so the fast
-// path needs no clamp.
-__device__ __forceinline__ uint2 quant8_fast(const float (&v)[8], float sc, float rcp) {
-    const float kMagic = 12582912.0f;   // 1.5 * 2^23
-    uint32_t q[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const float t = v[i] * rcp;
-        const float u = __fadd_rn(t, kMagic);
-        q[i] = __float_as_uint(u);      // low byte = code
-        if (fabsf(t - __fadd_rn(u, -kMagic)) > 0.4999f)
-            q[i] = (uint32_t)rne_clamp(__fdiv_rn(v[i], sc), -127.f, 127.f);
-    }
-    // gather the low bytes of eight words
-    const uint32_t a01 = __byte_perm(q[0], q[1], 0x0040), a23 = __byte_perm(q[2], q[3], 0x0040);
-    const uint32_t a45 = __byte_perm(q[4], q[5], 0x0040), a67 = __byte_perm(q[6], q[7], 0x0040);
-    return make_uint2(__byte_perm(a01, a23, 0x5410), __byte_perm(a45, a67, 0x5410));
 }
 
 // ---------------------------------------------------------------------------
@@ -344,279 +324,640 @@ quant_act_large_kernel(const __half* __restrict__ X, const float* __restrict__ s
 }
 
 // ---------------------------------------------------------------------------
-// many tokens, single pass over X: thread-block cluster split along K
+// many tokens: TMA ring + tcgen05 down projection, thread-block cluster split along K
 // ---------------------------------------------------------------------------
-// A cluster of CK CTAs owns 32 tokens; CTA `rank` owns the K-slice [rank*Kc, (rank+1)*Kc) with
-// Kc <= 2048, small enough to keep the raw fp16 activations of the slice in shared memory.
-// Sweep 1 (per 64-column chunk): x~ = x / s, row absmax, x~ rounded to fp16 and multiplied with
-// the L_A chunk on the tensor cores.  Then the CTAs exchange row maxima and partial T through
-// distributed shared memory, and sweep 2 quantizes the resident slice, so X is read from HBM
-// exactly once and L_A is re-read once per 32 tokens.
-constexpr int kCTok = 32;                   // tokens per cluster
-constexpr int kCThreads = 512;              // 16 threads per token row; 16 warps hide latencies
-constexpr int kCChunk = 128;                // columns per pipeline step
-constexpr int kCRow = kCChunk * 2 + 16;     // padded row of a staged fp16 chunk (272 B)
-// L_A chunks in flight: as many as shared memory allows beside the resident activations
-__host__ __device__ constexpr int cluster_stages(int r) { return r <= 64 ? 3 : 2; }
+// A cluster of CK CTAs owns 128 tokens (the MMA's M side); CTA `rank` owns the K-slice
+// [rank*Kc, (rank+1)*Kc) and streams it twice through a ring of 64-column stages filled by TMA
+// (128-byte swizzle, rows past M read as zero).
+//   Sweep 1: the consumer warps scan each stage for the row maximum of |x~|.  Where all 16
+//   divisors of a (row, 16-column) unit are 1 (all but the outlier channels), x~ is the fp16
+//   input itself and the stage is left as TMA wrote it; elsewhere x~ = x / s is computed in
+//   fp32 and written back as fp16 in place.  One thread then issues tcgen05.mma (kind::f16,
+//   M = 128 tokens, N = r) with the stage as the A operand and the L_A tile (TMA) as B; the
+//   partial T accumulates in tensor memory.
+//   Exchange: row maxima and partial T go through distributed shared memory; every CTA of the
+//   cluster gets the row scales, and the cluster's CTAs share the summation of T.
+//   Sweep 2: the slice is streamed again (it was just read, so it comes from L2), quantized,
+//   staged in shared memory (64-byte swizzle) and written by TMA stores, which also clip rows
+//   past M.
+// A warp handles one 16-column group for 32 rows (lane = row), so whether a unit needs the
+// division is uniform across the warp and the swizzled 16-byte accesses are conflict-free.
+constexpr int kTTok = 128;                  // tokens per cluster
+constexpr int kTCols = 64;                  // columns per stage: one 128-byte swizzle row of fp16
+constexpr int kTConsumerWarps = 16;         // warp = (32-row block, 16-column group)
+constexpr int kTConsumers = kTConsumerWarps * 32;
+constexpr int kTWarpProd = kTConsumerWarps;         // TMA producer warp
+constexpr int kTWarpMma = kTConsumerWarps + 1;      // MMA issuer warp, owns the tensor memory
+constexpr int kTThreads = kTConsumers + 64;
+constexpr int kTStages = 4;                 // activation / L_A ring depth
+constexpr int kTOut = 4;                    // int8 output tiles in flight
+constexpr int kXTileBytes = kTTok * 128;    // 128 rows x 64 fp16
+constexpr int kOutTileBytes = kTTok * 64;   // 128 rows x 64 int8
+constexpr long long kQaWaitLimitClocks = 4000000000ll;   // about 2 s of SM clocks per wait
 
-struct ClusterSmem {
-    int x_raw, s_vec, ones, a_stage, la_stage, t_part, amax_part, scale, total;
+struct TmaSmem {
+    int x_ring, region_b, la_bytes, ones, amax_cg, amax_slots, bars, tmem_slot, abort_flag, total;
 };
-__host__ __device__ inline ClusterSmem cluster_smem(int Kc, int r) {
-    ClusterSmem L;
+// Offsets from the 1 KiB-aligned base.  Region B holds, one after the other in time: the L_A
+// ring (sweep 1), the output tiles (sweep 2), and the partial T pushed by the cluster's CTAs for
+// the rows this CTA owns, as [source CTA][row][r] floats (128 * r floats in all).
+__host__ __device__ inline TmaSmem tma_smem(int Kc, int r) {
+    TmaSmem L;
     int off = 0;
-    L.x_raw = off;      off += kCTok * (Kc * 2 + 16);          // raw fp16 activations (padded rows)
-    L.s_vec = off;      off += Kc * 4;                         // smoothing divisors of the slice
-    L.ones = off;       off += ((Kc / 8 + 15) / 16) * 16;      // per 8 columns: all divisors are 1
-    L.a_stage = off;    off += 2 * kCTok * kCRow;              // x~ as fp16, double buffered
-    L.la_stage = off;                                          // L_A chunks; afterwards this CTA's
-    L.t_part = off;                                            // partial T (fp32) reuses the space
+    L.x_ring = off;     off += kTStages * kXTileBytes;
+    L.region_b = off;
+    L.la_bytes = r * 128;
     {
-        const int la = cluster_stages(r) * r * kCRow, tp = kCTok * r * 4;
-        off += (la > tp ? la : tp) + 16;
+        int b = kTStages * L.la_bytes;                         // = 128 * r * 4, the pushed partials
+        if (kTOut * kOutTileBytes > b) b = kTOut * kOutTileBytes;
+        off += (b + 1023) / 1024 * 1024;
     }
-    L.amax_part = off;  off += kCTok * 4;
-    L.scale = off;      off += kCTok * 4;
-    L.total = off;
+    L.ones = off;       off += (Kc / 16 + 15) / 16 * 16;       // per 16 columns: all divisors are 1
+    L.amax_cg = off;    off += 4 * kTTok * 4;                  // row maxima per 16-column group
+    L.amax_slots = off; off += 16 * kTTok * 4;                 // row maxima pushed by each CTA
+    L.bars = off;       off += (4 * kTStages + 2 * kTOut + 2) * 8;
+    L.tmem_slot = off;  off += 8;
+    L.abort_flag = off; off += 8;
+    L.total = off + 1024;                                      // slack for the alignment
     return L;
 }
+static_assert(kTStages == 4, "region B: the L_A ring and the pushed partial T have the same size");
 
 __device__ __forceinline__ uint32_t cluster_rank() {
     uint32_t r;
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
     return r;
 }
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+__device__ __forceinline__ void cluster_arrive() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
 }
-// Read a float from the same shared-memory offset in CTA `rank` of the cluster.
-__device__ __forceinline__ float dsmem_ld_f32(uint32_t local_addr, uint32_t rank) {
+__device__ __forceinline__ void cluster_wait() {
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Address of the same shared-memory offset in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t dsmem_addr(uint32_t local_addr, uint32_t rank) {
     uint32_t remote;
-    float v;
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
-    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
+    return remote;
+}
+// Stores into a peer's shared memory; the cluster barrier publishes them.
+__device__ __forceinline__ void dsmem_st_f32(uint32_t remote, float v) {
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
+}
+__device__ __forceinline__ void dsmem_st_v4(uint32_t remote, const uint32_t (&v)[4]) {
+    asm volatile("st.shared::cluster.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(remote), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]) : "memory");
+}
+
+// Bounded wait on an mbarrier phase.  On expiry (or when another thread of the CTA has given
+// up) it sets the CTA's abort flag and returns false; the caller leaves its loop.
+__device__ __noinline__ bool qa_wait_slow(uint32_t bar, uint32_t parity, volatile int* flag) {
+    uint32_t spins = 0;
+    long long t0 = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 255u) == 0) {
+            if (*flag) return false;
+            if (t0 == 0) {
+                t0 = clock64();
+            } else if (clock64() - t0 > kQaWaitLimitClocks) {
+                *flag = 1;
+                return false;
+            }
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ bool qa_wait(uint32_t bar, uint32_t parity, volatile int* flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return qa_wait_slow(bar, parity, flag);
+}
+// Warp-collective form: lane 0 polls, the outcome is broadcast.
+__device__ __forceinline__ bool qa_warp_wait(uint32_t bar, uint32_t parity, volatile int* flag, int lane) {
+    int ok = 1;
+    if (lane == 0) ok = qa_wait(bar, parity, flag) ? 1 : 0;
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, uint32_t src) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(map), "r"(x), "r"(y), "r"(src)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void tmem_ld4(uint32_t taddr, uint32_t (&v)[4]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3])
+                 : "r"(taddr)
+                 : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3])::"memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
     return v;
 }
+__device__ __forceinline__ void sts128(uint32_t addr, uint4 v) {
+    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
 
-// grid = (CK, ceil(M / 32)), cluster = (CK, 1, 1).  NTW = 8-column tiles of T per warp,
-// STG = L_A pipeline depth (cluster_stages(r)).
-template <int NTW, int STG>
-__global__ void __launch_bounds__(kCThreads)
-quant_act_cluster_kernel(const __half* __restrict__ X, const float* __restrict__ s,
-                         const __half* __restrict__ LA, int M, int K, int Kc, int r, int CK,
-                         int8_t* __restrict__ Xq, float* __restrict__ a_scale,
-                         __nv_bfloat16* __restrict__ T) {
-    extern __shared__ __align__(16) uint8_t smem[];
-    const ClusterSmem L = cluster_smem(Kc, r);
-    const int xrow_bytes = Kc * 2 + 16;            // padded: rows of a warp fall in different banks
-    const uint32_t sb = (uint32_t)__cvta_generic_to_shared(smem);
+// 8 fp16 -> 8 fp32
+__device__ __forceinline__ void cvt8(const uint4& raw, float (&v)[8]) {
+    const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float2 f = __half22float2(h2[i]);
+        v[2 * i] = f.x; v[2 * i + 1] = f.y;
+    }
+}
+// x~ = fp32(x) / s for 8 columns (IEEE divisions)
+__device__ __forceinline__ void div8(const uint4& raw, const float4& s0, const float4& s1, float (&v)[8]) {
+    cvt8(raw, v);
+    v[0] = __fdiv_rn(v[0], s0.x); v[1] = __fdiv_rn(v[1], s0.y);
+    v[2] = __fdiv_rn(v[2], s0.z); v[3] = __fdiv_rn(v[3], s0.w);
+    v[4] = __fdiv_rn(v[4], s1.x); v[5] = __fdiv_rn(v[5], s1.y);
+    v[6] = __fdiv_rn(v[6], s1.z); v[7] = __fdiv_rn(v[7], s1.w);
+}
+__device__ __forceinline__ uint4 pack8_half(const float (&v)[8]) {
+    uint4 pk;
+    __half2 p0 = __floats2half2_rn(v[0], v[1]), p1 = __floats2half2_rn(v[2], v[3]);
+    __half2 p2 = __floats2half2_rn(v[4], v[5]), p3 = __floats2half2_rn(v[6], v[7]);
+    pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
+    pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
+    return pk;
+}
+
+// Exact codes for eight values (the definition: IEEE quotient, round half to even, clamp).
+__device__ __noinline__ uint2 quant8_exact(float v0, float v1, float v2, float v3, float v4, float v5,
+                                           float v6, float v7, float sc) {
+    const float v[8] = {v0, v1, v2, v3, v4, v5, v6, v7};
+    uint32_t w[2] = {0, 0};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int q = rne_clamp(__fdiv_rn(v[i], sc), -127.f, 127.f);
+        w[i >> 2] |= (uint32_t)(q & 0xFF) << (8 * (i & 3));
+    }
+    return make_uint2(w[0], w[1]);
+}
+// Same codes as quant8 for sc > 0, on packed fp32 pairs: t = x~ * (1 / sc), rounded by adding
+// 1.5 * 2^23 (the low byte of the sum is the code); the distance of t to that integer tells the
+// near-ties, and a group with one takes the exact path as a whole.
+__device__ __forceinline__ uint2 quant8_pairs(const float (&v)[8], float sc, float rcp) {
+    const float kMagic = 12582912.0f;
+    const float2 r2 = make_float2(rcp, rcp), m2 = make_float2(kMagic, kMagic);
+    const float2 nm2 = make_float2(-kMagic, -kMagic), neg1 = make_float2(-1.f, -1.f);
+    uint32_t q[8];
+    bool tie = false;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float2 t = __fmul2_rn(make_float2(v[2 * i], v[2 * i + 1]), r2);
+        const float2 u = __fadd2_rn(t, m2);
+        const float2 w = __fadd2_rn(u, nm2);            // the rounded integer
+        const float2 d = __ffma2_rn(w, neg1, t);        // t - w, exact
+        q[2 * i] = __float_as_uint(u.x);
+        q[2 * i + 1] = __float_as_uint(u.y);
+        tie = tie || fabsf(d.x) > 0.4999f || fabsf(d.y) > 0.4999f;
+    }
+    if (tie) return quant8_exact(v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7], sc);
+    const uint32_t a01 = __byte_perm(q[0], q[1], 0x0040), a23 = __byte_perm(q[2], q[3], 0x0040);
+    const uint32_t a45 = __byte_perm(q[4], q[5], 0x0040), a67 = __byte_perm(q[6], q[7], 0x0040);
+    return make_uint2(__byte_perm(a01, a23, 0x5410), __byte_perm(a45, a67, 0x5410));
+}
+
+// grid = (CK, ceil(M / 128)), cluster = (CK, 1, 1) with CK a power of two <= 16, kTThreads threads.
+// map_x: X as fp16 [M, K], box 128 rows x 64 columns, 128-byte swizzle.
+// map_la: L_A as fp16 [r, K], box r rows x 64 columns, 128-byte swizzle (unused when r == 0).
+// map_q: Xq as bytes [M, K], box 128 rows x 64 columns, 64-byte swizzle.
+__global__ void __launch_bounds__(kTThreads, 2)
+quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_la,
+                     const __grid_constant__ CUtensorMap map_q, const float* __restrict__ s,
+                     int M, int K, int Kc, int r, int CK, float* __restrict__ a_scale,
+                     __nv_bfloat16* __restrict__ T) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t sraw = smem_u32(smem_raw);
+    const uint32_t sb = (sraw + 1023u) & ~1023u;            // swizzled tiles need 1 KiB alignment
+    uint8_t* smem = smem_raw + (sb - sraw);
+    const TmaSmem L = tma_smem(Kc, r);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t rank = cluster_rank();
-    const int m0 = blockIdx.y * kCTok;
+    const int m0 = blockIdx.y * kTTok;
     const int k0 = (int)rank * Kc;
-    const int nch = Kc / kCChunk;
-    const int trow = tid >> 4, tcg = tid & 15;     // this thread's token row and 8-column group
-    const bool row_ok = m0 + trow < M;
-    float* s_sm = reinterpret_cast<float*>(smem + L.s_vec);
-    float* t_part = reinterpret_cast<float*>(smem + L.t_part);
-    float* amax_part = reinterpret_cast<float*>(smem + L.amax_part);
-    float* scale_sm = reinterpret_cast<float*>(smem + L.scale);
-
-    // smoothing divisors of the slice (plain loads; ones when s is absent) and, per group of 8
-    // columns, whether all of them are 1: there x~ is the fp16 input itself
+    const int nst = Kc / kTCols;                            // stages per sweep
+    const int rows_owned = kTTok / CK;                      // rows of T this CTA sums and writes
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L.abort_flag);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L.tmem_slot);
     uint8_t* ones_sm = smem + L.ones;
-    for (int i = tid; i < Kc; i += kCThreads) s_sm[i] = s ? s[k0 + i] : 1.f;
-    for (int g8 = tid; g8 < Kc / 8; g8 += kCThreads) {
-        bool one = true;
-        if (s)
-            for (int i = 0; i < 8; ++i) one = one && (s[k0 + g8 * 8 + i] == 1.f);
-        ones_sm[g8] = one ? 1 : 0;
-    }
+    float* amax_cg = reinterpret_cast<float*>(smem + L.amax_cg);
+    float* amax_slots = reinterpret_cast<float*>(smem + L.amax_slots);
+    float* t_slots = reinterpret_cast<float*>(smem + L.region_b);
+    auto bar_full = [&](int st) { return sb + L.bars + st * 8; };
+    auto bar_ready = [&](int st) { return sb + L.bars + (kTStages + st) * 8; };
+    auto bar_free1 = [&](int st) { return sb + L.bars + (2 * kTStages + st) * 8; };
+    auto bar_free2 = [&](int st) { return sb + L.bars + (3 * kTStages + st) * 8; };
+    auto bar_out_full = [&](int o) { return sb + L.bars + (4 * kTStages + o) * 8; };
+    auto bar_out_free = [&](int o) { return sb + L.bars + (4 * kTStages + kTOut + o) * 8; };
+    const uint32_t bar_acc = sb + L.bars + (4 * kTStages + 2 * kTOut) * 8;
+    const uint32_t bar_tail = bar_acc + 8;      // the output tiles are no longer in use
+    uint32_t tmem_cols = 32;
+    while ((int)tmem_cols < r) tmem_cols <<= 1;
 
-    // Activations go to their final place, so they can be requested far ahead of use (the L_A
-    // ring cannot): kXAhead chunks = 64 KiB in flight per SM, what an HBM-bound stream needs.
-    constexpr int kXAhead = 8;
-    auto issue_x = [&](int c) {
-        // 32 rows x 256 B, one 16-byte copy per thread (zero rows past M)
-        const uint32_t xdst = sb + L.x_raw + trow * xrow_bytes + c * (kCChunk * 2) + tcg * 16;
-        if (row_ok) cp_async16(xdst, X + (size_t)(m0 + trow) * K + k0 + c * kCChunk + tcg * 8);
-        else *reinterpret_cast<uint4*>(smem + L.x_raw + trow * xrow_bytes + c * (kCChunk * 2) + tcg * 16) = make_uint4(0, 0, 0, 0);
-    };
-    auto issue_chunk = [&](int c) {
-        if (c + kXAhead < nch) issue_x(c + kXAhead);
-        // L_A chunk: r rows x 256 B
-        const uint32_t ldst = sb + L.la_stage + (c % STG) * r * kCRow;
-        for (int i = tid; i < r * 16; i += kCThreads) {
-            const int j = i >> 4, cc = i & 15;
-            cp_async16(ldst + j * kCRow + cc * 16, LA + (size_t)j * K + k0 + c * kCChunk + cc * 8);
-        }
-    };
-
-    float acc[NTW][4];
-#pragma unroll
-    for (int i = 0; i < NTW; ++i)
-#pragma unroll
-        for (int e = 0; e < 4; ++e) acc[i][e] = 0.f;
-    const int mt = warp & 1, nq = warp >> 1;
-    const int ntiles = r / 8;
-
-    for (int c = 0; c < kXAhead && c < nch; ++c) issue_x(c);   // joins the first commit group
-    for (int c = 0; c < STG - 1; ++c) {
-        if (c < nch) issue_chunk(c);
-        cp_async_commit();
-    }
-    float amax = 0.f;
-    __half2 hamax = __float2half2_rn(0.f);
-    for (int c = 0; c < nch; ++c) {
-        cp_async_wait<STG - 2>();      // chunk c has landed (for this thread's copies)
-        __syncthreads();                    // ... and for everyone's; chunk c-1 is fully consumed
-        if (c + STG - 1 < nch) issue_chunk(c + STG - 1);   // refills the stage of chunk c-1
-        cp_async_commit();
-        // x~ for this thread's 8 columns
-        {
-            const uint4 raw = *reinterpret_cast<const uint4*>(smem + L.x_raw + trow * xrow_bytes + c * (kCChunk * 2) + tcg * 16);
-            uint4 pk;
-            if (ones_sm[c * (kCChunk / 8) + tcg]) {
-                // x~ == x: maximum of |x| in fp16 arithmetic is exact, the MMA operand is the input
-                const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
-#pragma unroll
-                for (int i = 0; i < 4; ++i) hamax = __hmax2(hamax, __habs2(h2[i]));
-                pk = raw;
+    // Use i of the ring: i < nst is sweep 1 (X and L_A tiles), the rest sweep 2 (X only).
+    // A stage's previous use was released by the MMAs (sweep 1) or the consumers (sweep 2).
+    auto load_use = [&](int i) -> bool {
+        const int st = i % kTStages;
+        if (i >= kTStages) {
+            const int prev = i - kTStages;
+            bool ok;
+            if (prev < nst) {
+                ok = qa_wait(bar_free1(st), (uint32_t)(prev / kTStages) & 1u, abort_flag);
             } else {
-                const float4 s0 = *reinterpret_cast<const float4*>(s_sm + c * kCChunk + tcg * 8);
-                const float4 s1 = *reinterpret_cast<const float4*>(s_sm + c * kCChunk + tcg * 8 + 4);
-                RawChunk rc{raw, s0, s1};
-                float v[8];
-                smooth8(rc, v);
-#pragma unroll
-                for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(v[i]));
-                __half2 p0 = __floats2half2_rn(v[0], v[1]), p1 = __floats2half2_rn(v[2], v[3]);
-                __half2 p2 = __floats2half2_rn(v[4], v[5]), p3 = __floats2half2_rn(v[6], v[7]);
-                pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
-                pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
+                const int first = nst + ((st - nst % kTStages + kTStages) % kTStages);
+                ok = qa_wait(bar_free2(st), (uint32_t)((prev - first) / kTStages) & 1u, abort_flag);
             }
-            if (r > 0)
-                *reinterpret_cast<uint4*>(smem + L.a_stage + (c & 1) * kCTok * kCRow + trow * kCRow + tcg * 16) = pk;
+            if (!ok) return false;
         }
+        const uint32_t xdst = sb + L.x_ring + st * kXTileBytes;
+        if (i < nst) {
+            mbar_arrive_expect_tx(bar_full(st), (uint32_t)(kXTileBytes + L.la_bytes));
+            tma_load_2d(xdst, &map_x, k0 + i * kTCols, m0, bar_full(st));
+            if (r > 0) tma_load_2d(sb + L.region_b + st * L.la_bytes, &map_la, k0 + i * kTCols, 0, bar_full(st));
+        } else {
+            mbar_arrive_expect_tx(bar_full(st), (uint32_t)kXTileBytes);
+            tma_load_2d(xdst, &map_x, k0 + (i - nst) * kTCols, m0, bar_full(st));
+        }
+        return true;
+    };
+
+    // ---- setup ----
+    if (warp == kTWarpProd) {
+        // The producer sets up the barriers and fills the ring before anyone else is ready.
+        if (lane == 0) {
+            for (int st = 0; st < kTStages; ++st) {
+                mbar_init(bar_full(st), 1);                     // the producer's expect_tx arrival
+                mbar_init(bar_ready(st), kTConsumerWarps);      // consumers are done with the stage
+                mbar_init(bar_free1(st), 1);                    // sweep 1: the MMAs have read it
+                mbar_init(bar_free2(st), kTConsumerWarps);      // sweep 2: the consumers have read it
+            }
+            for (int o = 0; o < kTOut; ++o) {
+                mbar_init(bar_out_full(o), kTConsumerWarps);    // an output tile is written
+                mbar_init(bar_out_free(o), 1);                  // its store has read it
+            }
+            mbar_init(bar_acc, 1);
+            mbar_init(bar_tail, 1);
+            *abort_flag = 0;
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            fence_proxy_async_smem();
+            for (int i = 0; i < kTStages && i < 2 * nst; ++i) load_use(i);      // no waits yet
+        }
+        __syncwarp();
+    } else if (warp == kTWarpMma) {
         if (r > 0) {
-            __syncthreads();
-            const uint32_t a_base = sb + L.a_stage + (c & 1) * kCTok * kCRow + (mt * 16 + (lane & 15)) * kCRow + (lane >> 4) * 16;
-            const uint32_t b_base = sb + L.la_stage + (c % STG) * r * kCRow + (lane & 7) * kCRow + (lane >> 3) * 16;
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(tmem_slot)), "r"(tmem_cols)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
+        if (lane == 0) prefetch_tensormap(&map_q);
+    } else {
+        // per 16 columns of the slice: are all smoothing divisors 1?
+        for (int g = tid; g < Kc / 16; g += kTConsumers) {
+            bool one = true;
+            if (s) {
+                const float4* sp = reinterpret_cast<const float4*>(s + k0 + g * 16);
 #pragma unroll
-            for (int kk = 0; kk < kCChunk / 32; ++kk) {
-                uint32_t a0, a1, a2, a3, a4, a5, a6, a7;
-                ldmatrix_x4(a_base + kk * 64, a0, a1, a2, a3);
-                ldmatrix_x4(a_base + kk * 64 + 32, a4, a5, a6, a7);
+                for (int i = 0; i < 4; ++i) {
+                    const float4 v = __ldg(sp + i);
+                    one = one && v.x == 1.f && v.y == 1.f && v.z == 1.f && v.w == 1.f;
+                }
+            }
+            ones_sm[g] = one ? 1 : 0;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = (r > 0) ? *tmem_slot : 0u;
+
+    // this thread's unit inside a stage (consumer warps): row and 16-column group
+    const int rb = warp >> 2, cg = warp & 3;
+    const int row = rb * 32 + lane;
+    // 16-byte pieces 2cg and 2cg+1 of the row, at their swizzled places (they differ in bit 4)
+    const uint32_t x_off = (uint32_t)row * 128u + (uint32_t)(((2 * cg) ^ (row & 7)) << 4);
+
+    if (warp == kTWarpProd) {
+        // ================= TMA producer =================
+        // Uses whose stage is released by sweep 1 come before the exchange; the rest wait for
+        // the consumers' sweep 2, which starts after the cluster barrier this warp takes part in.
+        const int early = (2 * nst < nst + kTStages) ? 2 * nst : nst + kTStages;
+        bool ok = true;
+        if (lane == 0) {
+            for (int i = kTStages; i < early && ok; ++i) ok = load_use(i);
+        }
+        __syncwarp();
+        cluster_arrive();
+        cluster_wait();
+        if (lane == 0) {
+            for (int i = (early > kTStages ? early : kTStages); i < 2 * nst && ok; ++i) ok = load_use(i);
+        }
+        __syncwarp();
+        if (r > 0 && CK > 1) {      // the exchange of T at the end
+            cluster_arrive();
+            cluster_wait();
+            cluster_arrive();
+            cluster_wait();
+        }
+    } else if (warp == kTWarpMma) {
+        // ================= MMA issuer, then store issuer =================
+        bool ok = true;
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc(1u, 0u, (uint32_t)kTTok, (uint32_t)r);
+            for (int i = 0; i < nst; ++i) {
+                const int st = i % kTStages;
+                ok = qa_wait(bar_ready(st), (uint32_t)(i / kTStages) & 1u, abort_flag);
+                if (!ok) break;
+                if (r > 0) {
+                    tc_fence_after();
+                    const uint64_t adesc = smem_desc_sw128(sb + L.x_ring + st * kXTileBytes);
+                    const uint64_t bdesc = smem_desc_sw128(sb + L.region_b + st * L.la_bytes);
 #pragma unroll
-                for (int i = 0; i < NTW; ++i) {
-                    const int nt = nq + 8 * i;
-                    if (nt < ntiles) {
-                        uint32_t b0, b1, b2, b3;
-                        ldmatrix_x4(b_base + nt * 8 * kCRow + kk * 64, b0, b1, b2, b3);
-                        mma_f16(acc[i], a0, a1, a2, a3, b0, b1);
-                        mma_f16(acc[i], a4, a5, a6, a7, b2, b3);
+                    for (int kk = 0; kk < kTCols / 16; ++kk)
+                        mma_f16_ss(tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, (i != 0 || kk != 0) ? 1u : 0u);
+                    tc_commit(bar_free1(st));
+                } else {
+                    mbar_arrive(bar_free1(st));
+                }
+            }
+            if (r > 0) tc_commit(bar_acc);      // arrives when every MMA above has completed
+        }
+        __syncwarp();
+        cluster_arrive();
+        cluster_wait();
+        if (lane == 0) {
+            // Sweep 2: one TMA store per output tile.  A tile goes back to the consumers once
+            // the store has read it; the stores run two behind.
+            for (int j = 0; j < nst && ok; ++j) {
+                const int o = j % kTOut;
+                ok = qa_wait(bar_out_full(o), (uint32_t)(j / kTOut) & 1u, abort_flag);
+                if (!ok) break;
+                tma_store_2d(&map_q, k0 + j * kTCols, m0, sb + L.region_b + o * kOutTileBytes);
+                bulk_commit();
+                if (j >= 2) {
+                    bulk_wait_read<2>();
+                    mbar_arrive(bar_out_free((j - 2) % kTOut));
+                }
+            }
+            bulk_wait_read<0>();    // shared memory stays valid until the stores have read it
+            mbar_arrive(bar_tail);
+        }
+        __syncwarp();
+        if (r > 0 && CK > 1) {
+            cluster_arrive();
+            cluster_wait();
+            cluster_arrive();
+            cluster_wait();
+        }
+    } else {
+        // ================= consumers =================
+        // ---- sweep 1: row maxima; units with divisors get x~ written back as fp16 ----
+        float amax = 0.f;
+        __half2 hamax = __float2half2_rn(0.f);
+        bool ok = true;
+        for (int i = 0; i < nst; ++i) {
+            const int st = i % kTStages;
+            ok = qa_warp_wait(bar_full(st), (uint32_t)(i / kTStages) & 1u, abort_flag, lane);
+            if (!ok) break;
+            const uint32_t a0 = sb + L.x_ring + st * kXTileBytes + x_off, a1 = a0 ^ 16u;
+            const uint4 v0 = lds128(a0), v1 = lds128(a1);
+            if (ones_sm[i * 4 + cg]) {
+                const __half2* h0 = reinterpret_cast<const __half2*>(&v0);
+                const __half2* h1 = reinterpret_cast<const __half2*>(&v1);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    hamax = __hmax2(hamax, __habs2(h0[e]));
+                    hamax = __hmax2(hamax, __habs2(h1[e]));
+                }
+            } else {
+                const float4* sp = reinterpret_cast<const float4*>(s + k0 + i * kTCols + cg * 16);
+                float v[8];
+                div8(v0, __ldg(sp), __ldg(sp + 1), v);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(v[e]));
+                sts128(a0, pack8_half(v));
+                div8(v1, __ldg(sp + 2), __ldg(sp + 3), v);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(v[e]));
+                sts128(a1, pack8_half(v));
+                fence_proxy_async_smem();       // the MMA reads these through the async proxy
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_ready(st));
+        }
+        amax = fmaxf(amax, fmaxf(__low2float(hamax), __high2float(hamax)));
+        amax_cg[cg * kTTok + row] = amax;
+        named_bar_sync(1, kTConsumers);
+        // ---- row maxima: pushed to every CTA of the cluster (each needs all row scales) ----
+        if (tid < kTTok) {
+            const float a = fmaxf(fmaxf(amax_cg[tid], amax_cg[kTTok + tid]),
+                                  fmaxf(amax_cg[2 * kTTok + tid], amax_cg[3 * kTTok + tid]));
+            const uint32_t slot = sb + L.amax_slots + (rank * kTTok + tid) * 4;
+            for (int qq = 0; qq < CK; ++qq) dsmem_st_f32(dsmem_addr(slot, (uint32_t)qq), a);
+        }
+        cluster_arrive();
+        cluster_wait();         // all row maxima have landed
+
+        // ---- row scale of this thread's row; the owner of a row writes it out ----
+        float sc;
+        {
+            float a = 0.f;
+            for (int qq = 0; qq < CK; ++qq) a = fmaxf(a, amax_slots[qq * kTTok + row]);
+            sc = __fdiv_rn(a, 127.0f);
+        }
+        if (cg == 0 && (int)rank == row / rows_owned && m0 + row < M) a_scale[m0 + row] = sc;
+
+        // ---- sweep 2: int8 codes into the output tiles ----
+        // The tiles take the place of the L_A ring: the MMAs must have finished reading it.
+        if (r > 0 && ok) ok = qa_warp_wait(bar_acc, 0u, abort_flag, lane);
+        const float rcp = (sc > 0.f) ? __frcp_rn(sc) : 0.f;
+        for (int j = 0; j < nst && ok; ++j) {
+            const int i = nst + j, st = i % kTStages, o = j % kTOut;
+            ok = qa_warp_wait(bar_full(st), (uint32_t)(i / kTStages) & 1u, abort_flag, lane);
+            if (!ok) break;
+            const uint32_t a0 = sb + L.x_ring + st * kXTileBytes + x_off, a1 = a0 ^ 16u;
+            const uint4 v0 = lds128(a0), v1 = lds128(a1);
+            uint4 codes;
+            float v[8];
+            if (ones_sm[j * 4 + cg]) {
+                cvt8(v0, v);
+                const uint2 lo = quant8_pairs(v, sc, rcp);
+                cvt8(v1, v);
+                const uint2 hi = quant8_pairs(v, sc, rcp);
+                codes = make_uint4(lo.x, lo.y, hi.x, hi.y);
+            } else {
+                const float4* sp = reinterpret_cast<const float4*>(s + k0 + j * kTCols + cg * 16);
+                div8(v0, __ldg(sp), __ldg(sp + 1), v);
+                const uint2 lo = quant8_pairs(v, sc, rcp);
+                div8(v1, __ldg(sp + 2), __ldg(sp + 3), v);
+                const uint2 hi = quant8_pairs(v, sc, rcp);
+                codes = make_uint4(lo.x, lo.y, hi.x, hi.y);
+            }
+            // The stage is released only now that the loaded values have been consumed: an
+            // arrival issued straight after the loads let the next TMA write overtake them.
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_free2(st));
+            if (j >= kTOut) {       // the store that last read this tile is done with it
+                ok = qa_warp_wait(bar_out_free(o), (uint32_t)(j / kTOut - 1) & 1u, abort_flag, lane);
+                if (!ok) break;
+            }
+            // output tile: rows of 64 bytes, 16-byte piece cg at its 64-byte-swizzle place
+            sts128(sb + L.region_b + o * kOutTileBytes + (uint32_t)row * 64u + (uint32_t)((cg ^ ((row >> 1) & 3)) << 4), codes);
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_out_full(o));
+        }
+
+        // ---- T: partial sums from tensor memory to the CTA that owns the row ----
+        if (r > 0) {
+            if (ok) ok = qa_warp_wait(bar_acc, 0u, abort_flag, lane);
+            tc_fence_after();
+            // a warp reaches the 32 lanes of its quarter (warp % 4); the four warps of a quarter
+            // split the r columns
+            const int q = warp & 3, cpart = warp >> 2, ncol = r >> 2;
+            const int trow = q * 32 + lane;
+            uint32_t dst = 0;
+            if (CK > 1) {
+                // region B is free here once the stores have read the last output tiles, and
+                // at the peers once they say the same
+                if (ok) ok = qa_warp_wait(bar_tail, 0u, abort_flag, lane);
+                cluster_arrive();
+                cluster_wait();
+                const uint32_t owner = (uint32_t)(trow / rows_owned);
+                const int rl = trow - (int)owner * rows_owned;
+                dst = dsmem_addr(sb + L.region_b + (uint32_t)(((int)rank * rows_owned + rl) * r) * 4u, owner);
+            }
+            for (int c4 = 0; c4 < ncol; c4 += 4) {
+                const int col = cpart * ncol + c4;
+                uint32_t v[4];
+                tmem_ld4(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)col, v);
+                if (CK > 1) {
+                    dsmem_st_v4(dst + (uint32_t)col * 4u, v);
+                } else if (m0 + trow < M) {
+                    // a single CTA holds the whole sum
+                    const __nv_bfloat162 p0 = __floats2bfloat162_rn(__uint_as_float(v[0]), __uint_as_float(v[1]));
+                    const __nv_bfloat162 p1 = __floats2bfloat162_rn(__uint_as_float(v[2]), __uint_as_float(v[3]));
+                    uint2 pk;
+                    pk.x = *reinterpret_cast<const uint32_t*>(&p0);
+                    pk.y = *reinterpret_cast<const uint32_t*>(&p1);
+                    *reinterpret_cast<uint2*>(T + (size_t)(m0 + trow) * r + col) = pk;
+                }
+            }
+            tc_fence_before();
+            if (CK > 1) {
+                cluster_arrive();
+                cluster_wait();     // all partial sums have landed; only local reads from here
+                const int pairs = r >> 1;
+                for (int e = tid; e < rows_owned * pairs; e += kTConsumers) {
+                    const int rl = e / pairs, col = (e - rl * pairs) * 2;
+                    const int orow = (int)rank * rows_owned + rl;
+                    float s0 = 0.f, s1 = 0.f;
+                    for (int qq = 0; qq < CK; ++qq) {
+                        const float2 pv = *reinterpret_cast<const float2*>(t_slots + (qq * rows_owned + rl) * r + col);
+                        s0 += pv.x; s1 += pv.y;
                     }
+                    if (m0 + orow < M)
+                        *reinterpret_cast<__nv_bfloat162*>(T + (size_t)(m0 + orow) * r + col) = __floats2bfloat162_rn(s0, s1);
                 }
             }
         }
+        if (*abort_flag && cg == 0 && m0 + row < M) a_scale[m0 + row] = __int_as_float(0x7fc00000);   // a wait gave up: poison the rows
     }
-    cp_async_wait<0>();
-    __syncthreads();        // every warp is done with the L_A stages: their space now holds T
-
-    // ---- publish this CTA's partial results for the cluster ----
-    amax = fmaxf(amax, fmaxf(__low2float(hamax), __high2float(hamax)));
-    // row maximum over this thread's 8-column groups: the 16 threads of a row are adjacent lanes
-#pragma unroll
-    for (int o = 8; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-    if (tcg == 0) amax_part[trow] = amax;
-    if (r > 0) {
-        const int g = lane >> 2, tq = lane & 3;
-#pragma unroll
-        for (int i = 0; i < NTW; ++i) {
-            const int nt = nq + 8 * i;
-            if (nt < ntiles) {
-                const int j = nt * 8 + tq * 2;
-                *reinterpret_cast<float2*>(t_part + (mt * 16 + g) * r + j) = make_float2(acc[i][0], acc[i][1]);
-                *reinterpret_cast<float2*>(t_part + (mt * 16 + g + 8) * r + j) = make_float2(acc[i][2], acc[i][3]);
-            }
-        }
-    }
-    cluster_sync_all();
-
-    // ---- row scales: maximum over the K-slices (every CTA needs them for its own slice) ----
-    if (tid < kCTok) {
-        float a = 0.f;
-        for (int q = 0; q < CK; ++q) a = fmaxf(a, dsmem_ld_f32(sb + L.amax_part + tid * 4, q));
-        const float sc = __fdiv_rn(a, 127.0f);
-        scale_sm[tid] = sc;
-        if (rank == 0 && m0 + tid < M) a_scale[m0 + tid] = sc;
-    }
-    // ---- T: sum of the partial products; the cluster's CTAs share the elements ----
-    if (r > 0) {
-        for (int e = (int)rank * kCThreads + tid; e < kCTok * r; e += CK * kCThreads) {
-            float sum = 0.f;
-            for (int q = 0; q < CK; ++q) sum += dsmem_ld_f32(sb + L.t_part + e * 4, q);
-            const int row = e / r, j = e - row * r;
-            if (m0 + row < M) T[(size_t)(m0 + row) * r + j] = __float2bfloat16_rn(sum);
-        }
-    }
-    cluster_sync_all();      // nobody leaves (or reuses shared memory) while peers still read it
-
-    // ---- sweep 2: int8 codes of the resident slice ----
-    if (!row_ok) return;
-    const float sc = scale_sm[trow];
-    int8_t* out = Xq + (size_t)(m0 + trow) * K + k0;
-    if (!(sc > 0.f)) {   // all-zero token: codes 0
-        for (int c = 0; c < nch; ++c) *reinterpret_cast<uint2*>(out + c * kCChunk + tcg * 8) = make_uint2(0, 0);
-        return;
-    }
-    const float rcp = __frcp_rn(sc);
-    for (int c = 0; c < nch; ++c) {
-        const uint4 raw = *reinterpret_cast<const uint4*>(smem + L.x_raw + trow * xrow_bytes + c * (kCChunk * 2) + tcg * 16);
-        float v[8];
-        if (ones_sm[c * (kCChunk / 8) + tcg]) {
-            const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const float2 f = __half22float2(h2[i]);
-                v[2 * i] = f.x; v[2 * i + 1] = f.y;
-            }
-        } else {
-            const float4 s0 = *reinterpret_cast<const float4*>(s_sm + c * kCChunk + tcg * 8);
-            const float4 s1 = *reinterpret_cast<const float4*>(s_sm + c * kCChunk + tcg * 8 + 4);
-            RawChunk rc{raw, s0, s1};
-            smooth8(rc, v);
-        }
-        *reinterpret_cast<uint2*>(out + c * kCChunk + tcg * 8) = quant8_fast(v, sc, rcp);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kTWarpMma && r > 0) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols) : "memory");
     }
 }
 
-// Smallest cluster size (<= 8) whose K-slice fits shared memory and is a whole number of chunks.
-int pick_cluster(int K, int r) {
-    for (int ck = 1; ck <= 8; ++ck) {
-        if (K % ck) continue;
-        const int kc = K / ck;
-        if (kc % kCChunk) continue;
-        if (cluster_smem(kc, r).total <= 226 * 1024 && kc <= 2048) return ck;
-    }
-    return 0;
-}
-
-template <int NTW, int STG>
-int launch_cluster(const __half* X, const float* s, const __half* LA, int M, int K, int r, int ck,
-                   int8_t* Xq, float* a_scale, __nv_bfloat16* T, cudaStream_t st) {
-    const int kc = K / ck;
-    const size_t smem = (size_t)cluster_smem(kc, r).total;
-    static size_t configured = 0;
-    if (smem > configured) {
-        cudaError_t e = cudaFuncSetAttribute(quant_act_cluster_kernel<NTW, STG>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return record_cuda_error(e, "quant_act_cluster smem attribute");
-        configured = smem;
-    }
+// Clusters of `ck` CTAs of this kernel that the device keeps resident at once (0 if it cannot
+// schedule that size).  Queried once per (size, shared memory) pair.
+int tma_active_clusters(int ck, size_t smem) {
+    static int cached[17];
+    static size_t cached_smem[17];
+    if (cached_smem[ck] == smem && smem != 0) return cached[ck];
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(ck, (M + kCTok - 1) / kCTok, 1);
-    cfg.blockDim = dim3(kCThreads, 1, 1);
+    cfg.gridDim = dim3(ck, 1, 1);
+    cfg.blockDim = dim3(kTThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = ck;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, quant_act_tma_kernel, &cfg) != cudaSuccess) {
+        (void)cudaGetLastError();
+        n = 0;
+    }
+    cached[ck] = n;
+    cached_smem[ck] = smem;
+    return n;
+}
+
+// Cluster size for the TMA kernel: a power of two (the CTAs split the 128 rows of T) that
+// divides the K / 64 column blocks.  Larger clusters shorten a CTA's two sweeps but fewer of
+// them are resident at once; the estimate is waves x (fixed cost + stages), in stage units.
+int pick_tma_cluster(int M, int K, int r, int max_ck) {
+    const int tiles = (M + kTTok - 1) / kTTok, blocks = K / kTCols;
+    int best = 0;
+    long long best_cost = 0;
+    for (int ck = 1; ck <= max_ck; ck *= 2) {
+        if (blocks % ck || blocks / ck < 2) continue;
+        const size_t smem = (size_t)tma_smem(K / ck, r).total;
+        if (smem > 227 * 1024) continue;
+        const int active = tma_active_clusters(ck, smem);
+        if (active < 1) continue;
+        const long long waves = (tiles + active - 1) / active;
+        const long long cost = waves * (6 + blocks / ck);
+        if (best == 0 || cost < best_cost) { best = ck; best_cost = cost; }
+    }
+    return best;
+}
+
+int launch_tma(const __half* X, const float* s, const __half* LA, int M, int K, int r,
+               int8_t* Xq, float* a_scale, __nv_bfloat16* T, cudaStream_t st, bool* unsupported) {
+    *unsupported = false;
+    static int max_ck = 0;      // 16 where the device allows clusters beyond the portable 8
+    if (max_ck == 0) {
+        cudaError_t e = cudaFuncSetAttribute(quant_act_tma_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        max_ck = (e == cudaSuccess) ? 16 : 8;
+        if (e != cudaSuccess) (void)cudaGetLastError();
+        e = cudaFuncSetAttribute(quant_act_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e != cudaSuccess) return record_cuda_error(e, "quant_act_tma smem attribute");
+    }
+    if ((M + kTTok - 1) / kTTok > 65535) { *unsupported = true; return ASER_OK; }
+    const int ck = pick_tma_cluster(M, K, r, max_ck);
+    if (ck == 0) { *unsupported = true; return ASER_OK; }
+    const int kc = K / ck;
+    const size_t smem = (size_t)tma_smem(kc, r).total;
+    CUtensorMap mx, mla, mq;
+    int rc = encode_map_2d(&mx, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, X, M, K, kTTok, kTCols, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (rc != ASER_OK) return rc;
+    if (r > 0) {
+        rc = encode_map_2d(&mla, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, LA, r, K, r, kTCols, CU_TENSOR_MAP_SWIZZLE_128B);
+        if (rc != ASER_OK) return rc;
+    } else {
+        mla = mx;
+    }
+    rc = encode_map_2d(&mq, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Xq, M, K, kTTok, kTCols, CU_TENSOR_MAP_SWIZZLE_64B);
+    if (rc != ASER_OK) return rc;
+
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(ck, (M + kTTok - 1) / kTTok, 1);
+    cfg.blockDim = dim3(kTThreads, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -626,10 +967,9 @@ int launch_cluster(const __half* X, const float* s, const __half* LA, int M, int
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, quant_act_cluster_kernel<NTW, STG>, X, s, LA, M, K, kc, r, ck,
-                                       Xq, a_scale, T);
-    if (e != cudaSuccess) return record_cuda_error(e, "quant_act_cluster_kernel");
-    return check_launch("quant_act_cluster_kernel");
+    cudaError_t e = cudaLaunchKernelEx(&cfg, quant_act_tma_kernel, mx, mla, mq, s, M, K, kc, r, ck, a_scale, T);
+    if (e != cudaSuccess) return record_cuda_error(e, "quant_act_tma_kernel");
+    return check_launch("quant_act_tma_kernel");
 }
 
 template <int MAXT>
@@ -666,12 +1006,9 @@ int launch_quant_act(const __half* X, const float* s, const __half* LA, int M, i
         quant_act_small_kernel<<<grid, kSmallThreads, smem, st>>>(X, s, LA, M, K, r, Xq, a_scale, T);
         return check_launch("quant_act_small_kernel");
     }
-    const int ck = pick_cluster(K, r);
-    if (ck > 0 && (long long)((M + kCTok - 1) / kCTok) <= 65535) {
-        if (r <= 64) return launch_cluster<1, 3>(X, s, LA, M, K, r, ck, Xq, a_scale, T, st);
-        if (r <= 128) return launch_cluster<2, 2>(X, s, LA, M, K, r, ck, Xq, a_scale, T, st);
-        return launch_cluster<4, 2>(X, s, LA, M, K, r, ck, Xq, a_scale, T, st);
-    }
+    bool unsupported = false;
+    const int rc = launch_tma(X, s, LA, M, K, r, Xq, a_scale, T, st, &unsupported);
+    if (!unsupported) return rc;
     if (r <= 64) return launch_large<1>(X, s, LA, M, K, r, Xq, a_scale, T, st);
     if (r <= 128) return launch_large<2>(X, s, LA, M, K, r, Xq, a_scale, T, st);
     return launch_large<4>(X, s, LA, M, K, r, Xq, a_scale, T, st);

@@ -326,62 +326,80 @@ quant_act_large_kernel(const __half* __restrict__ X, const float* __restrict__ s
 // ---------------------------------------------------------------------------
 // many tokens: TMA ring + tcgen05 down projection, thread-block cluster split along K
 // ---------------------------------------------------------------------------
-// A cluster of CK CTAs owns 128 tokens (the MMA's M side); CTA `rank` owns the K-slice
-// [rank*Kc, (rank+1)*Kc) and streams it twice through a ring of 64-column stages filled by TMA
-// (128-byte swizzle, rows past M read as zero).
+// A cluster of CK CTAs owns 64 tokens; CTA `rank` owns the K-slice [rank*Kc, (rank+1)*Kc) and
+// streams it twice through a ring of 128-column stages filled by TMA (two 64-column tiles per
+// stage, 128-byte swizzle, rows past M read as zero).
 //   Sweep 1: the consumer warps scan each stage for the row maximum of |x~|.  Where all 16
 //   divisors of a (row, 16-column) unit are 1 (all but the outlier channels), x~ is the fp16
 //   input itself and the stage is left as TMA wrote it; elsewhere x~ = x / s is computed in
-//   fp32 and written back as fp16 in place.  One thread then issues tcgen05.mma (kind::f16,
-//   M = 128 tokens, N = r) with the stage as the A operand and the L_A tile (TMA) as B; the
-//   partial T accumulates in tensor memory.
-//   Exchange: row maxima and partial T go through distributed shared memory; every CTA of the
-//   cluster gets the row scales, and the cluster's CTAs share the summation of T.
+//   fp32 and written back as fp16 in place.  One thread then issues tcgen05.mma (kind::f16)
+//   with the L_A tile (TMA) on the M side and the stage's 64 tokens on the N side, so the
+//   partial T accumulates transposed, D[j, token], in tensor memory.  L_A has fewer than 128
+//   rows when r < 128; the MMA then also reads the shared memory behind the tile and the
+//   accumulator rows j >= r are never looked at.
+//   Exchange: every CTA stores its row maxima into all CTAs of the cluster and its partial T
+//   into the CTA that owns the token (64 / CK tokens each), through distributed shared memory;
+//   one cluster barrier publishes both.  The owner sums the CK partials and writes T.
 //   Sweep 2: the slice is streamed again (it was just read, so it comes from L2), quantized,
-//   staged in shared memory (64-byte swizzle) and written by TMA stores, which also clip rows
-//   past M.
+//   staged in shared memory and written by TMA stores, which also clip rows past M.
 // A warp handles one 16-column group for 32 rows (lane = row), so whether a unit needs the
 // division is uniform across the warp and the swizzled 16-byte accesses are conflict-free.
-constexpr int kTTok = 128;                  // tokens per cluster
-constexpr int kTCols = 64;                  // columns per stage: one 128-byte swizzle row of fp16
+// A kernel that allocates tensor memory gets one CTA per SM, so the CTA uses most of the SM's
+// shared memory.
+constexpr int kTTok = 64;                   // tokens per cluster (the MMA's N)
+constexpr int kTAtom = 64;                  // columns of one swizzled tile: 128 bytes of fp16
+constexpr int kTCols = 128;                 // columns per stage (two tiles)
 constexpr int kTConsumerWarps = 16;         // warp = (32-row block, 16-column group)
 constexpr int kTConsumers = kTConsumerWarps * 32;
 constexpr int kTWarpProd = kTConsumerWarps;         // TMA producer warp
 constexpr int kTWarpMma = kTConsumerWarps + 1;      // MMA issuer warp, owns the tensor memory
 constexpr int kTThreads = kTConsumers + 64;
-constexpr int kTStages = 4;                 // activation / L_A ring depth
+constexpr int kTMaxStages = 4;              // activation / L_A ring depth (3 when r > 64)
 constexpr int kTOut = 4;                    // int8 output tiles in flight
-constexpr int kXTileBytes = kTTok * 128;    // 128 rows x 64 fp16
-constexpr int kOutTileBytes = kTTok * 64;   // 128 rows x 64 int8
+constexpr int kTMaxRank = 128;              // larger r takes the mma.sync kernel
+constexpr int kXAtomBytes = kTTok * 128;    // 64 rows x 64 fp16
+constexpr int kXStageBytes = 2 * kXAtomBytes;
+constexpr int kOutTileBytes = kTTok * kTCols;   // 64 rows x 128 int8
 constexpr long long kQaWaitLimitClocks = 4000000000ll;   // about 2 s of SM clocks per wait
 
+__host__ __device__ constexpr int tma_stages(int r) { return r <= 64 ? 4 : 3; }
+
 struct TmaSmem {
-    int x_ring, region_b, la_bytes, ones, amax_cg, amax_slots, bars, tmem_slot, abort_flag, total;
+    int x_ring, region_b, la_atom_bytes, la_stage_bytes, t_slots, ones, amax_cg, amax_slots, bars,
+        tmem_slot, abort_flag, total;
 };
-// Offsets from the 1 KiB-aligned base.  Region B holds, one after the other in time: the L_A
-// ring (sweep 1), the output tiles (sweep 2), and the partial T pushed by the cluster's CTAs for
-// the rows this CTA owns, as [source CTA][row][r] floats (128 * r floats in all).
-__host__ __device__ inline TmaSmem tma_smem(int Kc, int r) {
+// Offsets from the 1 KiB-aligned base.  Region B holds the L_A ring in sweep 1 and the output
+// tiles in sweep 2.  t_slots receives the partial T of the tokens this CTA owns from every CTA
+// of the cluster, as [source CTA][token][r] floats (64 * r floats in all).  It follows region B
+// so that an MMA whose L_A tile has fewer than 128 rows still reads inside the allocation.
+__host__ __device__ inline TmaSmem tma_smem(int Kc, int r, int CK) {
     TmaSmem L;
+    const int ns = tma_stages(r);
     int off = 0;
-    L.x_ring = off;     off += kTStages * kXTileBytes;
+    L.x_ring = off;     off += ns * kXStageBytes;
     L.region_b = off;
-    L.la_bytes = r * 128;
+    L.la_atom_bytes = r * 128;
+    L.la_stage_bytes = 2 * L.la_atom_bytes;
     {
-        int b = kTStages * L.la_bytes;                         // = 128 * r * 4, the pushed partials
+        int b = ns * L.la_stage_bytes;
         if (kTOut * kOutTileBytes > b) b = kTOut * kOutTileBytes;
         off += (b + 1023) / 1024 * 1024;
     }
+    L.t_slots = off;
+    {
+        int b = (CK > 1) ? kTTok * r * 4 : 0;
+        if (b < 16 * 1024) b = 16 * 1024;                      // readable space behind the L_A ring
+        off += b;
+    }
     L.ones = off;       off += (Kc / 16 + 15) / 16 * 16;       // per 16 columns: all divisors are 1
-    L.amax_cg = off;    off += 4 * kTTok * 4;                  // row maxima per 16-column group
-    L.amax_slots = off; off += 16 * kTTok * 4;                 // row maxima pushed by each CTA
-    L.bars = off;       off += (4 * kTStages + 2 * kTOut + 2) * 8;
+    L.amax_cg = off;    off += 8 * kTTok * 4;                  // row maxima per 16-column group
+    L.amax_slots = off; off += 16 * kTTok * 4;                 // row maxima stored by each CTA
+    L.bars = off;       off += (4 * kTMaxStages + 2 * kTOut + 1) * 8;
     L.tmem_slot = off;  off += 8;
     L.abort_flag = off; off += 8;
     L.total = off + 1024;                                      // slack for the alignment
     return L;
 }
-static_assert(kTStages == 4, "region B: the L_A ring and the pushed partial T have the same size");
 
 __device__ __forceinline__ uint32_t cluster_rank() {
     uint32_t r;
@@ -403,9 +421,6 @@ __device__ __forceinline__ uint32_t dsmem_addr(uint32_t local_addr, uint32_t ran
 // Stores into a peer's shared memory; the cluster barrier publishes them.
 __device__ __forceinline__ void dsmem_st_f32(uint32_t remote, float v) {
     asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
-}
-__device__ __forceinline__ void dsmem_st_v4(uint32_t remote, const uint32_t (&v)[4]) {
-    asm volatile("st.shared::cluster.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(remote), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]) : "memory");
 }
 
 // Bounded wait on an mbarrier phase.  On expiry (or when another thread of the CTA has given
@@ -446,13 +461,6 @@ __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.comm
 template <int N>
 __device__ __forceinline__ void bulk_wait_read() {
     asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
-}
-__device__ __forceinline__ void tmem_ld4(uint32_t taddr, uint32_t (&v)[4]) {
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3])
-                 : "r"(taddr)
-                 : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3])::"memory");
 }
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     uint4 v;
@@ -526,11 +534,12 @@ __device__ __forceinline__ uint2 quant8_pairs(const float (&v)[8], float sc, flo
     return make_uint2(__byte_perm(a01, a23, 0x5410), __byte_perm(a45, a67, 0x5410));
 }
 
-// grid = (CK, ceil(M / 128)), cluster = (CK, 1, 1) with CK a power of two <= 16, kTThreads threads.
-// map_x: X as fp16 [M, K], box 128 rows x 64 columns, 128-byte swizzle.
+// grid = (CK, ceil(M / 64)), cluster = (CK, 1, 1) with CK a power of two <= 16, kTThreads threads,
+// r <= 128.
+// map_x: X as fp16 [M, K], box 64 rows x 64 columns, 128-byte swizzle.
 // map_la: L_A as fp16 [r, K], box r rows x 64 columns, 128-byte swizzle (unused when r == 0).
-// map_q: Xq as bytes [M, K], box 128 rows x 64 columns, 64-byte swizzle.
-__global__ void __launch_bounds__(kTThreads, 2)
+// map_q: Xq as bytes [M, K], box 64 rows x 128 columns, 128-byte swizzle.
+__global__ void __launch_bounds__(kTThreads, 1)
 quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_la,
                      const __grid_constant__ CUtensorMap map_q, const float* __restrict__ s,
                      int M, int K, int Kc, int r, int CK, float* __restrict__ a_scale,
@@ -539,53 +548,60 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     const uint32_t sraw = smem_u32(smem_raw);
     const uint32_t sb = (sraw + 1023u) & ~1023u;            // swizzled tiles need 1 KiB alignment
     uint8_t* smem = smem_raw + (sb - sraw);
-    const TmaSmem L = tma_smem(Kc, r);
+    const TmaSmem L = tma_smem(Kc, r, CK);
+    const int NS = tma_stages(r);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t rank = cluster_rank();
     const int m0 = blockIdx.y * kTTok;
     const int k0 = (int)rank * Kc;
     const int nst = Kc / kTCols;                            // stages per sweep
-    const int rows_owned = kTTok / CK;                      // rows of T this CTA sums and writes
+    const int rows_owned = kTTok / CK;                      // tokens whose T this CTA sums and writes
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L.abort_flag);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L.tmem_slot);
     uint8_t* ones_sm = smem + L.ones;
     float* amax_cg = reinterpret_cast<float*>(smem + L.amax_cg);
     float* amax_slots = reinterpret_cast<float*>(smem + L.amax_slots);
-    float* t_slots = reinterpret_cast<float*>(smem + L.region_b);
+    float* t_slots = reinterpret_cast<float*>(smem + L.t_slots);
     auto bar_full = [&](int st) { return sb + L.bars + st * 8; };
-    auto bar_ready = [&](int st) { return sb + L.bars + (kTStages + st) * 8; };
-    auto bar_free1 = [&](int st) { return sb + L.bars + (2 * kTStages + st) * 8; };
-    auto bar_free2 = [&](int st) { return sb + L.bars + (3 * kTStages + st) * 8; };
-    auto bar_out_full = [&](int o) { return sb + L.bars + (4 * kTStages + o) * 8; };
-    auto bar_out_free = [&](int o) { return sb + L.bars + (4 * kTStages + kTOut + o) * 8; };
-    const uint32_t bar_acc = sb + L.bars + (4 * kTStages + 2 * kTOut) * 8;
-    const uint32_t bar_tail = bar_acc + 8;      // the output tiles are no longer in use
-    uint32_t tmem_cols = 32;
-    while ((int)tmem_cols < r) tmem_cols <<= 1;
+    auto bar_ready = [&](int st) { return sb + L.bars + (kTMaxStages + st) * 8; };
+    auto bar_free1 = [&](int st) { return sb + L.bars + (2 * kTMaxStages + st) * 8; };
+    auto bar_free2 = [&](int st) { return sb + L.bars + (3 * kTMaxStages + st) * 8; };
+    auto bar_out_full = [&](int o) { return sb + L.bars + (4 * kTMaxStages + o) * 8; };
+    auto bar_out_free = [&](int o) { return sb + L.bars + (4 * kTMaxStages + kTOut + o) * 8; };
+    const uint32_t bar_acc = sb + L.bars + (4 * kTMaxStages + 2 * kTOut) * 8;
+    constexpr uint32_t kTmemCols = 64;                      // D[j, token]: 64 token columns
 
     // Use i of the ring: i < nst is sweep 1 (X and L_A tiles), the rest sweep 2 (X only).
     // A stage's previous use was released by the MMAs (sweep 1) or the consumers (sweep 2).
     auto load_use = [&](int i) -> bool {
-        const int st = i % kTStages;
-        if (i >= kTStages) {
-            const int prev = i - kTStages;
+        const int st = i % NS;
+        if (i >= NS) {
+            const int prev = i - NS;
             bool ok;
             if (prev < nst) {
-                ok = qa_wait(bar_free1(st), (uint32_t)(prev / kTStages) & 1u, abort_flag);
+                ok = qa_wait(bar_free1(st), (uint32_t)(prev / NS) & 1u, abort_flag);
             } else {
-                const int first = nst + ((st - nst % kTStages + kTStages) % kTStages);
-                ok = qa_wait(bar_free2(st), (uint32_t)((prev - first) / kTStages) & 1u, abort_flag);
+                const int first = nst + ((st - nst % NS + NS) % NS);
+                ok = qa_wait(bar_free2(st), (uint32_t)((prev - first) / NS) & 1u, abort_flag);
             }
             if (!ok) return false;
         }
-        const uint32_t xdst = sb + L.x_ring + st * kXTileBytes;
+        const uint32_t xdst = sb + L.x_ring + st * kXStageBytes;
         if (i < nst) {
-            mbar_arrive_expect_tx(bar_full(st), (uint32_t)(kXTileBytes + L.la_bytes));
-            tma_load_2d(xdst, &map_x, k0 + i * kTCols, m0, bar_full(st));
-            if (r > 0) tma_load_2d(sb + L.region_b + st * L.la_bytes, &map_la, k0 + i * kTCols, 0, bar_full(st));
+            const int kcol = k0 + i * kTCols;
+            mbar_arrive_expect_tx(bar_full(st), (uint32_t)(kXStageBytes + L.la_stage_bytes));
+            tma_load_2d(xdst, &map_x, kcol, m0, bar_full(st));
+            tma_load_2d(xdst + kXAtomBytes, &map_x, kcol + kTAtom, m0, bar_full(st));
+            if (r > 0) {
+                const uint32_t ldst = sb + L.region_b + st * L.la_stage_bytes;
+                tma_load_2d(ldst, &map_la, kcol, 0, bar_full(st));
+                tma_load_2d(ldst + L.la_atom_bytes, &map_la, kcol + kTAtom, 0, bar_full(st));
+            }
         } else {
-            mbar_arrive_expect_tx(bar_full(st), (uint32_t)kXTileBytes);
-            tma_load_2d(xdst, &map_x, k0 + (i - nst) * kTCols, m0, bar_full(st));
+            const int kcol = k0 + (i - nst) * kTCols;
+            mbar_arrive_expect_tx(bar_full(st), (uint32_t)kXStageBytes);
+            tma_load_2d(xdst, &map_x, kcol, m0, bar_full(st));
+            tma_load_2d(xdst + kXAtomBytes, &map_x, kcol + kTAtom, m0, bar_full(st));
         }
         return true;
     };
@@ -594,7 +610,7 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     if (warp == kTWarpProd) {
         // The producer sets up the barriers and fills the ring before anyone else is ready.
         if (lane == 0) {
-            for (int st = 0; st < kTStages; ++st) {
+            for (int st = 0; st < kTMaxStages; ++st) {
                 mbar_init(bar_full(st), 1);                     // the producer's expect_tx arrival
                 mbar_init(bar_ready(st), kTConsumerWarps);      // consumers are done with the stage
                 mbar_init(bar_free1(st), 1);                    // sweep 1: the MMAs have read it
@@ -605,17 +621,16 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 mbar_init(bar_out_free(o), 1);                  // its store has read it
             }
             mbar_init(bar_acc, 1);
-            mbar_init(bar_tail, 1);
             *abort_flag = 0;
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
             fence_proxy_async_smem();
-            for (int i = 0; i < kTStages && i < 2 * nst; ++i) load_use(i);      // no waits yet
+            for (int i = 0; i < NS && i < 2 * nst; ++i) load_use(i);      // no waits yet
         }
         __syncwarp();
     } else if (warp == kTWarpMma) {
         if (r > 0) {
             asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                         ::"r"(smem_u32(tmem_slot)), "r"(tmem_cols)
+                         ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols)
                          : "memory");
             asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
         }
@@ -640,50 +655,42 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     tc_fence_after();
     const uint32_t tmem = (r > 0) ? *tmem_slot : 0u;
 
-    // this thread's unit inside a stage (consumer warps): row and 16-column group
-    const int rb = warp >> 2, cg = warp & 3;
-    const int row = rb * 32 + lane;
-    // 16-byte pieces 2cg and 2cg+1 of the row, at their swizzled places (they differ in bit 4)
-    const uint32_t x_off = (uint32_t)row * 128u + (uint32_t)(((2 * cg) ^ (row & 7)) << 4);
-
     if (warp == kTWarpProd) {
         // ================= TMA producer =================
         // Uses whose stage is released by sweep 1 come before the exchange; the rest wait for
         // the consumers' sweep 2, which starts after the cluster barrier this warp takes part in.
-        const int early = (2 * nst < nst + kTStages) ? 2 * nst : nst + kTStages;
+        const int early = (2 * nst < nst + NS) ? 2 * nst : nst + NS;
         bool ok = true;
         if (lane == 0) {
-            for (int i = kTStages; i < early && ok; ++i) ok = load_use(i);
+            for (int i = NS; i < early && ok; ++i) ok = load_use(i);
         }
         __syncwarp();
         cluster_arrive();
         cluster_wait();
         if (lane == 0) {
-            for (int i = (early > kTStages ? early : kTStages); i < 2 * nst && ok; ++i) ok = load_use(i);
+            for (int i = (early > NS ? early : NS); i < 2 * nst && ok; ++i) ok = load_use(i);
         }
         __syncwarp();
-        if (r > 0 && CK > 1) {      // the exchange of T at the end
-            cluster_arrive();
-            cluster_wait();
-            cluster_arrive();
-            cluster_wait();
-        }
     } else if (warp == kTWarpMma) {
         // ================= MMA issuer, then store issuer =================
         bool ok = true;
         if (lane == 0) {
-            const uint32_t idesc = make_idesc(1u, 0u, (uint32_t)kTTok, (uint32_t)r);
+            // M = 128 rows of L_A (r of them real), N = 64 tokens
+            const uint32_t idesc = make_idesc(1u, 0u, 128u, (uint32_t)kTTok);
             for (int i = 0; i < nst; ++i) {
-                const int st = i % kTStages;
-                ok = qa_wait(bar_ready(st), (uint32_t)(i / kTStages) & 1u, abort_flag);
+                const int st = i % NS;
+                ok = qa_wait(bar_ready(st), (uint32_t)(i / NS) & 1u, abort_flag);
                 if (!ok) break;
                 if (r > 0) {
                     tc_fence_after();
-                    const uint64_t adesc = smem_desc_sw128(sb + L.x_ring + st * kXTileBytes);
-                    const uint64_t bdesc = smem_desc_sw128(sb + L.region_b + st * L.la_bytes);
 #pragma unroll
-                    for (int kk = 0; kk < kTCols / 16; ++kk)
-                        mma_f16_ss(tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, (i != 0 || kk != 0) ? 1u : 0u);
+                    for (int a = 0; a < 2; ++a) {
+                        const uint64_t adesc = smem_desc_sw128(sb + L.region_b + st * L.la_stage_bytes + a * L.la_atom_bytes);
+                        const uint64_t bdesc = smem_desc_sw128(sb + L.x_ring + st * kXStageBytes + a * kXAtomBytes);
+#pragma unroll
+                        for (int kk = 0; kk < kTAtom / 16; ++kk)
+                            mma_f16_ss(tmem, adesc + 2 * kk, bdesc + 2 * kk, idesc, (i != 0 || a != 0 || kk != 0) ? 1u : 0u);
+                    }
                     tc_commit(bar_free1(st));
                 } else {
                     mbar_arrive(bar_free1(st));
@@ -709,28 +716,27 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 }
             }
             bulk_wait_read<0>();    // shared memory stays valid until the stores have read it
-            mbar_arrive(bar_tail);
         }
         __syncwarp();
-        if (r > 0 && CK > 1) {
-            cluster_arrive();
-            cluster_wait();
-            cluster_arrive();
-            cluster_wait();
-        }
     } else {
         // ================= consumers =================
+        // this thread's unit inside a stage: row and 16-column group (two 16-byte pieces of one
+        // swizzled tile; their places differ in address bit 4)
+        const int rb = warp >> 3, cg = warp & 7;
+        const int row = rb * 32 + lane;
+        const uint32_t x_off = (uint32_t)(cg >> 2) * kXAtomBytes + (uint32_t)row * 128u +
+                               (uint32_t)(((2 * (cg & 3)) ^ (row & 7)) << 4);
         // ---- sweep 1: row maxima; units with divisors get x~ written back as fp16 ----
         float amax = 0.f;
         __half2 hamax = __float2half2_rn(0.f);
         bool ok = true;
         for (int i = 0; i < nst; ++i) {
-            const int st = i % kTStages;
-            ok = qa_warp_wait(bar_full(st), (uint32_t)(i / kTStages) & 1u, abort_flag, lane);
+            const int st = i % NS;
+            ok = qa_warp_wait(bar_full(st), (uint32_t)(i / NS) & 1u, abort_flag, lane);
             if (!ok) break;
-            const uint32_t a0 = sb + L.x_ring + st * kXTileBytes + x_off, a1 = a0 ^ 16u;
+            const uint32_t a0 = sb + L.x_ring + st * kXStageBytes + x_off, a1 = a0 ^ 16u;
             const uint4 v0 = lds128(a0), v1 = lds128(a1);
-            if (ones_sm[i * 4 + cg]) {
+            if (ones_sm[i * 8 + cg]) {
                 const __half2* h0 = reinterpret_cast<const __half2*>(&v0);
                 const __half2* h1 = reinterpret_cast<const __half2*>(&v1);
 #pragma unroll
@@ -757,15 +763,45 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         amax = fmaxf(amax, fmaxf(__low2float(hamax), __high2float(hamax)));
         amax_cg[cg * kTTok + row] = amax;
         named_bar_sync(1, kTConsumers);
-        // ---- row maxima: pushed to every CTA of the cluster (each needs all row scales) ----
+        // ---- row maxima: stored into every CTA of the cluster (each needs all row scales) ----
         if (tid < kTTok) {
-            const float a = fmaxf(fmaxf(amax_cg[tid], amax_cg[kTTok + tid]),
-                                  fmaxf(amax_cg[2 * kTTok + tid], amax_cg[3 * kTTok + tid]));
+            float a = amax_cg[tid];
+#pragma unroll
+            for (int g = 1; g < 8; ++g) a = fmaxf(a, amax_cg[g * kTTok + tid]);
             const uint32_t slot = sb + L.amax_slots + (rank * kTTok + tid) * 4;
             for (int qq = 0; qq < CK; ++qq) dsmem_st_f32(dsmem_addr(slot, (uint32_t)qq), a);
         }
+        // ---- partial T: tensor memory -> the CTA that owns the token ----
+        if (r > 0) {
+            if (ok) ok = qa_warp_wait(bar_acc, 0u, abort_flag, lane);
+            tc_fence_after();
+            // A warp reaches the 32 lanes (rows j of L_A) of its quarter, warp % 4; the four warps
+            // of a quarter take 16 tokens each.
+            const int q = warp & 3, t0 = (warp >> 2) * 16;
+            const int j = q * 32 + lane;
+            if (q * 32 < r) {
+                uint32_t v[16];
+                tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)t0, v);
+                tmem_wait_ld(v);
+                if (j < r) {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        const int t = t0 + e;
+                        if (CK > 1) {
+                            const uint32_t owner = (uint32_t)(t / rows_owned);
+                            const int tl = t - (int)owner * rows_owned;
+                            const uint32_t dst = sb + L.t_slots + (uint32_t)((((int)rank * rows_owned + tl) * r + j) * 4);
+                            dsmem_st_f32(dsmem_addr(dst, owner), __uint_as_float(v[e]));
+                        } else if (m0 + t < M) {
+                            T[(size_t)(m0 + t) * r + j] = __float2bfloat16_rn(__uint_as_float(v[e]));
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+        }
         cluster_arrive();
-        cluster_wait();         // all row maxima have landed
+        cluster_wait();         // row maxima and partial T have landed; only local accesses from here
 
         // ---- row scale of this thread's row; the owner of a row writes it out ----
         float sc;
@@ -776,26 +812,25 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         }
         if (cg == 0 && (int)rank == row / rows_owned && m0 + row < M) a_scale[m0 + row] = sc;
 
-        // ---- sweep 2: int8 codes into the output tiles ----
-        // The tiles take the place of the L_A ring: the MMAs must have finished reading it.
-        if (r > 0 && ok) ok = qa_warp_wait(bar_acc, 0u, abort_flag, lane);
+        // ---- sweep 2: int8 codes into the output tiles (they take the place of the L_A ring;
+        // the wait on the accumulator above says the MMAs are done reading it) ----
         const float rcp = (sc > 0.f) ? __frcp_rn(sc) : 0.f;
-        for (int j = 0; j < nst && ok; ++j) {
-            const int i = nst + j, st = i % kTStages, o = j % kTOut;
-            ok = qa_warp_wait(bar_full(st), (uint32_t)(i / kTStages) & 1u, abort_flag, lane);
+        for (int jj = 0; jj < nst && ok; ++jj) {
+            const int i = nst + jj, st = i % NS, o = jj % kTOut;
+            ok = qa_warp_wait(bar_full(st), (uint32_t)(i / NS) & 1u, abort_flag, lane);
             if (!ok) break;
-            const uint32_t a0 = sb + L.x_ring + st * kXTileBytes + x_off, a1 = a0 ^ 16u;
+            const uint32_t a0 = sb + L.x_ring + st * kXStageBytes + x_off, a1 = a0 ^ 16u;
             const uint4 v0 = lds128(a0), v1 = lds128(a1);
             uint4 codes;
             float v[8];
-            if (ones_sm[j * 4 + cg]) {
+            if (ones_sm[jj * 8 + cg]) {
                 cvt8(v0, v);
                 const uint2 lo = quant8_pairs(v, sc, rcp);
                 cvt8(v1, v);
                 const uint2 hi = quant8_pairs(v, sc, rcp);
                 codes = make_uint4(lo.x, lo.y, hi.x, hi.y);
             } else {
-                const float4* sp = reinterpret_cast<const float4*>(s + k0 + j * kTCols + cg * 16);
+                const float4* sp = reinterpret_cast<const float4*>(s + k0 + jj * kTCols + cg * 16);
                 div8(v0, __ldg(sp), __ldg(sp + 1), v);
                 const uint2 lo = quant8_pairs(v, sc, rcp);
                 div8(v1, __ldg(sp + 2), __ldg(sp + 3), v);
@@ -806,68 +841,30 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             // arrival issued straight after the loads let the next TMA write overtake them.
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_free2(st));
-            if (j >= kTOut) {       // the store that last read this tile is done with it
-                ok = qa_warp_wait(bar_out_free(o), (uint32_t)(j / kTOut - 1) & 1u, abort_flag, lane);
+            if (jj >= kTOut) {      // the store that last read this tile is done with it
+                ok = qa_warp_wait(bar_out_free(o), (uint32_t)(jj / kTOut - 1) & 1u, abort_flag, lane);
                 if (!ok) break;
             }
-            // output tile: rows of 64 bytes, 16-byte piece cg at its 64-byte-swizzle place
-            sts128(sb + L.region_b + o * kOutTileBytes + (uint32_t)row * 64u + (uint32_t)((cg ^ ((row >> 1) & 3)) << 4), codes);
+            // output tile: rows of 128 bytes, 16-byte piece cg at its swizzled place
+            sts128(sb + L.region_b + o * kOutTileBytes + (uint32_t)row * 128u + (uint32_t)((cg ^ (row & 7)) << 4), codes);
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_out_full(o));
         }
 
-        // ---- T: partial sums from tensor memory to the CTA that owns the row ----
-        if (r > 0) {
-            if (ok) ok = qa_warp_wait(bar_acc, 0u, abort_flag, lane);
-            tc_fence_after();
-            // a warp reaches the 32 lanes of its quarter (warp % 4); the four warps of a quarter
-            // split the r columns
-            const int q = warp & 3, cpart = warp >> 2, ncol = r >> 2;
-            const int trow = q * 32 + lane;
-            uint32_t dst = 0;
-            if (CK > 1) {
-                // region B is free here once the stores have read the last output tiles, and
-                // at the peers once they say the same
-                if (ok) ok = qa_warp_wait(bar_tail, 0u, abort_flag, lane);
-                cluster_arrive();
-                cluster_wait();
-                const uint32_t owner = (uint32_t)(trow / rows_owned);
-                const int rl = trow - (int)owner * rows_owned;
-                dst = dsmem_addr(sb + L.region_b + (uint32_t)(((int)rank * rows_owned + rl) * r) * 4u, owner);
-            }
-            for (int c4 = 0; c4 < ncol; c4 += 4) {
-                const int col = cpart * ncol + c4;
-                uint32_t v[4];
-                tmem_ld4(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)col, v);
-                if (CK > 1) {
-                    dsmem_st_v4(dst + (uint32_t)col * 4u, v);
-                } else if (m0 + trow < M) {
-                    // a single CTA holds the whole sum
-                    const __nv_bfloat162 p0 = __floats2bfloat162_rn(__uint_as_float(v[0]), __uint_as_float(v[1]));
-                    const __nv_bfloat162 p1 = __floats2bfloat162_rn(__uint_as_float(v[2]), __uint_as_float(v[3]));
-                    uint2 pk;
-                    pk.x = *reinterpret_cast<const uint32_t*>(&p0);
-                    pk.y = *reinterpret_cast<const uint32_t*>(&p1);
-                    *reinterpret_cast<uint2*>(T + (size_t)(m0 + trow) * r + col) = pk;
+        // ---- T of the tokens this CTA owns: sum of the CK partials -> bf16 ----
+        if (CK > 1 && r > 0) {
+            const int pairs = r >> 1;
+            for (int e = tid; e < rows_owned * pairs; e += kTConsumers) {
+                const int tl = e / pairs, col = (e - tl * pairs) * 2;
+                const int t = (int)rank * rows_owned + tl;
+                float s0 = 0.f, s1 = 0.f;
+                for (int qq = 0; qq < CK; ++qq) {
+                    const float2 pv = *reinterpret_cast<const float2*>(t_slots + (qq * rows_owned + tl) * r + col);
+                    s0 += pv.x; s1 += pv.y;
                 }
-            }
-            tc_fence_before();
-            if (CK > 1) {
-                cluster_arrive();
-                cluster_wait();     // all partial sums have landed; only local reads from here
-                const int pairs = r >> 1;
-                for (int e = tid; e < rows_owned * pairs; e += kTConsumers) {
-                    const int rl = e / pairs, col = (e - rl * pairs) * 2;
-                    const int orow = (int)rank * rows_owned + rl;
-                    float s0 = 0.f, s1 = 0.f;
-                    for (int qq = 0; qq < CK; ++qq) {
-                        const float2 pv = *reinterpret_cast<const float2*>(t_slots + (qq * rows_owned + rl) * r + col);
-                        s0 += pv.x; s1 += pv.y;
-                    }
-                    if (m0 + orow < M)
-                        *reinterpret_cast<__nv_bfloat162*>(T + (size_t)(m0 + orow) * r + col) = __floats2bfloat162_rn(s0, s1);
-                }
+                if (m0 + t < M)
+                    *reinterpret_cast<__nv_bfloat162*>(T + (size_t)(m0 + t) * r + col) = __floats2bfloat162_rn(s0, s1);
             }
         }
         if (*abort_flag && cg == 0 && m0 + row < M) a_scale[m0 + row] = __int_as_float(0x7fc00000);   // a wait gave up: poison the rows
@@ -876,16 +873,21 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     __syncthreads();
     if (warp == kTWarpMma && r > 0) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
 }
 
 // Clusters of `ck` CTAs of this kernel that the device keeps resident at once (0 if it cannot
-// schedule that size).  Queried once per (size, shared memory) pair.
+// schedule that size).  Queried once per (size, shared memory) pair.  The query counts with
+// the kernel's opted-in maximum of dynamic shared memory, so that is set to the size asked for.
 int tma_active_clusters(int ck, size_t smem) {
     static int cached[17];
     static size_t cached_smem[17];
     if (cached_smem[ck] == smem && smem != 0) return cached[ck];
+    if (cudaFuncSetAttribute(quant_act_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return 0;
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(ck, 1, 1);
     cfg.blockDim = dim3(kTThreads, 1, 1);
@@ -907,16 +909,16 @@ int tma_active_clusters(int ck, size_t smem) {
     return n;
 }
 
-// Cluster size for the TMA kernel: a power of two (the CTAs split the 128 rows of T) that
-// divides the K / 64 column blocks.  Larger clusters shorten a CTA's two sweeps but fewer of
+// Cluster size for the TMA kernel: a power of two (the CTAs split the 64 tokens' T) that
+// divides the K / 128 stages.  Larger clusters shorten a CTA's two sweeps but fewer of
 // them are resident at once; the estimate is waves x (fixed cost + stages), in stage units.
 int pick_tma_cluster(int M, int K, int r, int max_ck) {
-    const int tiles = (M + kTTok - 1) / kTTok, blocks = K / kTCols;
+    const int tiles = (M + kTTok - 1) / kTTok, blocks = K / kTCols;      // 128-column stages
     int best = 0;
     long long best_cost = 0;
     for (int ck = 1; ck <= max_ck; ck *= 2) {
-        if (blocks % ck || blocks / ck < 2) continue;
-        const size_t smem = (size_t)tma_smem(K / ck, r).total;
+        if (blocks % ck) continue;
+        const size_t smem = (size_t)tma_smem(K / ck, r, ck).total;
         if (smem > 227 * 1024) continue;
         const int active = tma_active_clusters(ck, smem);
         if (active < 1) continue;
@@ -935,24 +937,28 @@ int launch_tma(const __half* X, const float* s, const __half* LA, int M, int K, 
         cudaError_t e = cudaFuncSetAttribute(quant_act_tma_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
         max_ck = (e == cudaSuccess) ? 16 : 8;
         if (e != cudaSuccess) (void)cudaGetLastError();
-        e = cudaFuncSetAttribute(quant_act_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e != cudaSuccess) return record_cuda_error(e, "quant_act_tma smem attribute");
     }
-    if ((M + kTTok - 1) / kTTok > 65535) { *unsupported = true; return ASER_OK; }
+    if ((M + kTTok - 1) / kTTok > 65535 || r > kTMaxRank) { *unsupported = true; return ASER_OK; }
     const int ck = pick_tma_cluster(M, K, r, max_ck);
     if (ck == 0) { *unsupported = true; return ASER_OK; }
     const int kc = K / ck;
-    const size_t smem = (size_t)tma_smem(kc, r).total;
+    const size_t smem = (size_t)tma_smem(kc, r, ck).total;
+    static size_t opted_in = 0;
+    if (smem != opted_in) {
+        cudaError_t e = cudaFuncSetAttribute(quant_act_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return record_cuda_error(e, "quant_act_tma smem attribute");
+        opted_in = smem;
+    }
     CUtensorMap mx, mla, mq;
-    int rc = encode_map_2d(&mx, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, X, M, K, kTTok, kTCols, CU_TENSOR_MAP_SWIZZLE_128B);
+    int rc = encode_map_2d(&mx, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, X, M, K, kTTok, kTAtom, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc != ASER_OK) return rc;
     if (r > 0) {
-        rc = encode_map_2d(&mla, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, LA, r, K, r, kTCols, CU_TENSOR_MAP_SWIZZLE_128B);
+        rc = encode_map_2d(&mla, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, LA, r, K, r, kTAtom, CU_TENSOR_MAP_SWIZZLE_128B);
         if (rc != ASER_OK) return rc;
     } else {
         mla = mx;
     }
-    rc = encode_map_2d(&mq, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Xq, M, K, kTTok, kTCols, CU_TENSOR_MAP_SWIZZLE_64B);
+    rc = encode_map_2d(&mq, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Xq, M, K, kTTok, kTCols, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc != ASER_OK) return rc;
 
     cudaLaunchConfig_t cfg = {};

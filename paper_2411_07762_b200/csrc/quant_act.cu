@@ -365,8 +365,8 @@ constexpr long long kQaWaitLimitClocks = 4000000000ll;   // about 2 s of SM cloc
 __host__ __device__ constexpr int tma_stages(int r) { return r <= 64 ? 4 : 3; }
 
 struct TmaSmem {
-    int x_ring, region_b, la_atom_bytes, la_stage_bytes, t_slots, ones, amax_cg, amax_slots, bars,
-        tmem_slot, abort_flag, total;
+    int x_ring, region_b, la_atom_bytes, la_stage_bytes, t_slots, t_stage, ones, amax_cg, amax_stage,
+        amax_slots, bars, tmem_slot, abort_flag, total;
 };
 // Offsets from the 1 KiB-aligned base.  Region B holds the L_A ring in sweep 1 and the output
 // tiles in sweep 2.  t_slots receives the partial T of the tokens this CTA owns from every CTA
@@ -391,10 +391,12 @@ __host__ __device__ inline TmaSmem tma_smem(int Kc, int r, int CK) {
         if (b < 16 * 1024) b = 16 * 1024;                      // readable space behind the L_A ring
         off += b;
     }
+    L.t_stage = off;    off += (CK > 1) ? kTTok * r * 4 : 0;   // this CTA's partial T, [token][r]
     L.ones = off;       off += (Kc / 16 + 15) / 16 * 16;       // per 16 columns: all divisors are 1
     L.amax_cg = off;    off += 8 * kTTok * 4;                  // row maxima per 16-column group
-    L.amax_slots = off; off += 16 * kTTok * 4;                 // row maxima stored by each CTA
-    L.bars = off;       off += (4 * kTMaxStages + 2 * kTOut + 1) * 8;
+    L.amax_stage = off; off += kTTok * 4;                      // row maxima of this CTA's slice
+    L.amax_slots = off; off += 16 * kTTok * 4;                 // row maxima copied in by each CTA
+    L.bars = off;       off += (4 * kTMaxStages + 2 * kTOut + 3) * 8;
     L.tmem_slot = off;  off += 8;
     L.abort_flag = off; off += 8;
     L.total = off + 1024;                                      // slack for the alignment
@@ -418,9 +420,14 @@ __device__ __forceinline__ uint32_t dsmem_addr(uint32_t local_addr, uint32_t ran
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
     return remote;
 }
-// Stores into a peer's shared memory; the cluster barrier publishes them.
-__device__ __forceinline__ void dsmem_st_f32(uint32_t remote, float v) {
-    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
+// Bulk copy from this CTA's shared memory into a peer's; the bytes are counted on the peer's
+// mbarrier, which is how the peer learns that they have landed.
+__device__ __forceinline__ void dsmem_bulk_copy(uint32_t remote_dst, uint32_t local_src, uint32_t bytes,
+                                                uint32_t remote_bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(remote_dst), "r"(local_src), "r"(bytes), "r"(remote_bar)
+        : "memory");
 }
 
 // Bounded wait on an mbarrier phase.  On expiry (or when another thread of the CTA has given
@@ -480,13 +487,18 @@ __device__ __forceinline__ void cvt8(const uint4& raw, float (&v)[8]) {
         v[2 * i] = f.x; v[2 * i + 1] = f.y;
     }
 }
-// x~ = fp32(x) / s for 8 columns (IEEE divisions)
+// x~ = fp32(x) / s for 8 columns (IEEE divisions).  A column's divisor is the same for every
+// lane of the warp (lanes are rows), so skipping the division where it is 1 does not diverge.
 __device__ __forceinline__ void div8(const uint4& raw, const float4& s0, const float4& s1, float (&v)[8]) {
     cvt8(raw, v);
-    v[0] = __fdiv_rn(v[0], s0.x); v[1] = __fdiv_rn(v[1], s0.y);
-    v[2] = __fdiv_rn(v[2], s0.z); v[3] = __fdiv_rn(v[3], s0.w);
-    v[4] = __fdiv_rn(v[4], s1.x); v[5] = __fdiv_rn(v[5], s1.y);
-    v[6] = __fdiv_rn(v[6], s1.z); v[7] = __fdiv_rn(v[7], s1.w);
+    if (s0.x != 1.f) v[0] = __fdiv_rn(v[0], s0.x);
+    if (s0.y != 1.f) v[1] = __fdiv_rn(v[1], s0.y);
+    if (s0.z != 1.f) v[2] = __fdiv_rn(v[2], s0.z);
+    if (s0.w != 1.f) v[3] = __fdiv_rn(v[3], s0.w);
+    if (s1.x != 1.f) v[4] = __fdiv_rn(v[4], s1.x);
+    if (s1.y != 1.f) v[5] = __fdiv_rn(v[5], s1.y);
+    if (s1.z != 1.f) v[6] = __fdiv_rn(v[6], s1.z);
+    if (s1.w != 1.f) v[7] = __fdiv_rn(v[7], s1.w);
 }
 __device__ __forceinline__ uint4 pack8_half(const float (&v)[8]) {
     uint4 pk;
@@ -517,7 +529,7 @@ __device__ __forceinline__ uint2 quant8_pairs(const float (&v)[8], float sc, flo
     const float2 r2 = make_float2(rcp, rcp), m2 = make_float2(kMagic, kMagic);
     const float2 nm2 = make_float2(-kMagic, -kMagic), neg1 = make_float2(-1.f, -1.f);
     uint32_t q[8];
-    bool tie = false;
+    float far = 0.f;        // largest distance of a product to its rounded integer (branch-free)
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const float2 t = __fmul2_rn(make_float2(v[2 * i], v[2 * i + 1]), r2);
@@ -526,9 +538,9 @@ __device__ __forceinline__ uint2 quant8_pairs(const float (&v)[8], float sc, flo
         const float2 d = __ffma2_rn(w, neg1, t);        // t - w, exact
         q[2 * i] = __float_as_uint(u.x);
         q[2 * i + 1] = __float_as_uint(u.y);
-        tie = tie || fabsf(d.x) > 0.4999f || fabsf(d.y) > 0.4999f;
+        far = fmaxf(far, fmaxf(fabsf(d.x), fabsf(d.y)));
     }
-    if (tie) return quant8_exact(v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7], sc);
+    if (far > 0.4999f) return quant8_exact(v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7], sc);
     const uint32_t a01 = __byte_perm(q[0], q[1], 0x0040), a23 = __byte_perm(q[2], q[3], 0x0040);
     const uint32_t a45 = __byte_perm(q[4], q[5], 0x0040), a67 = __byte_perm(q[6], q[7], 0x0040);
     return make_uint2(__byte_perm(a01, a23, 0x5410), __byte_perm(a45, a67, 0x5410));
@@ -560,8 +572,10 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L.tmem_slot);
     uint8_t* ones_sm = smem + L.ones;
     float* amax_cg = reinterpret_cast<float*>(smem + L.amax_cg);
+    float* amax_stage = reinterpret_cast<float*>(smem + L.amax_stage);
     float* amax_slots = reinterpret_cast<float*>(smem + L.amax_slots);
     float* t_slots = reinterpret_cast<float*>(smem + L.t_slots);
+    float* t_stage = reinterpret_cast<float*>(smem + L.t_stage);
     auto bar_full = [&](int st) { return sb + L.bars + st * 8; };
     auto bar_ready = [&](int st) { return sb + L.bars + (kTMaxStages + st) * 8; };
     auto bar_free1 = [&](int st) { return sb + L.bars + (2 * kTMaxStages + st) * 8; };
@@ -569,6 +583,8 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     auto bar_out_full = [&](int o) { return sb + L.bars + (4 * kTMaxStages + o) * 8; };
     auto bar_out_free = [&](int o) { return sb + L.bars + (4 * kTMaxStages + kTOut + o) * 8; };
     const uint32_t bar_acc = sb + L.bars + (4 * kTMaxStages + 2 * kTOut) * 8;
+    const uint32_t bar_amax = bar_acc + 8;      // the peers' row maxima have landed
+    const uint32_t bar_t = bar_acc + 16;        // the peers' partial T have landed
     constexpr uint32_t kTmemCols = 64;                      // D[j, token]: 64 token columns
 
     // Use i of the ring: i < nst is sweep 1 (X and L_A tiles), the rest sweep 2 (X only).
@@ -621,9 +637,15 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 mbar_init(bar_out_free(o), 1);                  // its store has read it
             }
             mbar_init(bar_acc, 1);
+            mbar_init(bar_amax, 1);
+            mbar_init(bar_t, 1);
             *abort_flag = 0;
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
             fence_proxy_async_smem();
+            if (CK > 1) {       // bytes the cluster's CTAs will copy in
+                mbar_arrive_expect_tx(bar_amax, (uint32_t)(CK * kTTok * 4));
+                if (r > 0) mbar_arrive_expect_tx(bar_t, (uint32_t)(kTTok * r * 4));
+            }
             for (int i = 0; i < NS && i < 2 * nst; ++i) load_use(i);      // no waits yet
         }
         __syncwarp();
@@ -653,24 +675,22 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    // "my barriers are ready for your copies": waited for before the first copy into a peer
+    if (CK > 1) cluster_arrive();
     const uint32_t tmem = (r > 0) ? *tmem_slot : 0u;
 
     if (warp == kTWarpProd) {
         // ================= TMA producer =================
-        // Uses whose stage is released by sweep 1 come before the exchange; the rest wait for
-        // the consumers' sweep 2, which starts after the cluster barrier this warp takes part in.
         const int early = (2 * nst < nst + NS) ? 2 * nst : nst + NS;
         bool ok = true;
         if (lane == 0) {
             for (int i = NS; i < early && ok; ++i) ok = load_use(i);
         }
-        __syncwarp();
-        cluster_arrive();
-        cluster_wait();
         if (lane == 0) {
             for (int i = (early > NS ? early : NS); i < 2 * nst && ok; ++i) ok = load_use(i);
         }
         __syncwarp();
+        if (CK > 1) cluster_wait();
     } else if (warp == kTWarpMma) {
         // ================= MMA issuer, then store issuer =================
         bool ok = true;
@@ -699,8 +719,7 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             if (r > 0) tc_commit(bar_acc);      // arrives when every MMA above has completed
         }
         __syncwarp();
-        cluster_arrive();
-        cluster_wait();
+        if (CK > 1) cluster_wait();
         if (lane == 0) {
             // Sweep 2: one TMA store per output tile.  A tile goes back to the consumers once
             // the store has read it; the stores run two behind.
@@ -762,16 +781,25 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         }
         amax = fmaxf(amax, fmaxf(__low2float(hamax), __high2float(hamax)));
         amax_cg[cg * kTTok + row] = amax;
+        if (CK > 1) cluster_wait();     // every CTA of the cluster has its barriers set up
         named_bar_sync(1, kTConsumers);
-        // ---- row maxima: stored into every CTA of the cluster (each needs all row scales) ----
+        // ---- row maxima of this slice; copied into every CTA of the cluster (each needs all
+        // row scales) ----
         if (tid < kTTok) {
             float a = amax_cg[tid];
 #pragma unroll
             for (int g = 1; g < 8; ++g) a = fmaxf(a, amax_cg[g * kTTok + tid]);
-            const uint32_t slot = sb + L.amax_slots + (rank * kTTok + tid) * 4;
-            for (int qq = 0; qq < CK; ++qq) dsmem_st_f32(dsmem_addr(slot, (uint32_t)qq), a);
+            amax_stage[tid] = a;
+            fence_proxy_async_smem();
         }
-        // ---- partial T: tensor memory -> the CTA that owns the token ----
+        if (CK > 1) {
+            if (warp < 2) named_bar_sync(2, 64);        // the 64 values are written (warps 0 and 1)
+            if (tid == 0)
+                for (int qq = 0; qq < CK; ++qq)
+                    dsmem_bulk_copy(dsmem_addr(sb + L.amax_slots + rank * (kTTok * 4), (uint32_t)qq),
+                                    sb + L.amax_stage, kTTok * 4, dsmem_addr(bar_amax, (uint32_t)qq));
+        }
+        // ---- partial T: tensor memory -> shared memory -> the CTAs that own the tokens ----
         if (r > 0) {
             if (ok) ok = qa_warp_wait(bar_acc, 0u, abort_flag, lane);
             tc_fence_after();
@@ -787,28 +815,34 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
 #pragma unroll
                     for (int e = 0; e < 16; ++e) {
                         const int t = t0 + e;
-                        if (CK > 1) {
-                            const uint32_t owner = (uint32_t)(t / rows_owned);
-                            const int tl = t - (int)owner * rows_owned;
-                            const uint32_t dst = sb + L.t_slots + (uint32_t)((((int)rank * rows_owned + tl) * r + j) * 4);
-                            dsmem_st_f32(dsmem_addr(dst, owner), __uint_as_float(v[e]));
-                        } else if (m0 + t < M) {
-                            T[(size_t)(m0 + t) * r + j] = __float2bfloat16_rn(__uint_as_float(v[e]));
-                        }
+                        if (CK > 1) t_stage[t * r + j] = __uint_as_float(v[e]);
+                        else if (m0 + t < M) T[(size_t)(m0 + t) * r + j] = __float2bfloat16_rn(__uint_as_float(v[e]));
                     }
                 }
             }
             tc_fence_before();
+            if (CK > 1) {
+                fence_proxy_async_smem();
+                named_bar_sync(1, kTConsumers);
+                if (tid == 0) {
+                    const uint32_t bytes = (uint32_t)(rows_owned * r * 4);
+                    for (int qq = 0; qq < CK; ++qq)
+                        dsmem_bulk_copy(dsmem_addr(sb + L.t_slots + rank * bytes, (uint32_t)qq),
+                                        sb + L.t_stage + (uint32_t)qq * bytes, bytes, dsmem_addr(bar_t, (uint32_t)qq));
+                }
+            }
         }
-        cluster_arrive();
-        cluster_wait();         // row maxima and partial T have landed; only local accesses from here
 
         // ---- row scale of this thread's row; the owner of a row writes it out ----
         float sc;
-        {
+        if (CK > 1) {
+            if (ok) ok = qa_warp_wait(bar_amax, 0u, abort_flag, lane);     // all row maxima have landed
             float a = 0.f;
             for (int qq = 0; qq < CK; ++qq) a = fmaxf(a, amax_slots[qq * kTTok + row]);
             sc = __fdiv_rn(a, 127.0f);
+        } else {
+            named_bar_sync(1, kTConsumers);
+            sc = __fdiv_rn(amax_stage[row], 127.0f);
         }
         if (cg == 0 && (int)rank == row / rows_owned && m0 + row < M) a_scale[m0 + row] = sc;
 
@@ -854,6 +888,7 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
 
         // ---- T of the tokens this CTA owns: sum of the CK partials -> bf16 ----
         if (CK > 1 && r > 0) {
+            if (ok) ok = qa_warp_wait(bar_t, 0u, abort_flag, lane);        // all partials have landed
             const int pairs = r >> 1;
             for (int e = tid; e < rows_owned * pairs; e += kTConsumers) {
                 const int tl = e / pairs, col = (e - tl * pairs) * 2;
@@ -868,6 +903,11 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             }
         }
         if (*abort_flag && cg == 0 && m0 + row < M) a_scale[m0 + row] = __int_as_float(0x7fc00000);   // a wait gave up: poison the rows
+    }
+    // Nobody leaves while a peer may still copy from or into this CTA's shared memory.
+    if (CK > 1) {
+        cluster_arrive();
+        cluster_wait();
     }
     tc_fence_before();
     __syncthreads();

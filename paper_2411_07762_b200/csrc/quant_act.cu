@@ -548,8 +548,8 @@ __device__ __forceinline__ uint2 quant8_pairs(const float (&v)[8], float sc, flo
 
 // grid = (CK, ceil(M / 64)), cluster = (CK, 1, 1) with CK a power of two <= 16, kTThreads threads,
 // r <= 128.
-// map_x: X as fp16 [M, K], box 64 rows x 64 columns, 128-byte swizzle.
-// map_la: L_A as fp16 [r, K], box r rows x 64 columns, 128-byte swizzle (unused when r == 0).
+// map_x: X as fp16 [K / 64 blocks][M][64], box 2 blocks x 64 rows, 128-byte swizzle.
+// map_la: L_A as fp16 [K / 64 blocks][r][64], box 2 blocks x r rows (unused when r == 0).
 // map_q: Xq as bytes [M, K], box 64 rows x 128 columns, 128-byte swizzle.
 __global__ void __launch_bounds__(kTThreads, 1)
 quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_la,
@@ -606,18 +606,12 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         if (i < nst) {
             const int kcol = k0 + i * kTCols;
             mbar_arrive_expect_tx(bar_full(st), (uint32_t)(kXStageBytes + L.la_stage_bytes));
-            tma_load_2d(xdst, &map_x, kcol, m0, bar_full(st));
-            tma_load_2d(xdst + kXAtomBytes, &map_x, kcol + kTAtom, m0, bar_full(st));
-            if (r > 0) {
-                const uint32_t ldst = sb + L.region_b + st * L.la_stage_bytes;
-                tma_load_2d(ldst, &map_la, kcol, 0, bar_full(st));
-                tma_load_2d(ldst + L.la_atom_bytes, &map_la, kcol + kTAtom, 0, bar_full(st));
-            }
+            tma_load_3d(xdst, &map_x, 0, m0, kcol / kTAtom, bar_full(st));
+            if (r > 0) tma_load_3d(sb + L.region_b + st * L.la_stage_bytes, &map_la, 0, 0, kcol / kTAtom, bar_full(st));
         } else {
             const int kcol = k0 + (i - nst) * kTCols;
             mbar_arrive_expect_tx(bar_full(st), (uint32_t)kXStageBytes);
-            tma_load_2d(xdst, &map_x, kcol, m0, bar_full(st));
-            tma_load_2d(xdst + kXAtomBytes, &map_x, kcol + kTAtom, m0, bar_full(st));
+            tma_load_3d(xdst, &map_x, 0, m0, kcol / kTAtom, bar_full(st));
         }
         return true;
     };
@@ -794,10 +788,9 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         }
         if (CK > 1) {
             if (warp < 2) named_bar_sync(2, 64);        // the 64 values are written (warps 0 and 1)
-            if (tid == 0)
-                for (int qq = 0; qq < CK; ++qq)
-                    dsmem_bulk_copy(dsmem_addr(sb + L.amax_slots + rank * (kTTok * 4), (uint32_t)qq),
-                                    sb + L.amax_stage, kTTok * 4, dsmem_addr(bar_amax, (uint32_t)qq));
+            if (tid < CK)       // one lane per destination
+                dsmem_bulk_copy(dsmem_addr(sb + L.amax_slots + rank * (kTTok * 4), (uint32_t)tid),
+                                sb + L.amax_stage, kTTok * 4, dsmem_addr(bar_amax, (uint32_t)tid));
         }
         // ---- partial T: tensor memory -> shared memory -> the CTAs that own the tokens ----
         if (r > 0) {
@@ -824,11 +817,10 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             if (CK > 1) {
                 fence_proxy_async_smem();
                 named_bar_sync(1, kTConsumers);
-                if (tid == 0) {
+                if (tid < CK) {
                     const uint32_t bytes = (uint32_t)(rows_owned * r * 4);
-                    for (int qq = 0; qq < CK; ++qq)
-                        dsmem_bulk_copy(dsmem_addr(sb + L.t_slots + rank * bytes, (uint32_t)qq),
-                                        sb + L.t_stage + (uint32_t)qq * bytes, bytes, dsmem_addr(bar_t, (uint32_t)qq));
+                    dsmem_bulk_copy(dsmem_addr(sb + L.t_slots + rank * bytes, (uint32_t)tid),
+                                    sb + L.t_stage + (uint32_t)tid * bytes, bytes, dsmem_addr(bar_t, (uint32_t)tid));
                 }
             }
         }
@@ -990,10 +982,10 @@ int launch_tma(const __half* X, const float* s, const __half* LA, int M, int K, 
         opted_in = smem;
     }
     CUtensorMap mx, mla, mq;
-    int rc = encode_map_2d(&mx, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, X, M, K, kTTok, kTAtom, CU_TENSOR_MAP_SWIZZLE_128B);
+    int rc = encode_map_blocks(&mx, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, X, M, K, kTTok, 2);
     if (rc != ASER_OK) return rc;
     if (r > 0) {
-        rc = encode_map_2d(&mla, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, LA, r, K, r, kTAtom, CU_TENSOR_MAP_SWIZZLE_128B);
+        rc = encode_map_blocks(&mla, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, LA, r, K, r, 2);
         if (rc != ASER_OK) return rc;
     } else {
         mla = mx;

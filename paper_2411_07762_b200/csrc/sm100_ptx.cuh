@@ -204,4 +204,24 @@ inline int encode_map_2d(CUtensorMap* map, CUtensorMapDataType dt, int esize, co
     return ASER_OK;
 }
 
+// Row-major tensor [rows, cols] of `esize`-byte elements viewed as 128-byte column blocks:
+// [cols * esize / 128 blocks][rows][128 bytes].  A box takes `box_blocks` blocks x `box_rows` rows,
+// 128-byte swizzle; in shared memory each block's rows are contiguous (the K-major operand layout
+// of the MMA descriptors).  Coordinates: (0, row, block).
+inline int encode_map_blocks(CUtensorMap* map, CUtensorMapDataType dt, int esize, const void* base,
+                             uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t box_blocks) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return record_cuda_error(cudaErrorUnknown, "cuTensorMapEncodeTiled unavailable");
+    const uint64_t per_block = 128 / (uint64_t)esize;
+    cuuint64_t dims[3] = {per_block, rows, cols / per_block};
+    cuuint64_t strides[2] = {cols * (uint64_t)esize, 128};
+    cuuint32_t box[3] = {(cuuint32_t)per_block, box_rows, box_blocks};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(map, dt, 3, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return record_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled (blocks)");
+    return ASER_OK;
+}
+
 }  // namespace aser

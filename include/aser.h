@@ -152,9 +152,28 @@ int aser_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
 int aser_check_status(void* workspace, void* stream);
 
 /*
+ * aser_forward -- one whole forward pass of the layer (Sec. 4.2, Eq. 9 with the low-rank term
+ * of Sec. 4.1) from DEVICE buffers: aser_quant_act followed by aser_linear_w4a8_lr (the plain
+ * kernel when r == 0), enqueued on `stream`, no synchronisation.
+ * Because the library knows that the quantization kernel is what precedes the linear kernel,
+ * it launches the latter as a programmatic dependent: the linear kernel starts while the
+ * quantization still runs, streams the weights (which that kernel does not write) and waits
+ * for its completion before it reads Xq, a_scale or T.  Results are bit-identical to the two
+ * separate calls.
+ * X_f16 [M,K], s [K] or NULL, LA_f16 [r,K] / LB_f16 [N,r] (NULL when r == 0), Wk and w_scale as
+ * for aser_linear_w4a8_lr.  Xq [M,K], a_scale [M], T_bf16 [M,r] (NULL when r == 0) are the
+ * caller's intermediates (written), Y_f16 [M,N] the result.  Wk, w_scale and LB_f16 must not
+ * be written by work still in flight on `stream` when the call is made.
+ * Errors: as the two calls; nothing is enqueued when an argument is rejected.
+ */
+int aser_forward(const void* X_f16, const float* s, const void* LA_f16, const void* Wk,
+                 const float* w_scale, const void* LB_f16, int M, int N, int K, int r,
+                 int8_t* Xq, float* a_scale, void* T_bf16, void* Y_f16,
+                 void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * aser_forward_host -- one whole forward pass from HOST buffers: copies X (fp16 [M,K],
- * ideally pinned) to the device staging buffer X_dev, runs aser_quant_act and
- * aser_linear_w4a8_lr (the plain kernel when r == 0), and copies Y back to Y_host,
+ * ideally pinned) to the device staging buffer X_dev, runs aser_forward, and copies Y back to Y_host,
  * all enqueued on `stream`; returns without synchronising.  Device-side operands and
  * staging buffers are the caller's.
  */

@@ -12,7 +12,8 @@ lib_path = os.path.join(_HERE, "libaser.so")
 EXPORTED_SYMBOLS = (
     "aser_pack_w4", "aser_repacked_bytes", "aser_repack_w4", "aser_unrepack_w4",
     "aser_quant_act", "aser_linear_w4a8_lr", "aser_linear_w4a8", "aser_linear_w4a8_lr_simt", "aser_linear_w4a8_lr_static",
-    "aser_workspace_bytes", "aser_workspace_init", "aser_check_status", "aser_forward_host",
+    "aser_workspace_bytes", "aser_workspace_init", "aser_check_status", "aser_forward",
+    "aser_forward_host",
     "aser_last_error", "aser_version",
 )
 
@@ -37,6 +38,7 @@ lib.aser_workspace_bytes.argtypes = [_I, _I, _I, _I]
 lib.aser_workspace_bytes.restype = _Z
 lib.aser_workspace_init.argtypes = [_P, _Z, _P]
 lib.aser_check_status.argtypes = [_P, _P]
+lib.aser_forward.argtypes = [_P, _P, _P, _P, _P, _P, _I, _I, _I, _I, _P, _P, _P, _P, _P, _Z, _P]
 lib.aser_forward_host.argtypes = [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P,
                                   _I, _I, _I, _I, _P, _Z, _P]
 lib.aser_last_error.restype = C.c_char_p
@@ -229,10 +231,18 @@ class AserLinear:
                  "aser_linear_w4a8")
 
     def __call__(self, X: torch.Tensor, lowrank: bool = True) -> torch.Tensor:
+        """One forward pass through aser_forward (quantization and linear kernel overlapped)."""
         M = X.shape[0]
         assert M <= self.max_tokens
-        self.quant(X)
-        self.linear(M, lowrank)
+        if not lowrank and self.r:
+            self.quant(X)
+            self.linear(M, False)
+            return self.Y[:M]
+        r = self.r
+        _chk(lib.aser_forward(_ptr(X), _ptr(self.s), _ptr(self.L_A) if r else None, _ptr(self.Wk),
+                              _ptr(self.w_scale), _ptr(self.L_B) if r else None, M, self.N, self.K, r,
+                              _ptr(self.Xq), _ptr(self.a_scale), _ptr(self.T) if r else None,
+                              _ptr(self.Y), _ptr(self.ws), self.ws.numel(), _stream()), "aser_forward")
         return self.Y[:M]
 
     def forward_host(self, X_host: torch.Tensor, Y_host: torch.Tensor):

@@ -68,7 +68,8 @@ int check_device() {
 
 int linear_common(const int8_t* Xq, const float* a_scale, const void* Wk, const float* w_scale,
                   const void* T_bf16, const void* LB_f16, int M, int N, int K, int r, void* Y_f16,
-                  int32_t* acc_debug, void* workspace, size_t workspace_bytes, void* stream) {
+                  int32_t* acc_debug, void* workspace, size_t workspace_bytes, void* stream,
+                  bool overlap_prev = false) {
     if (!shape_ok(M, N, K, r)) return fail(ASER_ERR_SHAPE, "unsupported M, N, K or r");
     if (M == 0 || N == 0) return ASER_OK;
     ASER_REQUIRE_PTR(Xq);
@@ -90,7 +91,7 @@ int linear_common(const int8_t* Xq, const float* a_scale, const void* Wk, const 
                             static_cast<const __nv_bfloat16*>(T_bf16),
                             static_cast<const __half*>(LB_f16), M, N, K, r,
                             static_cast<__half*>(Y_f16), acc_debug, workspace, workspace_bytes,
-                            static_cast<cudaStream_t>(stream));
+                            static_cast<cudaStream_t>(stream), overlap_prev);
 }
 
 }  // namespace
@@ -232,6 +233,27 @@ int aser_check_status(void* workspace, void* stream) {
     return ASER_ERR_DEVICE_TIMEOUT;
 }
 
+int aser_forward(const void* X_f16, const float* s, const void* LA_f16, const void* Wk,
+                 const float* w_scale, const void* LB_f16, int M, int N, int K, int r,
+                 int8_t* Xq, float* a_scale, void* T_bf16, void* Y_f16, void* workspace,
+                 size_t workspace_bytes, void* stream) {
+    if (!shape_ok(M, N, K, r)) return fail(ASER_ERR_SHAPE, "unsupported M, N, K or r");
+    if (M == 0 || N == 0) return ASER_OK;
+    // validate the second launch's arguments before the first is enqueued
+    ASER_REQUIRE_PTR(Wk);
+    ASER_REQUIRE_PTR(w_scale);
+    ASER_REQUIRE_PTR(Y_f16);
+    if (r > 0) ASER_REQUIRE_PTR(LB_f16);
+    if (workspace == nullptr || misaligned16(workspace) ||
+        workspace_bytes < aser_workspace_bytes(M, N, K, r))
+        return fail(ASER_ERR_WORKSPACE, "workspace missing, misaligned or too small");
+    int rc = aser_quant_act(X_f16, s, LA_f16, M, K, r, Xq, a_scale, T_bf16, stream);
+    if (rc != ASER_OK) return rc;
+    return linear_common(Xq, a_scale, Wk, w_scale, r > 0 ? T_bf16 : nullptr, r > 0 ? LB_f16 : nullptr,
+                         M, N, K, r, Y_f16, nullptr, workspace, workspace_bytes, stream,
+                         /*overlap_prev=*/true);
+}
+
 int aser_forward_host(const void* X_host_f16, void* Y_host_f16, void* X_dev, int8_t* Xq_dev,
                       float* a_scale_dev, void* T_dev, void* Y_dev, const float* s,
                       const void* LA_f16, const void* Wk, const float* w_scale, const void* LB_f16,
@@ -246,11 +268,8 @@ int aser_forward_host(const void* X_host_f16, void* Y_host_f16, void* X_dev, int
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = cudaMemcpyAsync(X_dev, X_host_f16, (size_t)M * K * 2, cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return record_cuda_error(e, "copy X to device");
-    int rc = aser_quant_act(X_dev, s, LA_f16, M, K, r, Xq_dev, a_scale_dev, T_dev, stream);
-    if (rc != ASER_OK) return rc;
-    rc = linear_common(Xq_dev, a_scale_dev, Wk, w_scale, r > 0 ? T_dev : nullptr,
-                       r > 0 ? LB_f16 : nullptr, M, N, K, r, Y_dev, nullptr, workspace,
-                       workspace_bytes, stream);
+    int rc = aser_forward(X_dev, s, LA_f16, Wk, w_scale, LB_f16, M, N, K, r, Xq_dev, a_scale_dev,
+                          T_dev, Y_dev, workspace, workspace_bytes, stream);
     if (rc != ASER_OK) return rc;
     e = cudaMemcpyAsync(Y_host_f16, Y_dev, (size_t)M * N * 2, cudaMemcpyDeviceToHost, st);
     if (e != cudaSuccess) return record_cuda_error(e, "copy Y to host");

@@ -29,10 +29,15 @@ int launch_quant_act(const __half* X, const float* s, const __half* LA, int M, i
 int launch_linear_simt(const int8_t* Xq, const float* a_scale, const uint8_t* Wq,
                        const float* w_scale, const __nv_bfloat16* T, const __half* LB,
                        int M, int N, int K, int r, __half* Y, int32_t* acc_debug, cudaStream_t st);
+// `overlap_prev`: the kernel launched before this one on `st` is this library's quant_act for
+// the same step.  The linear kernel may then start while that one still runs: it streams the
+// weights (which that kernel does not write) and waits for its completion before it touches
+// Xq, a_scale or T.  Must be false when anything else precedes the launch.
 int launch_linear_tc(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
                      const float* w_scale, const __nv_bfloat16* T, const __half* LB,
                      int M, int N, int K, int r, __half* Y, int32_t* acc_debug,
-                     void* workspace, size_t workspace_bytes, cudaStream_t st);
+                     void* workspace, size_t workspace_bytes, cudaStream_t st,
+                     bool overlap_prev = false);
 size_t linear_tc_workspace_bytes(int M, int N, int K, int r);
 // Leading bytes of the workspace (status word + tile counters) that must be zero at launch.
 size_t linear_tc_zeroed_prefix_bytes(int M, int N, int K, int r);

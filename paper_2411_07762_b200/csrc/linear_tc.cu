@@ -317,6 +317,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     } else if (warp == C::WarpXProd) {
         // =================== activation + low-rank operand producer (one lane) ===================
         if (lane == 0) {
+            grid_dep_wait();        // Xq and T come from the kernel launched before this one
             Cursor cur;
             cur.init(u_begin, u_end, p);
             Work w{};
@@ -543,6 +544,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         // both integer accumulators start at zero: every integer MMA accumulates
         for (int c0 = 16 * half; c0 < 2 * BT; c0 += kChunkStep) tmem_zero16(tm_dint0 + lane_sel + c0);
         tmem_wait_st();
+        grid_dep_wait();            // a_scale comes from the kernel launched before this one
         tc_fence_before();
         __syncwarp();
         if (lane == 0) { mbar_arrive(bar(B_ACC_EMPTY + 0)); mbar_arrive(bar(B_ACC_EMPTY + 1)); }
@@ -766,7 +768,7 @@ Layout make_layout(int M, int N, int K, int r) {
 
 template <int BT>
 int launch_bt(const CUtensorMap& mx, const CUtensorMap& mlb, const CUtensorMap& mt, const Params& p,
-              int grid, cudaStream_t st) {
+              int grid, cudaStream_t st, bool overlap_prev) {
     using C = Cfg<BT>;
     static bool configured = false;
     if (!configured) {
@@ -775,7 +777,18 @@ int launch_bt(const CUtensorMap& mx, const CUtensorMap& mlb, const CUtensorMap& 
         if (e != cudaSuccess) return record_cuda_error(e, "linear_tc smem attribute");
         configured = true;
     }
-    linear_tc_kernel<BT><<<grid, C::Threads, C::SmemBytes, st>>>(mx, mlb, mt, p);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(C::Threads, 1, 1);
+    cfg.dynamicSmemBytes = C::SmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap_prev ? 1 : 0;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, linear_tc_kernel<BT>, mx, mlb, mt, p);
+    if (e != cudaSuccess) return record_cuda_error(e, "linear_tc_kernel");
     return check_launch("linear_tc_kernel");
 }
 
@@ -794,7 +807,7 @@ size_t linear_tc_zeroed_prefix_bytes(int M, int N, int K, int r) {
 int launch_linear_tc(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
                      const float* w_scale, const __nv_bfloat16* T, const __half* LB,
                      int M, int N, int K, int r, __half* Y, int32_t* acc_debug,
-                     void* workspace, size_t workspace_bytes, cudaStream_t st) {
+                     void* workspace, size_t workspace_bytes, cudaStream_t st, bool overlap_prev) {
     Layout L = make_layout(M, N, K, r);
     if (workspace_bytes < L.total) return ASER_ERR_WORKSPACE;
     if (L.units >= (1ll << 31) / kMaxCtas * kMaxCtas) return ASER_ERR_SHAPE;
@@ -837,10 +850,10 @@ int launch_linear_tc(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
     p.KB = L.KB; p.TT = L.TT; p.NT = L.NT; p.units = (int)L.units;
 
     switch (L.BT) {
-        case 16: return launch_bt<16>(mx, mlb, mt, p, grid, st);
-        case 32: return launch_bt<32>(mx, mlb, mt, p, grid, st);
-        case 64: return launch_bt<64>(mx, mlb, mt, p, grid, st);
-        default: return launch_bt<128>(mx, mlb, mt, p, grid, st);
+        case 16: return launch_bt<16>(mx, mlb, mt, p, grid, st, overlap_prev);
+        case 32: return launch_bt<32>(mx, mlb, mt, p, grid, st, overlap_prev);
+        case 64: return launch_bt<64>(mx, mlb, mt, p, grid, st, overlap_prev);
+        default: return launch_bt<128>(mx, mlb, mt, p, grid, st, overlap_prev);
     }
 }
 

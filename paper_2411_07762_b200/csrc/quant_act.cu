@@ -89,6 +89,7 @@ quant_act_small_kernel(const __half* __restrict__ X, const float* __restrict__ s
                        int8_t* __restrict__ Xq, float* __restrict__ a_scale,
                        __nv_bfloat16* __restrict__ T) {
     extern __shared__ __align__(16) float xs[];
+    grid_dep_launch();      // a dependent linear kernel may start streaming its weights
     __shared__ float red[kRowsPerCta][kSmallThreads / 32];
     const int m = blockIdx.y;
     const int chunks = K / 8;
@@ -205,6 +206,7 @@ quant_act_large_kernel(const __half* __restrict__ X, const float* __restrict__ s
                        int8_t* __restrict__ Xq, float* __restrict__ a_scale,
                        __nv_bfloat16* __restrict__ T) {
     extern __shared__ __align__(16) uint8_t smem[];
+    grid_dep_launch();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int m0 = blockIdx.x * kTileM;
     const int trow = tid >> 4;  // token row of this thread (0..15)
@@ -557,6 +559,7 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                      int M, int K, int Kc, int r, int CK, float* __restrict__ a_scale,
                      __nv_bfloat16* __restrict__ T) {
     extern __shared__ uint8_t smem_raw[];
+    grid_dep_launch();      // a dependent linear kernel may start streaming its weights
     const uint32_t sraw = smem_u32(smem_raw);
     const uint32_t sb = (sraw + 1023u) & ~1023u;            // swizzled tiles need 1 KiB alignment
     uint8_t* smem = smem_raw + (sb - sraw);

@@ -179,3 +179,38 @@ def test_config3_prefill_full_size_sampled_rows(aser, impl, which):
     s, Wq, w_scale, L_A, L_B = oracle_layer(lay, r, construct=False)
     rows = np.array([0, 1, 127, 128, 1000, 1023, 1024, 2046, 2047])
     run_path(aser, lay, s, Wq, w_scale, L_A, L_B, impl, rows=rows, use_dgemm=True)
+
+
+FORWARD_CASES = [  # M, N, K, r
+    (8, 512, 4096, 64), (1, 256, 512, 16), (33, 264, 512, 0), (130, 384, 1024, 64),
+    (300, 1152, 2048, 128), (2048, 512, 4096, 64),
+]
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("M,N,K,r", FORWARD_CASES)
+def test_forward_overlapped_is_bit_identical_to_separate_calls(aser, M, N, K, r):
+    """aser_forward launches the linear kernel as a programmatic dependent of the quantization
+    kernel; every output must equal that of the two plain calls, on repeated back-to-back runs
+    with alternating inputs (a missing wait would show as stale Xq, a_scale or T)."""
+    lay = synth.make_layer(M, N, K, seed=900 + M + N + K + r, n_cal=8, n_out=max(1, K // 100))
+    s = synth.standin_smoothing_vector(K, lay.outlier_idx, 9.0)
+    L_A, L_B = synth.standin_factors(N, K, r, seed=M + r, scale_a=0.02, scale_b=0.02) if r else (None, None)
+    layer = aser.AserLinear(to_dev(lay.W), to_dev(s), None if r == 0 else to_dev(L_A),
+                            None if r == 0 else to_dev(L_B), M)
+    X0 = to_dev(lay.X)
+    X1 = torch.roll(X0, shifts=3, dims=1).contiguous() * 0.5
+    want = []
+    for X in (X0, X1):
+        layer.quant(X)
+        layer.linear(M)
+        want.append((layer.Y[:M].clone(), layer.Xq[:M].clone(), layer.a_scale[:M].clone(),
+                     layer.T[:M].clone()))
+    aser.check_status(layer.ws)
+    for it in range(12):
+        X = (X0, X1)[it & 1]
+        Y = layer(X)
+        got = (Y, layer.Xq[:M], layer.a_scale[:M], layer.T[:M])
+        for g, w in zip(got, want[it & 1]):
+            assert torch.equal(g.view(torch.uint8), w.view(torch.uint8)), it
+    aser.check_status(layer.ws)

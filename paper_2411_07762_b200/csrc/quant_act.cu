@@ -82,7 +82,7 @@ constexpr int kRowsPerCta = 4;  // L_A rows handled by one projection CTA
 
 // grid = (1 + ceil(r / kRowsPerCta), M).  blockIdx.x == 0 quantizes token blockIdx.y,
 // the others compute kRowsPerCta entries of T for that token.
-// dynamic smem: K floats (the smoothed row).
+// dynamic smem: K floats (the smoothed row; used by the quantizing CTA).
 __global__ void __launch_bounds__(kSmallThreads)
 quant_act_small_kernel(const __half* __restrict__ X, const float* __restrict__ s,
                        const __half* __restrict__ LA, int M, int K, int r,
@@ -95,19 +95,18 @@ quant_act_small_kernel(const __half* __restrict__ X, const float* __restrict__ s
     const int chunks = K / 8;
     const __half* row = X + (size_t)m * K;
 
-    float amax = 0.f;
-    for (int c = threadIdx.x; c < chunks; c += kSmallThreads) {
-        RawChunk rc = load_raw(row, s, c * 8, true);
-        float v[8];
-        smooth8(rc, v);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(v[i]));
-        *reinterpret_cast<float4*>(xs + c * 8) = make_float4(v[0], v[1], v[2], v[3]);
-        *reinterpret_cast<float4*>(xs + c * 8 + 4) = make_float4(v[4], v[5], v[6], v[7]);
-    }
-
     if (blockIdx.x == 0) {
-        // ---- quantize this token ----
+        // ---- quantize this token: x~ to shared memory with the row maximum, then the codes ----
+        float amax = 0.f;
+        for (int c = threadIdx.x; c < chunks; c += kSmallThreads) {
+            RawChunk rc = load_raw(row, s, c * 8, true);
+            float v[8];
+            smooth8(rc, v);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(v[i]));
+            *reinterpret_cast<float4*>(xs + c * 8) = make_float4(v[0], v[1], v[2], v[3]);
+            *reinterpret_cast<float4*>(xs + c * 8 + 4) = make_float4(v[4], v[5], v[6], v[7]);
+        }
         amax = warp_max(amax);
         if ((threadIdx.x & 31) == 0) red[0][threadIdx.x >> 5] = amax;
         __syncthreads();
@@ -126,29 +125,34 @@ quant_act_small_kernel(const __half* __restrict__ X, const float* __restrict__ s
         return;
     }
 
-    // ---- down projection: kRowsPerCta rows of L_A against the smoothed token ----
-    __syncthreads();
+    // ---- down projection: kRowsPerCta rows of L_A against the smoothed token.  A thread
+    // smooths the chunks it multiplies, so all of its loads (activations, divisors, L_A rows)
+    // are in flight together and no barrier separates them. ----
     const int j0 = (blockIdx.x - 1) * kRowsPerCta;
     float acc[kRowsPerCta];
 #pragma unroll
     for (int jj = 0; jj < kRowsPerCta; ++jj) acc[jj] = 0.f;
+#pragma unroll 2
     for (int c = threadIdx.x; c < chunks; c += kSmallThreads) {
-        float4 x0 = *reinterpret_cast<const float4*>(xs + c * 8);
-        float4 x1 = *reinterpret_cast<const float4*>(xs + c * 8 + 4);
+        const RawChunk rc = load_raw(row, s, c * 8, true);
+        uint4 la[kRowsPerCta];
+#pragma unroll
+        for (int jj = 0; jj < kRowsPerCta; ++jj)
+            la[jj] = (j0 + jj < r) ? *reinterpret_cast<const uint4*>(LA + (size_t)(j0 + jj) * K + c * 8)
+                                   : make_uint4(0, 0, 0, 0);
+        float v[8];
+        smooth8(rc, v);
 #pragma unroll
         for (int jj = 0; jj < kRowsPerCta; ++jj) {
-            if (j0 + jj < r) {
-                uint4 raw = *reinterpret_cast<const uint4*>(LA + (size_t)(j0 + jj) * K + c * 8);
-                const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
-                float2 a = __half22float2(h2[0]), b = __half22float2(h2[1]);
-                float2 cc = __half22float2(h2[2]), d = __half22float2(h2[3]);
-                float t = acc[jj];
-                t = fmaf(a.x, x0.x, t); t = fmaf(a.y, x0.y, t);
-                t = fmaf(b.x, x0.z, t); t = fmaf(b.y, x0.w, t);
-                t = fmaf(cc.x, x1.x, t); t = fmaf(cc.y, x1.y, t);
-                t = fmaf(d.x, x1.z, t); t = fmaf(d.y, x1.w, t);
-                acc[jj] = t;
-            }
+            const __half2* h2 = reinterpret_cast<const __half2*>(&la[jj]);
+            const float2 a = __half22float2(h2[0]), b = __half22float2(h2[1]);
+            const float2 cc = __half22float2(h2[2]), d = __half22float2(h2[3]);
+            float t = acc[jj];
+            t = fmaf(a.x, v[0], t); t = fmaf(a.y, v[1], t);
+            t = fmaf(b.x, v[2], t); t = fmaf(b.y, v[3], t);
+            t = fmaf(cc.x, v[4], t); t = fmaf(cc.y, v[5], t);
+            t = fmaf(d.x, v[6], t); t = fmaf(d.y, v[7], t);
+            acc[jj] = t;
         }
     }
 #pragma unroll

@@ -187,11 +187,20 @@ __device__ __forceinline__ bool warp_mbar_wait(uint32_t bar, uint32_t parity, co
 // Group-collective form for a 128-thread unpack group: a single lane polls the mbarrier and the
 // outcome is spread by a hardware named barrier.  Keeps the mbarrier traffic of a group at one
 // wait per event instead of four.
+// The barrier numbers are literal (3 and 4) so that the kernel is known to use five hardware
+// barriers, not all sixteen.
+__device__ __forceinline__ bool group_bar_all(int group, bool pred) {
+    return group == 0 ? named_bar_all(3, 128, pred) : named_bar_all(4, 128, pred);
+}
+__device__ __forceinline__ void group_bar_sync(int group) {
+    if (group == 0) named_bar_sync(3, 128);
+    else named_bar_sync(4, 128);
+}
 __device__ __forceinline__ bool group_mbar_wait(uint32_t bar, uint32_t parity, const Abort& ab,
-                                                bool leader, int bar_id) {
+                                                bool leader, int group) {
     bool ok = true;
     if (leader) ok = mbar_wait(bar, parity, ab);
-    return named_bar_all(bar_id, 128, ok);
+    return group_bar_all(group, ok);
 }
 
 // ---------------------------------------------------------------------------
@@ -449,7 +458,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         const int gwarp = (warp - 2) & 3;          // warp within its group
         const int t128 = gwarp * 32 + lane;        // 0..127 within the group
         const bool leader = (t128 == 0);           // polls and signals the mbarriers for the group
-        const int gbar = 3 + group;                // hardware named barrier of the group
         Cursor cur;
         cur.init(u_begin, u_end, p);
         Work w;
@@ -460,14 +468,14 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 const int nkb = (w.kb1 - kb < KS) ? (w.kb1 - kb) : KS;
                 const int sw = cw % C::NW;   // cw counts stages
                 if ((int)(cw & 1u) != group) { ++cw; continue; }
-                ok = group_mbar_wait(bar(B_W_FULL + sw), (cw / C::NW) & 1, ab, leader, gbar);
+                ok = group_mbar_wait(bar(B_W_FULL + sw), (cw / C::NW) & 1, ab, leader, group);
                 if (!ok) break;
                 const uint8_t* wsrc = smem + C::OffW + sw * C::WBytes + row * 16;
 #pragma unroll
                 for (int sub = 0; sub < C::SPS; ++sub) {
                     const uint32_t cs = cw * C::SPS + sub;              // running A-slot counter
                     const int sa = cs % C::NA;
-                    ok = ok && group_mbar_wait(bar(B_FREE + sa), ((cs / C::NA) & 1) ^ 1, ab, leader, gbar);
+                    ok = ok && group_mbar_wait(bar(B_FREE + sa), ((cs / C::NA) & 1) ^ 1, ab, leader, group);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t a_tm = tm_a0 + sa * C::ASlotCols + ((uint32_t)(q * 32) << 16);
@@ -491,7 +499,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     }
                     tmem_wait_st();
                     tc_fence_before();
-                    named_bar_sync(gbar, 128);          // the whole group has written its rows
+                    group_bar_sync(group);              // the whole group has written its rows
                     if (leader) {
                         mbar_arrive(bar(B_READY + sa));
                         // ... and, after the last block, has the weight slot in registers: refill it
@@ -504,7 +512,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             if (ok && w.has_lr && group == 0) {
                 for (int c = 0; c < lr_chunks && ok; ++c) {
                     const int s = cl % C::NL;
-                    ok = group_mbar_wait(bar(B_FULL_LR + s), (cl / C::NL) & 1, ab, leader, gbar);
+                    ok = group_mbar_wait(bar(B_FULL_LR + s), (cl / C::NL) & 1, ab, leader, group);
                     if (!ok) break;
                     // T chunk: bf16 -> fp16 in place (same element size, same swizzled position)
                     uint8_t* tb = smem + C::OffT + s * C::TBytes;
@@ -521,7 +529,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                         *reinterpret_cast<uint4*>(tb + i * 16) = make_uint4(out[0], out[1], out[2], out[3]);
                     }
                     fence_proxy_async_smem();
-                    named_bar_sync(gbar, 128);
+                    group_bar_sync(group);
                     if (leader) mbar_arrive(bar(B_CONV_LR + s));
                     ++cl;
                 }

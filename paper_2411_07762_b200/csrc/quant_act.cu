@@ -854,26 +854,23 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             if (!ok) break;
             const uint32_t a0 = sb + L.x_ring + st * kXStageBytes + x_off, a1 = a0 ^ 16u;
             const uint4 v0 = lds128(a0), v1 = lds128(a1);
-            uint4 codes;
-            float v[8];
+            // x~ of the unit (all loaded words are consumed here) ...
+            float f0[8], f1[8];
             if (ones_sm[jj * 8 + cg]) {
-                cvt8(v0, v);
-                const uint2 lo = quant8_pairs(v, sc, rcp);
-                cvt8(v1, v);
-                const uint2 hi = quant8_pairs(v, sc, rcp);
-                codes = make_uint4(lo.x, lo.y, hi.x, hi.y);
+                cvt8(v0, f0);
+                cvt8(v1, f1);
             } else {
                 const float4* sp = reinterpret_cast<const float4*>(s + k0 + jj * kTCols + cg * 16);
-                div8(v0, __ldg(sp), __ldg(sp + 1), v);
-                const uint2 lo = quant8_pairs(v, sc, rcp);
-                div8(v1, __ldg(sp + 2), __ldg(sp + 3), v);
-                const uint2 hi = quant8_pairs(v, sc, rcp);
-                codes = make_uint4(lo.x, lo.y, hi.x, hi.y);
+                div8(v0, __ldg(sp), __ldg(sp + 1), f0);
+                div8(v1, __ldg(sp + 2), __ldg(sp + 3), f1);
             }
-            // The stage is released only now that the loaded values have been consumed: an
-            // arrival issued straight after the loads let the next TMA write overtake them.
+            // ... so the stage can be released now.  An arrival issued straight after the loads,
+            // before anything used their results, let the next TMA write overtake them.
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_free2(st));
+            const uint2 lo = quant8_pairs(f0, sc, rcp);
+            const uint2 hi = quant8_pairs(f1, sc, rcp);
+            const uint4 codes = make_uint4(lo.x, lo.y, hi.x, hi.y);
             if (jj >= kTOut) {      // the store that last read this tile is done with it
                 ok = qa_warp_wait(bar_out_free(o), (uint32_t)(jj / kTOut - 1) & 1u, abort_flag, lane);
                 if (!ok) break;
@@ -916,6 +913,20 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     }
 }
 
+// Opts the kernel in to `smem` bytes of dynamic shared memory (the one place that does it, so
+// that the value last set is known).
+int tma_set_smem(size_t smem) {
+    static size_t current = 0;
+    if (smem == current) return ASER_OK;
+    cudaError_t e = cudaFuncSetAttribute(quant_act_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) {
+        current = 0;
+        return record_cuda_error(e, "quant_act_tma smem attribute");
+    }
+    current = smem;
+    return ASER_OK;
+}
+
 // Clusters of `ck` CTAs of this kernel that the device keeps resident at once (0 if it cannot
 // schedule that size).  Queried once per (size, shared memory) pair.  The query counts with
 // the kernel's opted-in maximum of dynamic shared memory, so that is set to the size asked for.
@@ -923,7 +934,7 @@ int tma_active_clusters(int ck, size_t smem) {
     static int cached[17];
     static size_t cached_smem[17];
     if (cached_smem[ck] == smem && smem != 0) return cached[ck];
-    if (cudaFuncSetAttribute(quant_act_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+    if (tma_set_smem(smem) != ASER_OK) {
         (void)cudaGetLastError();
         return 0;
     }
@@ -982,11 +993,9 @@ int launch_tma(const __half* X, const float* s, const __half* LA, int M, int K, 
     if (ck == 0) { *unsupported = true; return ASER_OK; }
     const int kc = K / ck;
     const size_t smem = (size_t)tma_smem(kc, r, ck).total;
-    static size_t opted_in = 0;
-    if (smem != opted_in) {
-        cudaError_t e = cudaFuncSetAttribute(quant_act_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return record_cuda_error(e, "quant_act_tma smem attribute");
-        opted_in = smem;
+    {
+        const int rc = tma_set_smem(smem);
+        if (rc != ASER_OK) return rc;
     }
     CUtensorMap mx, mla, mq;
     int rc = encode_map_blocks(&mx, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, X, M, K, kTTok, 2);

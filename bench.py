@@ -42,6 +42,14 @@ WORKLOADS = {
     "c5_decode_m16_28672": (5, 16, 28672, 8192, 64, False, 50.0, 0.015, "hbm"),
     "c5_prefill_m4096_8192": (5, 4096, 8192, 8192, 64, False, 50.0, 0.015, "tensor"),
 }
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel (linear_tc) under
+# ncu, taken with the kernel as it stands in this tree; the summaries with the commands are under
+# profiles/ (linear_tc_<workload>.txt).  Workloads without a capture report null.
+NCU_DRAM_BYTES_PER_LAUNCH = {
+    "c2_decode_m8": 8.76e6,           # mean of two launches: 8.50 and 9.02 MB read, 0 written back
+    "c3_prefill_gate_up": 82.04e6,    # 45.4 MB read + 36.7 MB written
+}
 DEFAULT_WORKLOAD = "c2_decode_m8"
 
 
@@ -351,17 +359,18 @@ def run_ours(args, rank, world, local_rank):
 
     ms_step = ms_total / args.steps
     tops = whole_job_tops(ops, ms_step, world)
+    traffic = NCU_DRAM_BYTES_PER_LAUNCH.get(name)
     bytes_lin = algorithmic_bytes_linear(M, N, K, r)
     if b.bound == "hbm":
         achieved = bytes_lin / (ms_lin * 1e-3) / 1e9
         roof = dict(bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s",
-                    frac=achieved / peaks["hbm_gbs"], traffic=None,
+                    frac=achieved / peaks["hbm_gbs"], traffic=traffic,
                     peak_source=peaks["source"] + " copy bandwidth")
     else:
         peak = 2.0 * peaks["bf16_tflops"]   # int8 : bf16 dense nominal ratio is 2
         achieved = ops / (ms_lin * 1e-3) / 1e12
         roof = dict(bound="tensor", achieved=achieved, peak=peak, unit="TOP/s",
-                    frac=achieved / peak, traffic=None,
+                    frac=achieved / peak, traffic=traffic,
                     peak_source=peaks["source"] + " bf16 burst x2 (int8:bf16 nominal)")
     roof.update(kernel="linear_tc_kernel", us_per_launch=ms_lin * 1e3,
                 algorithmic_bytes=bytes_lin, ops=ops)

@@ -69,6 +69,9 @@ def test_repack_layout_by_definition(aser):
 ACT_CASES = [  # M, K, r
     (1, 512, 16), (3, 4096, 64), (8, 4096, 64), (16, 512, 16), (17, 1024, 0), (32, 8192, 32),
     (33, 512, 16), (127, 1024, 64), (129, 4096, 128), (300, 2048, 256), (64, 14336, 64),
+    # cluster kernel: one stage per CTA, r = 0, ranks that leave accumulator rows unused, ragged
+    # last token tile, every cluster size
+    (65, 128, 0), (200, 128, 48), (96, 8192, 32), (1000, 2048, 112), (2049, 512, 16), (40, 28672, 64),
 ]
 
 
@@ -90,6 +93,23 @@ def test_quant_act_parity(aser, M, K, r):
     if r:
         T_ref = F.down_proj(xs, L_A)
         assert_T_close(T.float().cpu().numpy(), T_ref)
+
+
+@pytest.mark.parametrize("M,K,r", [(8, 1024, 16), (300, 1024, 64), (2048, 512, 32)])
+def test_quant_act_dense_smoothing_vector(aser, M, K, r):
+    """Every divisor differs from 1 (a SmoothQuant-style vector): the division path everywhere,
+    including divisors below 1."""
+    lay = synth.make_layer(M, 8, K, seed=400 + M + K + r, n_cal=8)
+    rng = np.random.default_rng(M + K)
+    s = rng.uniform(0.25, 6.0, size=K).astype(np.float32)
+    s[::7] = 1.0
+    L_A = synth.standin_factors(8, K, r, seed=M, scale_a=0.05)[0]
+    xs = F.smooth_act(lay.X, s)
+    Xq_ref, sc_ref = F.quant_act(xs)
+    Xq, sc, T = aser.quant_act(to_dev(lay.X), to_dev(s), to_dev(L_A))
+    assert np.array_equal(Xq.cpu().numpy(), Xq_ref)
+    assert np.array_equal(bits(sc.cpu().numpy()), bits(sc_ref))
+    assert_T_close(T.float().cpu().numpy(), F.down_proj(xs, L_A))
 
 
 def test_quant_act_without_smoothing_vector(aser):

@@ -348,19 +348,21 @@ quant_act_large_kernel(const __half* __restrict__ X, const float* __restrict__ s
 //   one cluster barrier publishes both.  The owner sums the CK partials and writes T.
 //   Sweep 2: the slice is streamed again (it was just read, so it comes from L2), quantized,
 //   staged in shared memory and written by TMA stores, which also clip rows past M.
-// A warp handles one 16-column group for 32 rows (lane = row), so whether a unit needs the
-// division is uniform across the warp and the swizzled 16-byte accesses are conflict-free.
+// The 16 consumer warps form two groups that take alternate stages; inside its stage a warp
+// handles one 16-column group for all 64 rows (lane = row and row + 32), so whether a unit needs
+// the division is uniform across the warp and the swizzled 16-byte accesses are conflict-free.
 // A kernel that allocates tensor memory gets one CTA per SM, so the CTA uses most of the SM's
-// shared memory.
+// shared memory: the ring is as deep as fits (up to six stages).
 constexpr int kTTok = 64;                   // tokens per cluster (the MMA's N)
 constexpr int kTAtom = 64;                  // columns of one swizzled tile: 128 bytes of fp16
 constexpr int kTCols = 128;                 // columns per stage (two tiles)
-constexpr int kTConsumerWarps = 16;         // warp = (32-row block, 16-column group)
+constexpr int kTConsumerWarps = 16;         // two groups of eight: warp = (stage parity, 16-column group)
+constexpr int kTGroupWarps = 8;
 constexpr int kTConsumers = kTConsumerWarps * 32;
 constexpr int kTWarpProd = kTConsumerWarps;         // TMA producer warp
 constexpr int kTWarpMma = kTConsumerWarps + 1;      // MMA issuer warp, owns the tensor memory
 constexpr int kTThreads = kTConsumers + 64;
-constexpr int kTMaxStages = 4;              // activation / L_A ring depth (3 when r > 64)
+constexpr int kTMaxStages = 6;              // deepest activation / L_A ring
 constexpr int kTOut = 4;                    // int8 output tiles in flight
 constexpr int kTMaxRank = 128;              // larger r takes the mma.sync kernel
 constexpr int kXAtomBytes = kTTok * 128;    // 64 rows x 64 fp16
@@ -368,7 +370,19 @@ constexpr int kXStageBytes = 2 * kXAtomBytes;
 constexpr int kOutTileBytes = kTTok * kTCols;   // 64 rows x 128 int8
 constexpr long long kQaWaitLimitClocks = 4000000000ll;   // about 2 s of SM clocks per wait
 
-__host__ __device__ constexpr int tma_stages(int r) { return r <= 64 ? 4 : 3; }
+// Ring depth: as many stages (activation tile + L_A tile) as fit beside the exchange buffers.
+// A stage takes about 3 k cycles to go round (HBM latency plus the hand-overs between TMA,
+// consumers and MMA), so the depth sets the pace of sweep 1.
+__host__ __device__ constexpr int tma_stages(int r, int CK) {
+    const int per_stage = kXStageBytes + 256 * r;
+    const int exch = (CK > 1) ? 2 * kTTok * r * 4 : 0;
+    const int fixed = (exch > 16 * 1024 ? exch : 16 * 1024) + 12 * 1024;
+    int ns = (227 * 1024 - fixed) / per_stage;
+    if (ns * per_stage < kTOut * kOutTileBytes + kXStageBytes * ns) {      // region B must hold the output tiles
+        ns = (227 * 1024 - fixed - kTOut * kOutTileBytes) / kXStageBytes;
+    }
+    return ns > kTMaxStages ? kTMaxStages : (ns < 2 ? 2 : ns);
+}
 
 struct TmaSmem {
     int x_ring, region_b, la_atom_bytes, la_stage_bytes, t_slots, t_stage, ones, amax_cg, amax_stage,
@@ -380,7 +394,7 @@ struct TmaSmem {
 // so that an MMA whose L_A tile has fewer than 128 rows still reads inside the allocation.
 __host__ __device__ inline TmaSmem tma_smem(int Kc, int r, int CK) {
     TmaSmem L;
-    const int ns = tma_stages(r);
+    const int ns = tma_stages(r, CK);
     int off = 0;
     L.x_ring = off;     off += ns * kXStageBytes;
     L.region_b = off;
@@ -399,7 +413,7 @@ __host__ __device__ inline TmaSmem tma_smem(int Kc, int r, int CK) {
     }
     L.t_stage = off;    off += (CK > 1) ? kTTok * r * 4 : 0;   // this CTA's partial T, [token][r]
     L.ones = off;       off += (Kc / 16 + 15) / 16 * 16;       // per 16 columns: all divisors are 1
-    L.amax_cg = off;    off += 8 * kTTok * 4;                  // row maxima per 16-column group
+    L.amax_cg = off;    off += 16 * kTTok * 4;                 // row maxima per (stage parity, 16-column group)
     L.amax_stage = off; off += kTTok * 4;                      // row maxima of this CTA's slice
     L.amax_slots = off; off += 16 * kTTok * 4;                 // row maxima copied in by each CTA
     L.bars = off;       off += (4 * kTMaxStages + 2 * kTOut + 3) * 8;
@@ -568,7 +582,7 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     const uint32_t sb = (sraw + 1023u) & ~1023u;            // swizzled tiles need 1 KiB alignment
     uint8_t* smem = smem_raw + (sb - sraw);
     const TmaSmem L = tma_smem(Kc, r, CK);
-    const int NS = tma_stages(r);
+    const int NS = tma_stages(r, CK);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t rank = cluster_rank();
     const int m0 = blockIdx.y * kTTok;
@@ -629,12 +643,12 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         if (lane == 0) {
             for (int st = 0; st < kTMaxStages; ++st) {
                 mbar_init(bar_full(st), 1);                     // the producer's expect_tx arrival
-                mbar_init(bar_ready(st), kTConsumerWarps);      // consumers are done with the stage
+                mbar_init(bar_ready(st), kTGroupWarps);         // the stage's consumer group is done with it
                 mbar_init(bar_free1(st), 1);                    // sweep 1: the MMAs have read it
-                mbar_init(bar_free2(st), kTConsumerWarps);      // sweep 2: the consumers have read it
+                mbar_init(bar_free2(st), kTGroupWarps);         // sweep 2: the group has read it
             }
             for (int o = 0; o < kTOut; ++o) {
-                mbar_init(bar_out_full(o), kTConsumerWarps);    // an output tile is written
+                mbar_init(bar_out_full(o), kTGroupWarps);       // an output tile is written
                 mbar_init(bar_out_free(o), 1);                  // its store has read it
             }
             mbar_init(bar_acc, 1);
@@ -740,48 +754,67 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         __syncwarp();
     } else {
         // ================= consumers =================
-        // this thread's unit inside a stage: row and 16-column group (two 16-byte pieces of one
-        // swizzled tile; their places differ in address bit 4)
-        const int rb = warp >> 3, cg = warp & 7;
-        const int row = rb * 32 + lane;
+        // The 16 consumer warps form two groups that take alternate stages, so that two stages
+        // are worked on at any time.  Inside its stage a warp owns one 16-column group for all 64
+        // rows: lane = row and row + 32 (two 16-byte pieces each, of one swizzled tile; their
+        // places differ in address bit 4).
+        const int grp = warp >> 3, cg = warp & 7;
+        const int row = lane;                                   // and row + 32
         const uint32_t x_off = (uint32_t)(cg >> 2) * kXAtomBytes + (uint32_t)row * 128u +
                                (uint32_t)(((2 * (cg & 3)) ^ (row & 7)) << 4);
+        constexpr uint32_t kRow32 = 32u * 128u;                 // 32 rows further down the tile
         // ---- sweep 1: row maxima; units with divisors get x~ written back as fp16 ----
-        float amax = 0.f;
-        __half2 hamax = __float2half2_rn(0.f);
+        float amax0 = 0.f, amax1 = 0.f;
+        __half2 hamax0 = __float2half2_rn(0.f), hamax1 = hamax0;
         bool ok = true;
-        for (int i = 0; i < nst; ++i) {
+        for (int i = grp; i < nst; i += 2) {
             const int st = i % NS;
             ok = qa_warp_wait(bar_full(st), (uint32_t)(i / NS) & 1u, abort_flag, lane);
             if (!ok) break;
             const uint32_t a0 = sb + L.x_ring + st * kXStageBytes + x_off, a1 = a0 ^ 16u;
             const uint4 v0 = lds128(a0), v1 = lds128(a1);
+            const uint4 w0 = lds128(a0 + kRow32), w1 = lds128(a1 + kRow32);
             if (ones_sm[i * 8 + cg]) {
                 const __half2* h0 = reinterpret_cast<const __half2*>(&v0);
                 const __half2* h1 = reinterpret_cast<const __half2*>(&v1);
+                const __half2* g0 = reinterpret_cast<const __half2*>(&w0);
+                const __half2* g1 = reinterpret_cast<const __half2*>(&w1);
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    hamax = __hmax2(hamax, __habs2(h0[e]));
-                    hamax = __hmax2(hamax, __habs2(h1[e]));
+                    hamax0 = __hmax2(hamax0, __habs2(h0[e]));
+                    hamax1 = __hmax2(hamax1, __habs2(g0[e]));
+                    hamax0 = __hmax2(hamax0, __habs2(h1[e]));
+                    hamax1 = __hmax2(hamax1, __habs2(g1[e]));
                 }
             } else {
                 const float4* sp = reinterpret_cast<const float4*>(s + k0 + i * kTCols + cg * 16);
+                const float4 s0 = __ldg(sp), s1 = __ldg(sp + 1), s2 = __ldg(sp + 2), s3 = __ldg(sp + 3);
                 float v[8];
-                div8(v0, __ldg(sp), __ldg(sp + 1), v);
+                div8(v0, s0, s1, v);
 #pragma unroll
-                for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(v[e]));
+                for (int e = 0; e < 8; ++e) amax0 = fmaxf(amax0, fabsf(v[e]));
                 sts128(a0, pack8_half(v));
-                div8(v1, __ldg(sp + 2), __ldg(sp + 3), v);
+                div8(v1, s2, s3, v);
 #pragma unroll
-                for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(v[e]));
+                for (int e = 0; e < 8; ++e) amax0 = fmaxf(amax0, fabsf(v[e]));
                 sts128(a1, pack8_half(v));
+                div8(w0, s0, s1, v);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) amax1 = fmaxf(amax1, fabsf(v[e]));
+                sts128(a0 + kRow32, pack8_half(v));
+                div8(w1, s2, s3, v);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) amax1 = fmaxf(amax1, fabsf(v[e]));
+                sts128(a1 + kRow32, pack8_half(v));
                 fence_proxy_async_smem();       // the MMA reads these through the async proxy
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_ready(st));
         }
-        amax = fmaxf(amax, fmaxf(__low2float(hamax), __high2float(hamax)));
-        amax_cg[cg * kTTok + row] = amax;
+        amax0 = fmaxf(amax0, fmaxf(__low2float(hamax0), __high2float(hamax0)));
+        amax1 = fmaxf(amax1, fmaxf(__low2float(hamax1), __high2float(hamax1)));
+        amax_cg[warp * kTTok + row] = amax0;
+        amax_cg[warp * kTTok + row + 32] = amax1;
         if (CK > 1) cluster_wait();     // every CTA of the cluster has its barriers set up
         named_bar_sync(1, kTConsumers);
         // ---- row maxima of this slice; copied into every CTA of the cluster (each needs all
@@ -789,7 +822,7 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         if (tid < kTTok) {
             float a = amax_cg[tid];
 #pragma unroll
-            for (int g = 1; g < 8; ++g) a = fmaxf(a, amax_cg[g * kTTok + tid]);
+            for (int g = 1; g < 16; ++g) a = fmaxf(a, amax_cg[g * kTTok + tid]);
             amax_stage[tid] = a;
             fence_proxy_async_smem();
         }
@@ -832,51 +865,69 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             }
         }
 
-        // ---- row scale of this thread's row; the owner of a row writes it out ----
-        float sc;
+        // ---- row scales of this thread's two rows; the owner of a row writes its scale out ----
+        float sc0, sc1;
         if (CK > 1) {
             if (ok) ok = qa_warp_wait(bar_amax, 0u, abort_flag, lane);     // all row maxima have landed
-            float a = 0.f;
-            for (int qq = 0; qq < CK; ++qq) a = fmaxf(a, amax_slots[qq * kTTok + row]);
-            sc = __fdiv_rn(a, 127.0f);
+            float a = 0.f, b = 0.f;
+            for (int qq = 0; qq < CK; ++qq) {
+                a = fmaxf(a, amax_slots[qq * kTTok + row]);
+                b = fmaxf(b, amax_slots[qq * kTTok + row + 32]);
+            }
+            sc0 = __fdiv_rn(a, 127.0f);
+            sc1 = __fdiv_rn(b, 127.0f);
         } else {
             named_bar_sync(1, kTConsumers);
-            sc = __fdiv_rn(amax_stage[row], 127.0f);
+            sc0 = __fdiv_rn(amax_stage[row], 127.0f);
+            sc1 = __fdiv_rn(amax_stage[row + 32], 127.0f);
         }
-        if (cg == 0 && (int)rank == row / rows_owned && m0 + row < M) a_scale[m0 + row] = sc;
+        if (warp == 0) {
+            if ((int)rank == row / rows_owned && m0 + row < M) a_scale[m0 + row] = sc0;
+            if ((int)rank == (row + 32) / rows_owned && m0 + row + 32 < M) a_scale[m0 + row + 32] = sc1;
+        }
 
         // ---- sweep 2: int8 codes into the output tiles (they take the place of the L_A ring;
         // the wait on the accumulator above says the MMAs are done reading it) ----
-        const float rcp = (sc > 0.f) ? __frcp_rn(sc) : 0.f;
-        for (int jj = 0; jj < nst && ok; ++jj) {
+        const float rcp0 = (sc0 > 0.f) ? __frcp_rn(sc0) : 0.f;
+        const float rcp1 = (sc1 > 0.f) ? __frcp_rn(sc1) : 0.f;
+        for (int jj = grp; jj < nst && ok; jj += 2) {
             const int i = nst + jj, st = i % NS, o = jj % kTOut;
             ok = qa_warp_wait(bar_full(st), (uint32_t)(i / NS) & 1u, abort_flag, lane);
             if (!ok) break;
             const uint32_t a0 = sb + L.x_ring + st * kXStageBytes + x_off, a1 = a0 ^ 16u;
             const uint4 v0 = lds128(a0), v1 = lds128(a1);
-            // x~ of the unit (all loaded words are consumed here) ...
-            float f0[8], f1[8];
+            const uint4 w0 = lds128(a0 + kRow32), w1 = lds128(a1 + kRow32);
+            // x~ of the two units (all loaded words are consumed here) ...
+            float f0[8], f1[8], g0[8], g1[8];
             if (ones_sm[jj * 8 + cg]) {
                 cvt8(v0, f0);
                 cvt8(v1, f1);
+                cvt8(w0, g0);
+                cvt8(w1, g1);
             } else {
                 const float4* sp = reinterpret_cast<const float4*>(s + k0 + jj * kTCols + cg * 16);
-                div8(v0, __ldg(sp), __ldg(sp + 1), f0);
-                div8(v1, __ldg(sp + 2), __ldg(sp + 3), f1);
+                const float4 s0 = __ldg(sp), s1 = __ldg(sp + 1), s2 = __ldg(sp + 2), s3 = __ldg(sp + 3);
+                div8(v0, s0, s1, f0);
+                div8(v1, s2, s3, f1);
+                div8(w0, s0, s1, g0);
+                div8(w1, s2, s3, g1);
             }
             // ... so the stage can be released now.  An arrival issued straight after the loads,
             // before anything used their results, let the next TMA write overtake them.
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_free2(st));
-            const uint2 lo = quant8_pairs(f0, sc, rcp);
-            const uint2 hi = quant8_pairs(f1, sc, rcp);
-            const uint4 codes = make_uint4(lo.x, lo.y, hi.x, hi.y);
+            const uint2 lo0 = quant8_pairs(f0, sc0, rcp0);
+            const uint2 hi0 = quant8_pairs(f1, sc0, rcp0);
+            const uint2 lo1 = quant8_pairs(g0, sc1, rcp1);
+            const uint2 hi1 = quant8_pairs(g1, sc1, rcp1);
             if (jj >= kTOut) {      // the store that last read this tile is done with it
                 ok = qa_warp_wait(bar_out_free(o), (uint32_t)(jj / kTOut - 1) & 1u, abort_flag, lane);
                 if (!ok) break;
             }
             // output tile: rows of 128 bytes, 16-byte piece cg at its swizzled place
-            sts128(sb + L.region_b + o * kOutTileBytes + (uint32_t)row * 128u + (uint32_t)((cg ^ (row & 7)) << 4), codes);
+            const uint32_t od = sb + L.region_b + o * kOutTileBytes + (uint32_t)row * 128u + (uint32_t)((cg ^ (row & 7)) << 4);
+            sts128(od, make_uint4(lo0.x, lo0.y, hi0.x, hi0.y));
+            sts128(od + kRow32, make_uint4(lo1.x, lo1.y, hi1.x, hi1.y));
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_out_full(o));
@@ -898,7 +949,10 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                     *reinterpret_cast<__nv_bfloat162*>(T + (size_t)(m0 + t) * r + col) = __floats2bfloat162_rn(s0, s1);
             }
         }
-        if (*abort_flag && cg == 0 && m0 + row < M) a_scale[m0 + row] = __int_as_float(0x7fc00000);   // a wait gave up: poison the rows
+        if (*abort_flag && warp == 0) {     // a wait gave up: poison the rows
+            if (m0 + row < M) a_scale[m0 + row] = __int_as_float(0x7fc00000);
+            if (m0 + row + 32 < M) a_scale[m0 + row + 32] = __int_as_float(0x7fc00000);
+        }
     }
     // Nobody leaves while a peer may still copy from or into this CTA's shared memory.
     if (CK > 1) {

@@ -832,6 +832,17 @@ int launch_linear_tc(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
     long long want = (L.units + 1) / 2;   // at least two units per CTA on tiny problems
     if (want < 1) want = 1;
     if (grid > want) grid = (int)want;
+    // Tiles that have to be split anyway are split evenly: with a grid that divides the units
+    // into equal shares of a whole fraction of a tile, every CTA has exactly one (partial) work
+    // item instead of up to three, at the price of a few idle SMs.
+    {
+        const long long KBl = K / 128;
+        for (int g = grid; g >= grid - grid / 6 && g >= 1; --g) {
+            if (L.units % g) continue;
+            const long long share = L.units / g;
+            if (share < KBl && KBl % share == 0) { grid = g; break; }
+        }
+    }
 
     CUtensorMap mx, mlb, mt;
     const int ks = L.BT == 16 ? Cfg<16>::KS : L.BT == 32 ? Cfg<32>::KS : L.BT == 64 ? Cfg<64>::KS : Cfg<128>::KS;

@@ -234,3 +234,25 @@ def test_forward_overlapped_is_bit_identical_to_separate_calls(aser, M, N, K, r)
         for g, w in zip(got, want[it & 1]):
             assert torch.equal(g.view(torch.uint8), w.view(torch.uint8)), it
     aser.check_status(layer.ws)
+
+
+@pytest.mark.parametrize("name", ["k", "gate", "down"])
+def test_config4_block_linears_full_size_sampled_rows(aser, name):
+    """Decoder-block linears at 4096 tokens, rank 128 (the GQA projection, the widest and the
+    deepest layer): every int8 code and scale, and Y on sampled token rows."""
+    lay, r = synth.config4_block_layer(name)
+    s, Wq, w_scale, L_A, L_B = oracle_layer(lay, r, construct=False)
+    rows = np.array([0, 63, 64, 2047, 2048, 4031, 4095])
+    run_path(aser, lay, s, Wq, w_scale, L_A, L_B, "tc", rows=rows, use_dgemm=True)
+
+
+@pytest.mark.parametrize("M,N,r", [(16, 8192, 32), (128, 28672, 256), (1024, 8192, 128), (4096, 8192, 0)])
+def test_config5_sweep_points_sampled_rows(aser, M, N, r):
+    """Points of the 70B-class sweep (K = 8192), including rank 256 (the quantization kernel's
+    mma.sync path) and rank 0 (plain W4A8)."""
+    lay = synth.config5_point(M, N)
+    s, Wq, w_scale, L_A, L_B = oracle_layer(lay, r, construct=False)
+    if r == 0:
+        L_A = L_B = None
+    rows = np.unique(np.array([0, 1, M // 2, M - 2, M - 1]).clip(0, M - 1))
+    run_path(aser, lay, s, Wq, w_scale, L_A, L_B, "tc", rows=rows, use_dgemm=True)

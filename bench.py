@@ -439,6 +439,159 @@ def extra_points(args, dev, peaks, skip):
     return out
 
 
+# ---------------------------------------------------------------------------
+# sweeps over the other benchmark configurations (not the headline line)
+# ---------------------------------------------------------------------------
+class SweepLayer:
+    """One weight matrix packed once, stand-in factors of the largest rank, and rolled copies of
+    the packed weights; `point(M, r)` gives operand sets (views and fresh intermediates) for one
+    (tokens, rank) point, as many as it takes to exceed twice the L2 size between reuses."""
+
+    def __init__(self, dev, cfg, index, N, K, r_max, M_max, gain, sigma, gated=False):
+        import torch
+        import paper_2411_07762_b200 as aser
+        self.torch, self.aser, self.dev = torch, aser, dev
+        self.N, self.K, self.r_max = N, K, r_max
+        lay = synth.make_layer(M_max, N, K, seed=synth.seed_for(cfg, index), outlier_gain=gain,
+                               sigma_w=sigma, n_cal=8, gated_input=gated)
+        t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+        self.s = t(synth.standin_smoothing_vector(K, lay.outlier_idx, 24.0))
+        L_A, L_B = synth.standin_factors(N, K, max(r_max, 16), seed=lay.meta["seed"],
+                                         scale_a=0.01, scale_b=0.01)
+        self.L_A, self.L_B = t(L_A), t(L_B)
+        Wq, self.w_scale = aser.pack_w4(t(lay.W), self.s)
+        self.Wk = [aser.repack_w4(Wq)]
+        del Wq
+        self.X = t(lay.X)
+        torch.cuda.empty_cache()
+
+    def point(self, M, r):
+        torch, aser = self.torch, self.aser
+        N, K = self.N, self.K
+        per_set = N * K // 2 + 2 * r * (N + K) + 3 * M * K + 2 * M * N
+        n_sets = 1 if per_set > 2 * L2_BYTES else int(np.ceil(2.2 * L2_BYTES / per_set))
+        while len(self.Wk) < n_sets:
+            self.Wk.append(torch.roll(self.Wk[0], shifts=8192 * len(self.Wk)))
+        sets = []
+        for i in range(n_sets):
+            L = object.__new__(aser.AserLinear)
+            L.N, L.K, L.r, L.s, L.max_tokens = N, K, r, self.s, M
+            L.L_A = torch.roll(self.L_A[:r], shifts=i, dims=0).contiguous() if r else None
+            L.L_B = torch.roll(self.L_B[:, :r], shifts=i, dims=0).contiguous() if r else None
+            L.Wk, L.w_scale = self.Wk[i], self.w_scale
+            L.Xq = torch.empty((M, K), dtype=torch.int8, device=self.dev)
+            L.a_scale = torch.empty((M,), dtype=torch.float32, device=self.dev)
+            L.T = torch.empty((M, max(r, 1)), dtype=torch.bfloat16, device=self.dev)
+            L.Y = torch.empty((M, N), dtype=torch.float16, device=self.dev)
+            L.ws = aser.new_workspace(M, N, K, r, self.dev)
+            X = self.X[:M] if i == 0 else torch.roll(self.X[:M], shifts=i, dims=1).contiguous()
+            sets.append((L, X))
+        return sets
+
+
+def time_calls(torch, fn, steps):
+    """Device time (us per call) of `steps` calls of fn(i) replayed from one CUDA graph."""
+    side = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g, stream=side):
+            for i in range(steps):
+                fn(i)
+    torch.cuda.synchronize()
+    best = float("inf")
+    for _ in range(3):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        best = min(best, e0.elapsed_time(e1))
+    return best * 1e3 / steps
+
+
+def time_point(torch, aser, sets, M, N, K, r, peaks):
+    n = len(sets)
+    steps = 240 if M <= 128 else (48 if M <= 1024 else 16)
+    steps = max(steps, 2 * n)
+    for L, X in sets:                      # warm-up, every operand set touched
+        for _ in range(3):
+            L(X)
+    torch.cuda.synchronize()
+    us_step = time_calls(torch, lambda i: sets[i % n][0](sets[i % n][1]), steps)
+    us_lin = time_calls(torch, lambda i: sets[i % n][0].linear(M, True), steps)
+    us_act = time_calls(torch, lambda i: sets[i % n][0].quant(sets[i % n][1]), steps)
+    for L, _ in sets:
+        aser.check_status(L.ws)
+    ops = 2.0 * M * N * K
+    gbs = algorithmic_bytes_linear(M, N, K, r) / (us_lin * 1e-6) / 1e9
+    tops = ops / (us_lin * 1e-6) / 1e12
+    return dict(M=M, N=N, K=K, r=r, us_step=us_step, us_linear=us_lin, us_quant_act=us_act,
+                tops_linear=tops, tops_step=ops / (us_step * 1e-6) / 1e12, gbs_linear=gbs,
+                frac_hbm=gbs / peaks["hbm_gbs"], frac_tensor=tops / (2.0 * peaks["bf16_tflops"]),
+                quant_act_gbs=algorithmic_bytes_act(M, K, r) / (us_act * 1e-6) / 1e9,
+                operand_sets=n)
+
+
+def run_sweep(args, local_rank):
+    """`--sweep c4`: the seven linears of a decoder block at 4096 tokens, rank 128, each alone and
+    all back to back.  `--sweep c5`: the 70B-class grid (two shapes x five token counts x five
+    ranks) with the low-rank overhead against the rank-0 point.  One JSON line."""
+    import torch
+    import paper_2411_07762_b200 as aser
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    peaks = load_peaks()
+    points = []
+    with ClockSampler(local_rank) as clk:
+        if args.sweep == "c4":
+            M, r = 4096, 128
+            block = []
+            for i, (nm, K, N) in enumerate(synth.DECODER_BLOCK_LINEARS):
+                sl = SweepLayer(dev, 4, i, N, K, r, M, 30.0, 0.02)
+                sets = sl.point(M, r)
+                plain = sl.point(M, 0)
+                pt = time_point(torch, aser, sets, M, N, K, r, peaks)
+                p0 = time_point(torch, aser, plain, M, N, K, 0, peaks)
+                pt.update(layer=nm, us_linear_plain=p0["us_linear"], us_step_plain=p0["us_step"],
+                          lowrank_overhead_linear=pt["us_linear"] / p0["us_linear"] - 1.0,
+                          lowrank_overhead_step=pt["us_step"] / p0["us_step"] - 1.0)
+                points.append(pt)
+                block.append(sets[0])
+                del plain
+            def whole_block(i):
+                for L, X in block:
+                    L(X)
+            us_block = time_calls(torch, whole_block, 8)
+            ops_block = sum(2.0 * M * p["N"] * p["K"] for p in points)
+            summary = dict(us_block=us_block, sum_of_layers_us=sum(p["us_step"] for p in points),
+                           tops_block=ops_block / (us_block * 1e-6) / 1e12,
+                           frac_tensor_block=ops_block / (us_block * 1e-6) / 1e12 / (2.0 * peaks["bf16_tflops"]))
+        else:
+            summary = {}
+            for N in (8192, 28672):
+                sl = SweepLayer(dev, 5, N // 1024, N, 8192, 256, 4096, 50.0, 0.015)
+                for M in (1, 16, 128, 1024, 4096):
+                    base = None
+                    for r in (0, 32, 64, 128, 256):
+                        sets = sl.point(M, r)
+                        pt = time_point(torch, aser, sets, M, N, 8192, r, peaks)
+                        if r == 0:
+                            base = pt
+                        pt.update(lowrank_overhead_linear=pt["us_linear"] / base["us_linear"] - 1.0,
+                                  lowrank_overhead_step=pt["us_step"] / base["us_step"] - 1.0)
+                        points.append(pt)
+                        del sets
+                        torch.cuda.empty_cache()
+                del sl
+                torch.cuda.empty_cache()
+        clocks = clk.summary()
+    line = dict(sweep=args.sweep, unit_time="us per call, CUDA-graph replay, best of 3",
+                peaks=dict(hbm_gbs=peaks["hbm_gbs"], int8_tops=2.0 * peaks["bf16_tflops"],
+                           source=peaks["source"]),
+                points=points, clocks=clocks, **summary)
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -449,12 +602,18 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle timing")
     ap.add_argument("--no-extra", dest="extra", action="store_false",
                     help="skip the additional sweep points")
+    ap.add_argument("--sweep", choices=["c4", "c5"], default=None,
+                    help="time the decoder-block linears (c4) or the 70B-class grid (c5) instead")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
         run_reference(args, rank, world)
+        return
+    if args.sweep:
+        if rank == 0:
+            run_sweep(args, local_rank)
         return
     run_ours(args, rank, world, local_rank)
 

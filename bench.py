@@ -43,13 +43,18 @@ WORKLOADS = {
     "c5_prefill_m4096_8192": (5, 4096, 8192, 8192, 64, False, 50.0, 0.015, "tensor"),
 }
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel (linear_tc) under
-# ncu, taken with the kernel as it stands in this tree; the summaries with the commands are under
-# profiles/ (linear_tc_<workload>.txt).  Workloads without a capture report null.
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel under ncu, taken
+# with the kernel as it stands in this tree; the summaries with the commands are under profiles/
+# (<kernel>_<workload>.txt).  Workloads without a capture of the current kernel report null.
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    "c2_decode_m8": 8.76e6,           # mean of two launches: 8.50 and 9.02 MB read, 0 written back
     "c3_prefill_gate_up": 82.04e6,    # 45.4 MB read + 36.7 MB written
 }
+
+
+def dominant_kernel(M, N, K):
+    """Name of the kernel the library runs for the integer product at this shape (few tokens and
+    at most 64 MB of packed weights: the streaming kernel; otherwise the tensor-core kernel)."""
+    return "linear_decode_kernel" if M <= 16 and N * K // 2 <= (64 << 20) else "linear_tc_kernel"
 DEFAULT_WORKLOAD = "c2_decode_m8"
 
 
@@ -372,7 +377,7 @@ def run_ours(args, rank, world, local_rank):
         roof = dict(bound="tensor", achieved=achieved, peak=peak, unit="TOP/s",
                     frac=achieved / peak, traffic=traffic,
                     peak_source=peaks["source"] + " bf16 burst x2 (int8:bf16 nominal)")
-    roof.update(kernel="linear_tc_kernel", us_per_launch=ms_lin * 1e3,
+    roof.update(kernel=dominant_kernel(M, N, K), us_per_launch=ms_lin * 1e3,
                 algorithmic_bytes=bytes_lin, ops=ops)
 
     line = dict(

@@ -92,7 +92,9 @@ int aser_quant_act(const void* X_f16, const float* s, const void* LA_f16,
  * int32 accumulators [M,N] (bit-exact); pass NULL in timed runs.  workspace must hold
  * aser_workspace_bytes(M,N,K,r) bytes, must have been zeroed once with
  * aser_workspace_init, and may be reused by later calls on the same stream; two calls
- * that overlap in time need separate workspaces.
+ * that overlap in time need separate workspaces.  With at most 16 tokens and at most 64 MB of
+ * packed weights the call runs a streaming kernel that leaves the workspace untouched; the
+ * argument is validated all the same, so callers need not know which kernel serves a shape.
  * aser_linear_w4a8 is the same without the low-rank term (the plain W4A8 control).
  */
 int aser_linear_w4a8_lr(const int8_t* Xq, const float* a_scale, const void* Wk,
@@ -114,7 +116,8 @@ int aser_linear_w4a8_lr_simt(const int8_t* Xq, const float* a_scale, const uint8
                              void* stream);
 
 /*
- * aser_linear_w4a8_lr_static -- aser_linear_w4a8_lr for callers that must not allocate device
+ * aser_linear_w4a8_lr_static -- the tensor-core kernel of aser_linear_w4a8_lr (the one that needs
+ * scratch memory, at every shape this entry accepts) for callers that must not allocate device
  * memory and therefore have no workspace to hand over: code running inside a memory budget
  * that was fixed at start-up (a serving process that gave every free byte to its own pool, so
  * cudaMalloc would fail), or at a point where allocating is not allowed because it would

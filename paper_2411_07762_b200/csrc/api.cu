@@ -87,6 +87,12 @@ int linear_common(const int8_t* Xq, const float* a_scale, const void* Wk, const 
         return fail(ASER_ERR_WORKSPACE, "workspace missing, misaligned or too small");
     int rc = check_device();
     if (rc != ASER_OK) return rc;
+    if (linear_decode_prefers(M, N, K))   // few tokens: the streaming kernel (the workspace stays untouched)
+        return launch_linear_decode(Xq, a_scale, static_cast<const uint8_t*>(Wk), w_scale,
+                                    static_cast<const __nv_bfloat16*>(T_bf16),
+                                    static_cast<const __half*>(LB_f16), M, N, K, r,
+                                    static_cast<__half*>(Y_f16), acc_debug,
+                                    static_cast<cudaStream_t>(stream), overlap_prev);
     return launch_linear_tc(Xq, a_scale, static_cast<const uint8_t*>(Wk), w_scale,
                             static_cast<const __nv_bfloat16*>(T_bf16),
                             static_cast<const __half*>(LB_f16), M, N, K, r,

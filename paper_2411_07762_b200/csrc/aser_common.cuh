@@ -38,6 +38,14 @@ int launch_linear_tc(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
                      int M, int N, int K, int r, __half* Y, int32_t* acc_debug,
                      void* workspace, size_t workspace_bytes, cudaStream_t st,
                      bool overlap_prev = false);
+// Few-token kernel (M <= kLinearDecodeMaxTokens): streams the weights once, no workspace.
+// linear_decode_prefers: the shapes for which it is faster than the tensor-core kernel.
+constexpr int kLinearDecodeMaxTokens = 16;
+bool linear_decode_prefers(int M, int N, int K);
+int launch_linear_decode(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
+                         const float* w_scale, const __nv_bfloat16* T, const __half* LB,
+                         int M, int N, int K, int r, __half* Y, int32_t* acc_debug,
+                         cudaStream_t st, bool overlap_prev = false);
 size_t linear_tc_workspace_bytes(int M, int N, int K, int r);
 // Leading bytes of the workspace (status word + tile counters) that must be zero at launch.
 size_t linear_tc_zeroed_prefix_bytes(int M, int N, int K, int r);

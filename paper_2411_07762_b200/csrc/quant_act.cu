@@ -567,7 +567,7 @@ __device__ __forceinline__ uint2 quant8_pairs(const float (&v)[8], float sc, flo
 }
 
 // grid = (CK, ceil(M / 64)), cluster = (CK, 1, 1) with CK a power of two <= 16, kTThreads threads,
-// r <= 128.
+// r <= 128.  T has `ldt` elements per row (the launch may cover a column range of a wider T).
 // map_x: X as fp16 [K / 64 blocks][M][64], box 2 blocks x 64 rows, 128-byte swizzle.
 // map_la: L_A as fp16 [K / 64 blocks][r][64], box 2 blocks x r rows (unused when r == 0).
 // map_q: Xq as bytes [M, K], box 64 rows x 128 columns, 128-byte swizzle.
@@ -575,7 +575,7 @@ __global__ void __launch_bounds__(kTThreads, 1)
 quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_la,
                      const __grid_constant__ CUtensorMap map_q, const float* __restrict__ s,
                      int M, int K, int Kc, int r, int CK, float* __restrict__ a_scale,
-                     __nv_bfloat16* __restrict__ T) {
+                     __nv_bfloat16* __restrict__ T, int ldt) {
     extern __shared__ uint8_t smem_raw[];
     grid_dep_launch();      // a dependent linear kernel may start streaming its weights
     const uint32_t sraw = smem_u32(smem_raw);
@@ -849,7 +849,7 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                     for (int e = 0; e < 16; ++e) {
                         const int t = t0 + e;
                         if (CK > 1) t_stage[t * r + j] = __uint_as_float(v[e]);
-                        else if (m0 + t < M) T[(size_t)(m0 + t) * r + j] = __float2bfloat16_rn(__uint_as_float(v[e]));
+                        else if (m0 + t < M) T[(size_t)(m0 + t) * ldt + j] = __float2bfloat16_rn(__uint_as_float(v[e]));
                     }
                 }
             }
@@ -946,7 +946,7 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                     s0 += pv.x; s1 += pv.y;
                 }
                 if (m0 + t < M)
-                    *reinterpret_cast<__nv_bfloat162*>(T + (size_t)(m0 + t) * r + col) = __floats2bfloat162_rn(s0, s1);
+                    *reinterpret_cast<__nv_bfloat162*>(T + (size_t)(m0 + t) * ldt + col) = __floats2bfloat162_rn(s0, s1);
             }
         }
         if (*abort_flag && warp == 0) {     // a wait gave up: poison the rows
@@ -1034,7 +1034,7 @@ int pick_tma_cluster(int M, int K, int r, int max_ck) {
 }
 
 int launch_tma(const __half* X, const float* s, const __half* LA, int M, int K, int r,
-               int8_t* Xq, float* a_scale, __nv_bfloat16* T, cudaStream_t st, bool* unsupported) {
+               int8_t* Xq, float* a_scale, __nv_bfloat16* T, int ldt, cudaStream_t st, bool* unsupported) {
     *unsupported = false;
     static int max_ck = 0;      // 16 where the device allows clusters beyond the portable 8
     if (max_ck == 0) {
@@ -1075,7 +1075,7 @@ int launch_tma(const __half* X, const float* s, const __half* LA, int M, int K, 
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, quant_act_tma_kernel, mx, mla, mq, s, M, K, kc, r, ck, a_scale, T);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, quant_act_tma_kernel, mx, mla, mq, s, M, K, kc, r, ck, a_scale, T, ldt);
     if (e != cudaSuccess) return record_cuda_error(e, "quant_act_tma_kernel");
     return check_launch("quant_act_tma_kernel");
 }
@@ -1115,7 +1115,23 @@ int launch_quant_act(const __half* X, const float* s, const __half* LA, int M, i
         return check_launch("quant_act_small_kernel");
     }
     bool unsupported = false;
-    const int rc = launch_tma(X, s, LA, M, K, r, Xq, a_scale, T, st, &unsupported);
+    if (r > kTMaxRank && r <= 2 * kTMaxRank) {
+        // Two launches of the cluster kernel, each for one half of L_A's rows and the matching
+        // columns of T.  Both write the same codes and scales (the arithmetic is deterministic),
+        // which costs one extra sweep over X but keeps the projection on the tensor cores.
+        const int r1 = r - kTMaxRank;
+        int rc = launch_tma(X, s, LA, M, K, kTMaxRank, Xq, a_scale, T, r, st, &unsupported);
+        if (!unsupported) {
+            if (rc != ASER_OK) return rc;
+            rc = launch_tma(X, s, LA + (size_t)kTMaxRank * K, M, K, r1, Xq, a_scale, T + kTMaxRank, r, st,
+                            &unsupported);
+            // the shape test is the same for both halves, so the second cannot be refused alone
+            if (!unsupported) return rc;
+            return record_cuda_error(cudaErrorUnknown, "quant_act: second half refused");
+        }
+        return launch_large<4>(X, s, LA, M, K, r, Xq, a_scale, T, st);
+    }
+    const int rc = launch_tma(X, s, LA, M, K, r, Xq, a_scale, T, r, st, &unsupported);
     if (!unsupported) return rc;
     if (r <= 64) return launch_large<1>(X, s, LA, M, K, r, Xq, a_scale, T, st);
     if (r <= 128) return launch_large<2>(X, s, LA, M, K, r, Xq, a_scale, T, st);

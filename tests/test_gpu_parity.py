@@ -246,10 +246,11 @@ def test_config4_block_linears_full_size_sampled_rows(aser, name):
     run_path(aser, lay, s, Wq, w_scale, L_A, L_B, "tc", rows=rows, use_dgemm=True)
 
 
-@pytest.mark.parametrize("M,N,r", [(16, 8192, 32), (128, 28672, 256), (1024, 8192, 128), (4096, 8192, 0)])
+@pytest.mark.parametrize("M,N,r", [(16, 8192, 32), (16, 28672, 64), (128, 28672, 256), (1024, 8192, 128), (4096, 8192, 0)])
 def test_config5_sweep_points_sampled_rows(aser, M, N, r):
-    """Points of the 70B-class sweep (K = 8192), including rank 256 (the quantization kernel's
-    mma.sync path) and rank 0 (plain W4A8)."""
+    """Points of the 70B-class sweep (K = 8192): 16 tokens on both few-token paths (streaming
+    kernel up to 64 MB of packed weights, tensor-core kernel above), rank 256 (two launches of the
+    quantization cluster kernel) and rank 0 (plain W4A8)."""
     lay = synth.config5_point(M, N)
     s, Wq, w_scale, L_A, L_B = oracle_layer(lay, r, construct=False)
     if r == 0:

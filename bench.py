@@ -47,6 +47,7 @@ WORKLOADS = {
 # with the kernel as it stands in this tree; the summaries with the commands are under profiles/
 # (<kernel>_<workload>.txt).  Workloads without a capture of the current kernel report null.
 NCU_DRAM_BYTES_PER_LAUNCH = {
+    "c2_decode_m8": 8.71e6,           # linear_decode: mean of two launches, 8.45 and 8.98 MB read, 0 written back
     "c3_prefill_gate_up": 82.04e6,    # 45.4 MB read + 36.7 MB written
 }
 
@@ -376,7 +377,8 @@ def run_ours(args, rank, world, local_rank):
         achieved = ops / (ms_lin * 1e-3) / 1e12
         roof = dict(bound="tensor", achieved=achieved, peak=peak, unit="TOP/s",
                     frac=achieved / peak, traffic=traffic,
-                    peak_source=peaks["source"] + " bf16 burst x2 (int8:bf16 nominal)")
+                    peak_source=peaks["source"] + " bf16 burst x2 (int8:bf16 nominal)",
+                    library_int8_gemm_8192_tops=library_int8_gemm_tops(torch, dev))
     roof.update(kernel=dominant_kernel(M, N, K), us_per_launch=ms_lin * 1e3,
                 algorithmic_bytes=bytes_lin, ops=ops)
 
@@ -537,6 +539,28 @@ def time_point(torch, aser, sets, M, N, K, r, peaks):
                 operand_sets=n)
 
 
+def library_int8_gemm_tops(torch, dev, n=8192, reps=10):
+    """Yardstick only: the vendor library's plain int8 x int8 -> int32 GEMM at n^3 (best of `reps`),
+    printed beside the int8 peak that the fractions use (2 x the measured bf16 figure)."""
+    try:
+        a = torch.randint(-127, 128, (n, n), dtype=torch.int8, device=dev)
+        b = torch.randint(-127, 128, (n, n), dtype=torch.int8, device=dev)
+        for _ in range(3):
+            torch._int_mm(a, b)
+        torch.cuda.synchronize()
+        best = float("inf")
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            torch._int_mm(a, b)
+            e1.record()
+            torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        return 2.0 * n ** 3 / (best * 1e-3) / 1e12
+    except Exception as exc:    # the yardstick is optional; the product path never depends on it
+        return "unavailable: %s" % type(exc).__name__
+
+
 def run_sweep(args, local_rank):
     """`--sweep c4`: the seven linears of a decoder block at 4096 tokens, rank 128, each alone and
     all back to back.  `--sweep c5`: the 70B-class grid (two shapes x five token counts x five
@@ -547,6 +571,7 @@ def run_sweep(args, local_rank):
     dev = torch.device("cuda", local_rank)
     peaks = load_peaks()
     points = []
+    lib_int8 = library_int8_gemm_tops(torch, dev)
     with ClockSampler(local_rank) as clk:
         if args.sweep == "c4":
             M, r = 4096, 128
@@ -592,7 +617,7 @@ def run_sweep(args, local_rank):
         clocks = clk.summary()
     line = dict(sweep=args.sweep, unit_time="us per call, CUDA-graph replay, best of 3",
                 peaks=dict(hbm_gbs=peaks["hbm_gbs"], int8_tops=2.0 * peaks["bf16_tflops"],
-                           source=peaks["source"]),
+                           source=peaks["source"], library_int8_gemm_8192_tops=lib_int8),
                 points=points, clocks=clocks, **summary)
     print(json.dumps(line), flush=True)
 

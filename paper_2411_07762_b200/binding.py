@@ -189,6 +189,24 @@ def linear_w4a8_lr_static(Xq, a_scale, Wk, w_scale, T, L_B, N: int, Y=None, acc_
     return Y
 
 
+def pad_rank(L_A: torch.Tensor, L_B: torch.Tensor, multiple: int = 16):
+    """Factors of a rank that is not a multiple of 16 (a per-layer rank chosen by the paper's
+    singular-value threshold, Sec. 4.1) -> the same factors with zero rows appended to L_A
+    [r,K] and zero columns to L_B [N,r], which adds exact zeros to T L_B^T.  The kernels take
+    ranks in steps of 16 up to 256."""
+    r = L_A.shape[0]
+    if L_B.shape[1] != r:
+        raise ValueError("L_A has %d rows but L_B has %d columns" % (r, L_B.shape[1]))
+    rp = (r + multiple - 1) // multiple * multiple
+    if rp == r:
+        return L_A.contiguous(), L_B.contiguous()
+    A = torch.zeros((rp, L_A.shape[1]), dtype=L_A.dtype, device=L_A.device)
+    B = torch.zeros((L_B.shape[0], rp), dtype=L_B.dtype, device=L_B.device)
+    A[:r] = L_A
+    B[:, :r] = L_B
+    return A, B
+
+
 class AserLinear:
     """Device-resident operands of one ASER-quantized linear layer plus preallocated
     intermediates for up to `max_tokens` tokens.  __call__ runs aser_quant_act followed by

@@ -139,6 +139,25 @@ __device__ __forceinline__ void set_work(Work& w, const Params& p, int tile, int
     w.whole = (kb0 == 0) && (kb1 == p.KB);
 }
 
+// Low-rank chunks inside a tile.  With a one-slot chunk ring (128-token tiles) and several chunks
+// (r > 64), loading, converting and multiplying them one after the other at the END of a tile
+// leaves the integer pipeline idle for a TMA round trip per chunk.  Where the tile is long enough
+// all chunks but the last are therefore worked off in MID-TILE: chunk c is multiplied when stage
+// lr_mma_stage(c) comes up (kLrSpacing stages per chunk, counted back from the end of the tile:
+// a TMA round trip is three to four stages, conversion and MMAs one more) and converted two
+// stages before; the slot is refilled as soon as those MMAs have retired, so the last chunk is
+// in shared memory when the tile ends.  The first chunk can only be loaded once the previous
+// tile's last chunk has been multiplied, i.e. around stage 4, hence the nine stages of head room.
+// All three roles derive the schedule from the same numbers (stages of the work item, chunk
+// count), so they agree without talking to each other.
+constexpr int kLrSpacing = 5;
+__device__ __forceinline__ bool lr_mid_tile(int ring_slots, bool has_lr, int chunks, int nst) {
+    return ring_slots == 1 && has_lr && chunks >= 2 && nst >= 9 + kLrSpacing * (chunks - 1);
+}
+__device__ __forceinline__ int lr_mma_stage(int c, int chunks, int nst) {
+    return nst - (chunks - 1 - c) * kLrSpacing;
+}
+
 // Next work item (the part of one tile inside this CTA's range).
 __device__ __forceinline__ bool next_work(Cursor& c, const Params& p, Work& w) {
     if (c.phase == 0) {
@@ -351,13 +370,22 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             Work w{};
             uint32_t cx = 0, cl = 0;
             bool ok = true;
-            auto issue_lr = [&](int c) {
+            auto load_lr = [&](int c) {
                 const int s = cl % C::NL;
-                if (!mbar_wait(bar(B_EMPTY_LR + s), ((cl / C::NL) & 1) ^ 1, ab)) return false;
                 mbar_arrive_expect_tx(bar(B_FULL_LR + s), C::LbBytes + C::TBytes);
                 tma_load_2d(sbase + C::OffLb + s * C::LbBytes, &map_lb, c * 64, w.nt * 128, bar(B_FULL_LR + s));
                 tma_load_2d(sbase + C::OffT + s * C::TBytes, &map_t, c * 64, w.tt * BT, bar(B_FULL_LR + s));
                 ++cl;
+            };
+            auto issue_lr = [&](int c) {
+                if (!mbar_wait(bar(B_EMPTY_LR + cl % C::NL), ((cl / C::NL) & 1) ^ 1, ab)) return false;
+                load_lr(c);
+                return true;
+            };
+            // the same without waiting: false when the slot is still in use
+            auto try_issue_lr = [&](int c) {
+                if (!mbar_try_wait(bar(B_EMPTY_LR + cl % C::NL), ((cl / C::NL) & 1) ^ 1)) return false;
+                load_lr(c);
                 return true;
             };
             while (ok && next_work(cur, p, w)) {
@@ -370,9 +398,11 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 // first, so they go out four stages before the end of the tile instead.
                 const int nst = (w.kb1 - w.kb0 + KS - 1) / KS;
                 const int lr_at = (C::NL == 1 && nst > 5) ? nst - 4 : 1;
+                const bool mid = lr_mid_tile(C::NL, w.has_lr, lr_chunks, nst);
+                int mid_next = 0;          // mid-tile schedule: next chunk to load
                 int st_idx = 0;
                 for (int kb = w.kb0; kb < w.kb1 && ok; kb += KS, ++st_idx) {
-                    if (st_idx == lr_at)
+                    if (!mid && st_idx == lr_at)
                         for (int c = 0; c < early && ok; ++c) ok = issue_lr(c);
                     if (!ok) break;
                     const int s = cx % C::NX;
@@ -382,8 +412,13 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     mbar_arrive_expect_tx(bar(B_X_FULL + s), C::XBytes);
                     tma_load_3d(sbase + C::OffX + s * C::XBytes, &map_x, 0, w.tt * BT, kb, bar(B_X_FULL + s));
                     ++cx;
+                    // mid-tile schedule: the next chunk goes out as soon as the slot is free; never
+                    // wait here (the activation stages must keep flowing)
+                    if (mid && mid_next < lr_chunks && try_issue_lr(mid_next)) ++mid_next;
                 }
-                if (w.has_lr) {
+                if (mid) {
+                    for (int c = mid_next; c < lr_chunks && ok; ++c) ok = issue_lr(c);
+                } else if (w.has_lr) {
                     if (w.kb1 - w.kb0 <= KS)   // single-stage item: the early chunks are still due
                         for (int c = 0; c < early && ok; ++c) ok = issue_lr(c);
                     for (int c = early; c < lr_chunks && ok; ++c) ok = issue_lr(c);
@@ -415,9 +450,36 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 ok = mbar_wait(bar(B_ACC_EMPTY + buf), (ci >> 1) & 1, ab);
                 if (!ok) break;
                 tc_fence_after();
-                for (int kb = w.kb0; kb < w.kb1 && ok; kb += KS) {
+                const int nst = (w.kb1 - w.kb0 + KS - 1) / KS;
+                const bool mid = issuer == 0 && lr_mid_tile(C::NL, w.has_lr, lr_chunks, nst);
+                int lc = 0;                // low-rank chunks of this item multiplied so far
+                // one chunk: wait for its conversion, multiply, hand the slot back
+                auto lr_chunk = [&](int c) {
+                    const int s = cl % C::NL;
+                    if (!mbar_wait(bar(B_CONV_LR + s), (cl / C::NL) & 1, ab)) return false;
+                    tc_fence_after();
+                    const uint64_t adesc = smem_desc_sw128(sbase + C::OffLb + s * C::LbBytes);
+                    const uint64_t bdesc = smem_desc_sw128(sbase + C::OffT + s * C::TBytes);
+                    int steps = (p.r - c * 64) / 16;
+                    if (steps > 4) steps = 4;
+                    for (int kk = 0; kk < steps; ++kk)
+                        mma_f16_ss(tm_dlr, adesc + 2 * kk, bdesc + 2 * kk, idesc_f16,
+                                   (c != 0 || kk != 0) ? 1u : 0u);
+                    tc_commit(bar(B_EMPTY_LR + s));
+                    ++cl;
+                    return true;
+                };
+                int st_idx = 0;
+                for (int kb = w.kb0; kb < w.kb1 && ok; kb += KS, ++st_idx) {
                     const int nkb = (w.kb1 - kb < KS) ? (w.kb1 - kb) : KS;
                     const int sx = ca % C::NX;   // ca counts stages
+                    if (mid && lc < lr_chunks - 1 && st_idx == lr_mma_stage(lc, lr_chunks, nst)) {
+                        // the epilogue of the previous item has read the low-rank accumulator
+                        if (lc == 0) ok = mbar_wait(bar(B_DLR_EMPTY), (clr_items & 1) ^ 1, ab);
+                        ok = ok && lr_chunk(lc);
+                        if (!ok) break;
+                        ++lc;
+                    }
                     if ((int)(ca & 1u) != issuer) { ++ca; continue; }
                     ok = mbar_wait(bar(B_X_FULL + sx), (ca / C::NX) & 1, ab);
                     if (!ok) break;
@@ -447,22 +509,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     ++ca;
                 }
                 if (ok && w.has_lr && issuer == 0) {
-                    ok = mbar_wait(bar(B_DLR_EMPTY), (clr_items & 1) ^ 1, ab);
-                    for (int c = 0; c < lr_chunks && ok; ++c) {
-                        const int s = cl % C::NL;
-                        ok = mbar_wait(bar(B_CONV_LR + s), (cl / C::NL) & 1, ab);
-                        if (!ok) break;
-                        tc_fence_after();
-                        const uint64_t adesc = smem_desc_sw128(sbase + C::OffLb + s * C::LbBytes);
-                        const uint64_t bdesc = smem_desc_sw128(sbase + C::OffT + s * C::TBytes);
-                        int steps = (p.r - c * 64) / 16;
-                        if (steps > 4) steps = 4;
-                        for (int kk = 0; kk < steps; ++kk)
-                            mma_f16_ss(tm_dlr, adesc + 2 * kk, bdesc + 2 * kk, idesc_f16,
-                                       (c != 0 || kk != 0) ? 1u : 0u);
-                        tc_commit(bar(B_EMPTY_LR + s));
-                        ++cl;
-                    }
+                    if (lc == 0) ok = mbar_wait(bar(B_DLR_EMPTY), (clr_items & 1) ^ 1, ab);
+                    for (int c = lc; c < lr_chunks && ok; ++c) ok = lr_chunk(c);
                     ++clr_items;
                 }
                 if (ok) tc_commit(bar(B_ACC_FULL + buf));
@@ -482,10 +530,42 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         Work w;
         uint32_t cw = 0, cl = 0;
         bool ok = true;
+        // T chunk in slot cl % NL: bf16 -> fp16 in place (same element size, same swizzled position)
+        auto convert_chunk = [&]() {
+            const int s = cl % C::NL;
+            if (!group_mbar_wait(bar(B_FULL_LR + s), (cl / C::NL) & 1, ab, leader, group)) return false;
+            uint8_t* tb = smem + C::OffT + s * C::TBytes;
+            for (int i = t128; i < C::TBytes / 16; i += 128) {
+                uint4 raw = *reinterpret_cast<uint4*>(tb + i * 16);
+                uint32_t in[4] = {raw.x, raw.y, raw.z, raw.w}, out[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    float lo = __uint_as_float(in[e] << 16);
+                    float hi = __uint_as_float(in[e] & 0xFFFF0000u);
+                    __half2 h = __floats2half2_rn(lo, hi);
+                    out[e] = *reinterpret_cast<uint32_t*>(&h);
+                }
+                *reinterpret_cast<uint4*>(tb + i * 16) = make_uint4(out[0], out[1], out[2], out[3]);
+            }
+            fence_proxy_async_smem();
+            group_bar_sync(group);
+            if (leader) mbar_arrive(bar(B_CONV_LR + s));
+            ++cl;
+            return true;
+        };
         while (ok && next_work(cur, p, w)) {
-            for (int kb = w.kb0; kb < w.kb1 && ok; kb += KS) {
+            const int nst = (w.kb1 - w.kb0 + KS - 1) / KS;
+            const bool mid = group == 0 && lr_mid_tile(C::NL, w.has_lr, lr_chunks, nst);
+            int lc = 0;                    // low-rank chunks of this item converted so far
+            int st_idx = 0;
+            for (int kb = w.kb0; kb < w.kb1 && ok; kb += KS, ++st_idx) {
                 const int nkb = (w.kb1 - kb < KS) ? (w.kb1 - kb) : KS;
                 const int sw = cw % C::NW;   // cw counts stages
+                if (mid && lc < lr_chunks - 1 && st_idx == lr_mma_stage(lc, lr_chunks, nst) - 2) {
+                    ok = convert_chunk();
+                    if (!ok) break;
+                    ++lc;
+                }
                 if ((int)(cw & 1u) != group) { ++cw; continue; }
                 ok = group_mbar_wait(bar(B_W_FULL + sw), (cw / C::NW) & 1, ab, leader, group);
                 if (!ok) break;
@@ -528,31 +608,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 if (!ok) break;
                 ++cw;
             }
-            if (ok && w.has_lr && group == 0) {
-                for (int c = 0; c < lr_chunks && ok; ++c) {
-                    const int s = cl % C::NL;
-                    ok = group_mbar_wait(bar(B_FULL_LR + s), (cl / C::NL) & 1, ab, leader, group);
-                    if (!ok) break;
-                    // T chunk: bf16 -> fp16 in place (same element size, same swizzled position)
-                    uint8_t* tb = smem + C::OffT + s * C::TBytes;
-                    for (int i = t128; i < C::TBytes / 16; i += 128) {
-                        uint4 raw = *reinterpret_cast<uint4*>(tb + i * 16);
-                        uint32_t in[4] = {raw.x, raw.y, raw.z, raw.w}, out[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            float lo = __uint_as_float(in[e] << 16);
-                            float hi = __uint_as_float(in[e] & 0xFFFF0000u);
-                            __half2 h = __floats2half2_rn(lo, hi);
-                            out[e] = *reinterpret_cast<uint32_t*>(&h);
-                        }
-                        *reinterpret_cast<uint4*>(tb + i * 16) = make_uint4(out[0], out[1], out[2], out[3]);
-                    }
-                    fence_proxy_async_smem();
-                    group_bar_sync(group);
-                    if (leader) mbar_arrive(bar(B_CONV_LR + s));
-                    ++cl;
-                }
-            }
+            if (ok && w.has_lr && group == 0)
+                for (int c = lc; c < lr_chunks && ok; ++c) ok = convert_chunk();
         }
     } else if (warp < 10 + C::EW) {
         // =================== epilogue warps ===================

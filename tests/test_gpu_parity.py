@@ -257,3 +257,27 @@ def test_config5_sweep_points_sampled_rows(aser, M, N, r):
         L_A = L_B = None
     rows = np.unique(np.array([0, 1, M // 2, M - 2, M - 1]).clip(0, M - 1))
     run_path(aser, lay, s, Wq, w_scale, L_A, L_B, "tc", rows=rows, use_dgemm=True)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("M,N,K,r", [(8, 256, 1024, 40), (200, 384, 2048, 72)])
+def test_rank_not_a_multiple_of_16_is_padded_with_zeros(aser, M, N, K, r):
+    """A per-layer rank from the singular-value threshold (Sec. 4.1) is any integer: pad_rank
+    appends zero rows / columns; the result must match the oracle run on the UNPADDED factors."""
+    lay = synth.make_layer(M, N, K, seed=700 + r, n_cal=8)
+    s, Wq_ref, w_scale_ref, L_A, L_B = oracle_layer(lay, r, construct=False)
+    dLA, dLB = aser.pad_rank(to_dev(L_A), to_dev(L_B))
+    assert dLA.shape[0] % 16 == 0 and dLB.shape[1] == dLA.shape[0]
+    ds = to_dev(s)
+    Wq, wsc = aser.pack_w4(to_dev(lay.W), ds)
+    Wk = aser.repack_w4(Wq)
+    Xq, sc, T = aser.quant_act(to_dev(lay.X), ds, dLA)
+    ws = aser.new_workspace(M, N, K, dLA.shape[0])
+    acc = torch.zeros((M, N), dtype=torch.int32, device="cuda")
+    Y = aser.linear_w4a8_lr(Xq, sc, Wk, wsc, T, dLB, N, ws, acc_debug=acc)
+    aser.check_status(ws)
+    torch.cuda.synchronize()
+    ref = F.forward(lay.X, s, Wq_ref, w_scale_ref, L_A, L_B)
+    assert np.array_equal(acc.cpu().numpy(), ref.acc)
+    assert bool((T[:, r:] == 0).all())
+    assert_rows_close(Y.cpu().numpy(), ref.y)

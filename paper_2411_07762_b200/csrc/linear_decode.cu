@@ -75,23 +75,24 @@ __device__ __forceinline__ void mma_s8_16x8x32(int (&c)[4], uint32_t a0, uint32_
 // NT = number of 8-token groups (1 for M <= 8, 2 for M <= 16).  R = 16-row tiles per warp: a
 // CTA owns 16 R output channels; the activation fragment of a column block is loaded once and
 // used for all R tiles, which is what keeps the L1 traffic (two bytes of activations per byte of
-// packed weights at R = 1, sixteen tokens) below the weight stream's.  Batch column blocks per
-// warp are in flight: Batch * R * 32 bytes of packed weights per thread.
-template <int NT, int R>
+// packed weights at R = 1, sixteen tokens) below the weight stream's.  B column blocks per warp
+// are in flight: B * R * 32 bytes of packed weights per thread (128 bytes at three CTAs per SM,
+// 256 bytes at two).
+template <int NT, int R, int B>
 struct DecCfg {
-    static constexpr int Batch = 4 / R;
+    static constexpr int Batch = B;
     static constexpr int Rows = 16 * R;
     static constexpr int Regs = R * NT * 4;          // accumulator registers per thread
-    static constexpr int MinCtas = (NT * R <= 2) ? 3 : 2;
+    static constexpr int MinCtas = (R * B <= 4) ? 3 : 2;
 };
 
-template <int NT, int R>
-__global__ void __launch_bounds__(kDecThreads, DecCfg<NT, R>::MinCtas)
+template <int NT, int R, int B>
+__global__ void __launch_bounds__(kDecThreads, DecCfg<NT, R, B>::MinCtas)
 linear_decode_kernel(const int8_t* Xq, const float* a_scale, const uint8_t* __restrict__ Wk,
                      const float* __restrict__ w_scale, const __nv_bfloat16* T,
                      const __half* __restrict__ LB, int M, int N, int K, int r,
                      __half* __restrict__ Y, int32_t* __restrict__ acc_debug) {
-    using C = DecCfg<NT, R>;
+    using C = DecCfg<NT, R, B>;
     constexpr int BATCH = C::Batch;
     // partial sums of the eight warps: integer accumulators and fp32 accumulators of the low-rank term
     __shared__ int red[kDecWarps][C::Regs][32];
@@ -272,12 +273,12 @@ linear_decode_kernel(const int8_t* Xq, const float* a_scale, const uint8_t* __re
     }
 }
 
-template <int NT, int R>
+template <int NT, int R, int B>
 int launch_cfg(const int8_t* Xq, const float* a_scale, const uint8_t* Wk, const float* w_scale,
                const __nv_bfloat16* T, const __half* LB, int M, int N, int K, int r, __half* Y,
                int32_t* acc_debug, cudaStream_t st, bool overlap_prev) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((N + DecCfg<NT, R>::Rows - 1) / DecCfg<NT, R>::Rows, 1, 1);
+    cfg.gridDim = dim3((N + DecCfg<NT, R, B>::Rows - 1) / DecCfg<NT, R, B>::Rows, 1, 1);
     cfg.blockDim = dim3(kDecThreads, 1, 1);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = st;
@@ -286,7 +287,7 @@ int launch_cfg(const int8_t* Xq, const float* a_scale, const uint8_t* Wk, const 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = overlap_prev ? 1 : 0;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, linear_decode_kernel<NT, R>, Xq, a_scale, Wk, w_scale, T, LB,
+    cudaError_t e = cudaLaunchKernelEx(&cfg, linear_decode_kernel<NT, R, B>, Xq, a_scale, Wk, w_scale, T, LB,
                                        M, N, K, r, Y, acc_debug);
     if (e != cudaSuccess) return record_cuda_error(e, "linear_decode_kernel");
     return check_launch("linear_decode_kernel");
@@ -305,9 +306,14 @@ int launch_nt(const int8_t* Xq, const float* a_scale, const uint8_t* Wk, const f
         if (e == cudaSuccess) e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) { num_sms = 0; return record_cuda_error(e, "query SM count"); }
     }
-    if (N >= 32 * 3 * num_sms / 2)
-        return launch_cfg<NT, 2>(Xq, a_scale, Wk, w_scale, T, LB, M, N, K, r, Y, acc_debug, st, overlap_prev);
-    return launch_cfg<NT, 1>(Xq, a_scale, Wk, w_scale, T, LB, M, N, K, r, Y, acc_debug, st, overlap_prev);
+    if (N >= 32 * 3 * num_sms / 2) {
+        // two CTAs per SM with twice the bytes in flight per thread where all CTAs are resident
+        // at once that way; otherwise three lighter CTAs per SM
+        if ((N + 31) / 32 <= 2 * num_sms)
+            return launch_cfg<NT, 2, 4>(Xq, a_scale, Wk, w_scale, T, LB, M, N, K, r, Y, acc_debug, st, overlap_prev);
+        return launch_cfg<NT, 2, 2>(Xq, a_scale, Wk, w_scale, T, LB, M, N, K, r, Y, acc_debug, st, overlap_prev);
+    }
+    return launch_cfg<NT, 1, 4>(Xq, a_scale, Wk, w_scale, T, LB, M, N, K, r, Y, acc_debug, st, overlap_prev);
 }
 
 }  // namespace

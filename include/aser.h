@@ -84,6 +84,19 @@ int aser_quant_act(const void* X_f16, const float* s, const void* LA_f16,
                    int8_t* Xq, float* a_scale, void* T_bf16, void* stream);
 
 /*
+ * aser_quant_act_bits -- aser_quant_act with activation codes of act_bits bits (2..8), the
+ * paper's W4A6 setting being act_bits = 6 (Sec. 5.2, the W4A6 rows of the main results):
+ *   qmax = 2^(act_bits-1) - 1;  a_scale[m] = max_k |x~| / qmax;
+ *   Xq[m,k] = clamp(rne(x~ / a_scale[m]), -qmax, qmax)
+ * The codes are stored in the same int8 array, so the linear kernels need no change: the scale
+ * carries the coarser step.  act_bits = 8 is aser_quant_act.  Everything else (arguments,
+ * layouts, T, bit-exactness of Xq and a_scale) as there; other widths return ASER_ERR_SHAPE.
+ */
+int aser_quant_act_bits(const void* X_f16, const float* s, const void* LA_f16,
+                        int M, int K, int r, int act_bits,
+                        int8_t* Xq, float* a_scale, void* T_bf16, void* stream);
+
+/*
  * aser_linear_w4a8_lr -- integer GEMM, dequantisation and up projection
  * (Sec. 4.2: W_q X + L_A L_B X in the paper's letters):
  *   acc[m,n] = sum_k Xq[m,k] * q[n,k]                               (exact int32)

@@ -83,12 +83,15 @@ void aser_oracle_smooth_act(const uint16_t* X, const float* s, long M, long K, f
 }
 
 /* ---------------------------------------------------------------------------
- * Per-token symmetric int8 round-to-nearest (Sec. 5.1 "per-token for
- * activations").  a_scale[m] = max_k |x~| / 127; code = rne(x~ / a_scale)
- * clamped to [-127, 127].  An all-zero token gets scale 0 and codes 0.
+ * Per-token symmetric round-to-nearest of the activations to `bits`-bit codes
+ * (Sec. 5.1 "per-token for activations"; 8 bits in the W4A8 setting, 6 in the
+ * W4A6 setting of Sec. 5.2).  qmax = 2^(bits-1) - 1; a_scale[m] = max_k |x~| / qmax;
+ * code = rne(x~ / a_scale) clamped to [-qmax, qmax], stored in an int8.  An
+ * all-zero token gets scale 0 and codes 0.
  * ------------------------------------------------------------------------- */
-void aser_oracle_quant_act(const float* xs, long M, long K, int8_t* Xq, float* a_scale)
+void aser_oracle_quant_act_bits(const float* xs, long M, long K, int bits, int8_t* Xq, float* a_scale)
 {
+    const float qmax = (float)((1 << (bits - 1)) - 1);
 #pragma omp parallel for num_threads(g_threads) schedule(static)
     for (long m = 0; m < M; ++m) {
         float amax = 0.0f;
@@ -96,18 +99,24 @@ void aser_oracle_quant_act(const float* xs, long M, long K, int8_t* Xq, float* a
             float a = fabsf(xs[m * K + k]);
             if (a > amax) amax = a;
         }
-        float sc = amax / 127.0f;
+        float sc = amax / qmax;
         a_scale[m] = sc;
         for (long k = 0; k < K; ++k) {
             float c = 0.0f;
             if (amax > 0.0f) {
                 c = rintf(xs[m * K + k] / sc);
-                if (c > 127.0f) c = 127.0f;
-                if (c < -127.0f) c = -127.0f;
+                if (c > qmax) c = qmax;
+                if (c < -qmax) c = -qmax;
             }
             Xq[m * K + k] = (int8_t)c;
         }
     }
+}
+
+/* The W4A8 setting: 8-bit codes, a_scale[m] = max_k |x~| / 127, codes in [-127, 127]. */
+void aser_oracle_quant_act(const float* xs, long M, long K, int8_t* Xq, float* a_scale)
+{
+    aser_oracle_quant_act_bits(xs, M, K, 8, Xq, a_scale);
 }
 
 /* ---------------------------------------------------------------------------

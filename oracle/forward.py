@@ -23,6 +23,7 @@ _lib.aser_oracle_get_threads.restype = C.c_int
 _lib.aser_oracle_max_threads.restype = C.c_int
 _lib.aser_oracle_smooth_act.argtypes = [_P, _P, _L, _L, _P]
 _lib.aser_oracle_quant_act.argtypes = [_P, _L, _L, _P, _P]
+_lib.aser_oracle_quant_act_bits.argtypes = [_P, _L, _L, C.c_int, _P, _P]
 _lib.aser_oracle_quant_w4.argtypes = [_P, _P, _L, _L, _P, _P, _P]
 _lib.aser_oracle_pack_w4.argtypes = [_P, _L, _L, _P]
 _lib.aser_oracle_unpack_w4.argtypes = [_P, _L, _L, _P]
@@ -70,13 +71,18 @@ def smooth_act(X: np.ndarray, s: np.ndarray | None) -> np.ndarray:
     return xs
 
 
-def quant_act(xs: np.ndarray) -> tuple[np.ndarray, np.ndarray]:
-    """Per-token int8 codes and fp32 scales of the smoothed activation."""
+def quant_act(xs: np.ndarray, act_bits: int = 8) -> tuple[np.ndarray, np.ndarray]:
+    """Per-token codes (act_bits wide, int8 container) and fp32 scales of the smoothed activation."""
     xs = _c(xs, np.float32)
     M, K = xs.shape
     Xq = np.empty((M, K), np.int8)
     a_scale = np.empty(M, np.float32)
-    _lib.aser_oracle_quant_act(_ptr(xs), M, K, _ptr(Xq), _ptr(a_scale))
+    if act_bits == 8:
+        _lib.aser_oracle_quant_act(_ptr(xs), M, K, _ptr(Xq), _ptr(a_scale))
+    else:
+        if not 2 <= act_bits <= 8:
+            raise ValueError("act_bits must be 2..8")
+        _lib.aser_oracle_quant_act_bits(_ptr(xs), M, K, int(act_bits), _ptr(Xq), _ptr(a_scale))
     return Xq, a_scale
 
 
@@ -195,16 +201,16 @@ class ForwardResult:
 
 
 def forward(X, s, Wq_packed, w_scale, L_A=None, L_B=None, rows=None,
-            use_dgemm: bool = False) -> ForwardResult:
+            use_dgemm: bool = False, act_bits: int = 8) -> ForwardResult:
     """Inference pass of one ASER linear (Sec. 4.2): smooth, quantize per token,
     integer product with the int4 weights, dequantize, add L_B (L_A x~).
 
     `rows` restricts the expensive products to a subset of tokens (quantization
     still covers every token).  `use_dgemm` swaps the triple loop for the exact
-    fp64 library product on large shapes.
+    fp64 library product on large shapes.  `act_bits` = 6 is the W4A6 setting.
     """
     xs = smooth_act(X, s)
-    Xq, a_scale = quant_act(xs)
+    Xq, a_scale = quant_act(xs, act_bits)
     q = unpack_w4(Wq_packed)
     acc = (int_matmul_dgemm if use_dgemm else int_matmul)(Xq, q, rows)
     T = None

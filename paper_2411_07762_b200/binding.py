@@ -11,7 +11,7 @@ lib_path = os.path.join(_HERE, "libaser.so")
 
 EXPORTED_SYMBOLS = (
     "aser_pack_w4", "aser_repacked_bytes", "aser_repack_w4", "aser_unrepack_w4",
-    "aser_quant_act", "aser_linear_w4a8_lr", "aser_linear_w4a8", "aser_linear_w4a8_lr_simt", "aser_linear_w4a8_lr_static",
+    "aser_quant_act", "aser_quant_act_bits", "aser_linear_w4a8_lr", "aser_linear_w4a8", "aser_linear_w4a8_lr_simt", "aser_linear_w4a8_lr_static",
     "aser_workspace_bytes", "aser_workspace_init", "aser_check_status", "aser_forward",
     "aser_forward_host",
     "aser_last_error", "aser_version",
@@ -30,6 +30,7 @@ lib.aser_repacked_bytes.restype = _Z
 lib.aser_repack_w4.argtypes = [_P, _I, _I, _P, _P]
 lib.aser_unrepack_w4.argtypes = [_P, _I, _I, _P, _P]
 lib.aser_quant_act.argtypes = [_P, _P, _P, _I, _I, _I, _P, _P, _P, _P]
+lib.aser_quant_act_bits.argtypes = [_P, _P, _P, _I, _I, _I, _I, _P, _P, _P, _P]
 lib.aser_linear_w4a8_lr.argtypes = [_P, _P, _P, _P, _P, _P, _I, _I, _I, _I, _P, _P, _P, _Z, _P]
 lib.aser_linear_w4a8.argtypes = [_P, _P, _P, _P, _I, _I, _I, _P, _P, _P, _Z, _P]
 lib.aser_linear_w4a8_lr_simt.argtypes = [_P, _P, _P, _P, _P, _P, _I, _I, _I, _I, _P, _P, _P]
@@ -108,8 +109,9 @@ def unrepack_w4(Wk: torch.Tensor, N: int, K: int) -> torch.Tensor:
 
 
 def quant_act(X: torch.Tensor, s: torch.Tensor | None, L_A: torch.Tensor | None,
-              out=None):
-    """X fp16 [M,K] -> (Xq int8 [M,K], a_scale fp32 [M], T bf16 [M,r])."""
+              out=None, act_bits: int = 8):
+    """X fp16 [M,K] -> (Xq int8 [M,K], a_scale fp32 [M], T bf16 [M,r]).  act_bits != 8 goes
+    through aser_quant_act_bits (codes of that width in the int8 container)."""
     _dev(X, torch.float16, "X")
     M, K = X.shape
     r = 0 if L_A is None else L_A.shape[0]
@@ -119,6 +121,11 @@ def quant_act(X: torch.Tensor, s: torch.Tensor | None, L_A: torch.Tensor | None,
         T = torch.empty((M, r), dtype=torch.bfloat16, device=X.device)
     else:
         Xq, a_scale, T = out
+    if act_bits != 8:
+        _chk(lib.aser_quant_act_bits(_ptr(X), _ptr(s), _ptr(L_A) if r else None, M, K, r, act_bits,
+                                     _ptr(Xq), _ptr(a_scale), _ptr(T) if r else None, _stream()),
+             "aser_quant_act_bits")
+        return Xq, a_scale, T
     _chk(lib.aser_quant_act(_ptr(X), _ptr(s), _ptr(L_A) if r else None, M, K, r, _ptr(Xq),
                             _ptr(a_scale), _ptr(T) if r else None, _stream()), "aser_quant_act")
     return Xq, a_scale, T

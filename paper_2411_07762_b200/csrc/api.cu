@@ -155,7 +155,13 @@ int aser_unrepack_w4(const void* Wk, int N, int K, uint8_t* Wq, void* stream) {
 
 int aser_quant_act(const void* X_f16, const float* s, const void* LA_f16, int M, int K, int r,
                    int8_t* Xq, float* a_scale, void* T_bf16, void* stream) {
+    return aser_quant_act_bits(X_f16, s, LA_f16, M, K, r, 8, Xq, a_scale, T_bf16, stream);
+}
+
+int aser_quant_act_bits(const void* X_f16, const float* s, const void* LA_f16, int M, int K, int r,
+                        int act_bits, int8_t* Xq, float* a_scale, void* T_bf16, void* stream) {
     if (!shape_ok(M, 0, K, r)) return fail(ASER_ERR_SHAPE, "unsupported M, K or r");
+    if (act_bits < 2 || act_bits > 8) return fail(ASER_ERR_SHAPE, "act_bits must be 2..8");
     if (M == 0) return ASER_OK;
     ASER_REQUIRE_PTR(X_f16);
     ASER_OPTIONAL_PTR(s);
@@ -169,7 +175,7 @@ int aser_quant_act(const void* X_f16, const float* s, const void* LA_f16, int M,
     if (rc != ASER_OK) return rc;
     return launch_quant_act(static_cast<const __half*>(X_f16), s, static_cast<const __half*>(LA_f16),
                             M, K, r, Xq, a_scale, static_cast<__nv_bfloat16*>(T_bf16),
-                            static_cast<cudaStream_t>(stream));
+                            static_cast<cudaStream_t>(stream), act_bits);
 }
 
 int aser_linear_w4a8_lr(const int8_t* Xq, const float* a_scale, const void* Wk,

@@ -24,8 +24,9 @@ inline bool misaligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p)
 int launch_pack_w4(const __half* W, const float* s, int N, int K, uint8_t* Wq, float* w_scale,
                    cudaStream_t st);
 int launch_repack_w4(const uint8_t* Wq, int N, int K, uint8_t* Wk, bool inverse, cudaStream_t st);
+// act_bits: width of the symmetric activation codes (2..8); they are stored in int8 either way.
 int launch_quant_act(const __half* X, const float* s, const __half* LA, int M, int K, int r,
-                     int8_t* Xq, float* a_scale, __nv_bfloat16* T, cudaStream_t st);
+                     int8_t* Xq, float* a_scale, __nv_bfloat16* T, cudaStream_t st, int act_bits = 8);
 int launch_linear_simt(const int8_t* Xq, const float* a_scale, const uint8_t* Wq,
                        const float* w_scale, const __nv_bfloat16* T, const __half* LB,
                        int M, int N, int K, int r, __half* Y, int32_t* acc_debug, cudaStream_t st);

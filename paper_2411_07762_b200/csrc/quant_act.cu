@@ -57,7 +57,7 @@ __device__ __forceinline__ void smooth8(const RawChunk& rc, float (&v)[8]) {
 // differs from the rounded quotient by less than 4 * 2^-24 * 127 < 3.1e-5: whenever that product
 // is at least 1e-4 away from every half-integer, both round to the same integer and the
 // multiplication stands in for the division.  Only the rare near-ties take the real division.
-__device__ __forceinline__ uint2 quant8(const float (&v)[8], float sc, bool nonzero) {
+__device__ __forceinline__ uint2 quant8(const float (&v)[8], float sc, bool nonzero, float qmax) {
     uint32_t w[2] = {0, 0};
     const float rcp = nonzero ? __frcp_rn(sc) : 0.f;
 #pragma unroll
@@ -66,8 +66,8 @@ __device__ __forceinline__ uint2 quant8(const float (&v)[8], float sc, bool nonz
         if (nonzero) {
             const float t = v[i] * rcp;
             const float fr = fabsf(t) - floorf(fabsf(t));          // fractional part in [0, 1)
-            if (fabsf(fr - 0.5f) >= 1e-4f && fabsf(t) < 1e6f) q = rne_clamp(t, -127.f, 127.f);
-            else q = rne_clamp(__fdiv_rn(v[i], sc), -127.f, 127.f);
+            if (fabsf(fr - 0.5f) >= 1e-4f && fabsf(t) < 1e6f) q = rne_clamp(t, -qmax, qmax);
+            else q = rne_clamp(__fdiv_rn(v[i], sc), -qmax, qmax);
         }
         w[i >> 2] |= (uint32_t)(q & 0xFF) << (8 * (i & 3));
     }
@@ -87,7 +87,7 @@ __global__ void __launch_bounds__(kSmallThreads)
 quant_act_small_kernel(const __half* __restrict__ X, const float* __restrict__ s,
                        const __half* __restrict__ LA, int M, int K, int r,
                        int8_t* __restrict__ Xq, float* __restrict__ a_scale,
-                       __nv_bfloat16* __restrict__ T) {
+                       __nv_bfloat16* __restrict__ T, float qmax) {
     extern __shared__ __align__(16) float xs[];
     grid_dep_launch();      // a dependent linear kernel may start streaming its weights
     __shared__ float red[kRowsPerCta][kSmallThreads / 32];
@@ -113,14 +113,14 @@ quant_act_small_kernel(const __half* __restrict__ X, const float* __restrict__ s
         amax = red[0][0];
 #pragma unroll
         for (int i = 1; i < kSmallThreads / 32; ++i) amax = fmaxf(amax, red[0][i]);
-        const float sc = __fdiv_rn(amax, 127.0f);
+        const float sc = __fdiv_rn(amax, qmax);
         if (threadIdx.x == 0) a_scale[m] = sc;
         int8_t* out = Xq + (size_t)m * K;
         for (int c = threadIdx.x; c < chunks; c += kSmallThreads) {
             float v[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) v[i] = xs[c * 8 + i];
-            *reinterpret_cast<uint2*>(out + c * 8) = quant8(v, sc, amax > 0.f);
+            *reinterpret_cast<uint2*>(out + c * 8) = quant8(v, sc, amax > 0.f, qmax);
         }
         return;
     }
@@ -208,7 +208,7 @@ __global__ void __launch_bounds__(kLargeThreads)
 quant_act_large_kernel(const __half* __restrict__ X, const float* __restrict__ s,
                        const __half* __restrict__ LA, int M, int K, int r,
                        int8_t* __restrict__ Xq, float* __restrict__ a_scale,
-                       __nv_bfloat16* __restrict__ T) {
+                       __nv_bfloat16* __restrict__ T, float qmax) {
     extern __shared__ __align__(16) uint8_t smem[];
     grid_dep_launch();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -295,7 +295,7 @@ quant_act_large_kernel(const __half* __restrict__ X, const float* __restrict__ s
     // ---- per-token scale: the 16 threads of a row are 16 consecutive lanes ----
 #pragma unroll
     for (int o = 8; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-    const float sc = __fdiv_rn(amax, 127.0f);
+    const float sc = __fdiv_rn(amax, qmax);
     if (tcol == 0 && row_ok) a_scale[m] = sc;
 
     // ---- T tile (fp32 accumulators -> bf16) ----
@@ -325,7 +325,7 @@ quant_act_large_kernel(const __half* __restrict__ X, const float* __restrict__ s
         if (c + 1 < nch) rc = load_raw(xrow, s, (c + 1) * kChunkK + tcol * 8, true);
         float v[8];
         smooth8(cur, v);
-        *reinterpret_cast<uint2*>(out + c * kChunkK + tcol * 8) = quant8(v, sc, amax > 0.f);
+        *reinterpret_cast<uint2*>(out + c * kChunkK + tcol * 8) = quant8(v, sc, amax > 0.f, qmax);
     }
 }
 
@@ -531,12 +531,12 @@ __device__ __forceinline__ uint4 pack8_half(const float (&v)[8]) {
 
 // Exact codes for eight values (the definition: IEEE quotient, round half to even, clamp).
 __device__ __noinline__ uint2 quant8_exact(float v0, float v1, float v2, float v3, float v4, float v5,
-                                           float v6, float v7, float sc) {
+                                           float v6, float v7, float sc, float qmax) {
     const float v[8] = {v0, v1, v2, v3, v4, v5, v6, v7};
     uint32_t w[2] = {0, 0};
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        const int q = rne_clamp(__fdiv_rn(v[i], sc), -127.f, 127.f);
+        const int q = rne_clamp(__fdiv_rn(v[i], sc), -qmax, qmax);
         w[i >> 2] |= (uint32_t)(q & 0xFF) << (8 * (i & 3));
     }
     return make_uint2(w[0], w[1]);
@@ -544,7 +544,7 @@ __device__ __noinline__ uint2 quant8_exact(float v0, float v1, float v2, float v
 // Same codes as quant8 for sc > 0, on packed fp32 pairs: t = x~ * (1 / sc), rounded by adding
 // 1.5 * 2^23 (the low byte of the sum is the code); the distance of t to that integer tells the
 // near-ties, and a group with one takes the exact path as a whole.
-__device__ __forceinline__ uint2 quant8_pairs(const float (&v)[8], float sc, float rcp) {
+__device__ __forceinline__ uint2 quant8_pairs(const float (&v)[8], float sc, float rcp, float qmax) {
     const float kMagic = 12582912.0f;
     const float2 r2 = make_float2(rcp, rcp), m2 = make_float2(kMagic, kMagic);
     const float2 nm2 = make_float2(-kMagic, -kMagic), neg1 = make_float2(-1.f, -1.f);
@@ -560,7 +560,7 @@ __device__ __forceinline__ uint2 quant8_pairs(const float (&v)[8], float sc, flo
         q[2 * i + 1] = __float_as_uint(u.y);
         far = fmaxf(far, fmaxf(fabsf(d.x), fabsf(d.y)));
     }
-    if (far > 0.4999f) return quant8_exact(v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7], sc);
+    if (far > 0.4999f) return quant8_exact(v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7], sc, qmax);
     const uint32_t a01 = __byte_perm(q[0], q[1], 0x0040), a23 = __byte_perm(q[2], q[3], 0x0040);
     const uint32_t a45 = __byte_perm(q[4], q[5], 0x0040), a67 = __byte_perm(q[6], q[7], 0x0040);
     return make_uint2(__byte_perm(a01, a23, 0x5410), __byte_perm(a45, a67, 0x5410));
@@ -575,7 +575,7 @@ __global__ void __launch_bounds__(kTThreads, 1)
 quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_la,
                      const __grid_constant__ CUtensorMap map_q, const float* __restrict__ s,
                      int M, int K, int Kc, int r, int CK, float* __restrict__ a_scale,
-                     __nv_bfloat16* __restrict__ T, int ldt) {
+                     __nv_bfloat16* __restrict__ T, int ldt, float qmax) {
     extern __shared__ uint8_t smem_raw[];
     grid_dep_launch();      // a dependent linear kernel may start streaming its weights
     const uint32_t sraw = smem_u32(smem_raw);
@@ -874,12 +874,12 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 a = fmaxf(a, amax_slots[qq * kTTok + row]);
                 b = fmaxf(b, amax_slots[qq * kTTok + row + 32]);
             }
-            sc0 = __fdiv_rn(a, 127.0f);
-            sc1 = __fdiv_rn(b, 127.0f);
+            sc0 = __fdiv_rn(a, qmax);
+            sc1 = __fdiv_rn(b, qmax);
         } else {
             named_bar_sync(1, kTConsumers);
-            sc0 = __fdiv_rn(amax_stage[row], 127.0f);
-            sc1 = __fdiv_rn(amax_stage[row + 32], 127.0f);
+            sc0 = __fdiv_rn(amax_stage[row], qmax);
+            sc1 = __fdiv_rn(amax_stage[row + 32], qmax);
         }
         if (warp == 0) {
             if ((int)rank == row / rows_owned && m0 + row < M) a_scale[m0 + row] = sc0;
@@ -916,10 +916,10 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             // before anything used their results, let the next TMA write overtake them.
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_free2(st));
-            const uint2 lo0 = quant8_pairs(f0, sc0, rcp0);
-            const uint2 hi0 = quant8_pairs(f1, sc0, rcp0);
-            const uint2 lo1 = quant8_pairs(g0, sc1, rcp1);
-            const uint2 hi1 = quant8_pairs(g1, sc1, rcp1);
+            const uint2 lo0 = quant8_pairs(f0, sc0, rcp0, qmax);
+            const uint2 hi0 = quant8_pairs(f1, sc0, rcp0, qmax);
+            const uint2 lo1 = quant8_pairs(g0, sc1, rcp1, qmax);
+            const uint2 hi1 = quant8_pairs(g1, sc1, rcp1, qmax);
             if (jj >= kTOut) {      // the store that last read this tile is done with it
                 ok = qa_warp_wait(bar_out_free(o), (uint32_t)(jj / kTOut - 1) & 1u, abort_flag, lane);
                 if (!ok) break;
@@ -1034,7 +1034,8 @@ int pick_tma_cluster(int M, int K, int r, int max_ck) {
 }
 
 int launch_tma(const __half* X, const float* s, const __half* LA, int M, int K, int r,
-               int8_t* Xq, float* a_scale, __nv_bfloat16* T, int ldt, cudaStream_t st, bool* unsupported) {
+               int8_t* Xq, float* a_scale, __nv_bfloat16* T, int ldt, float qmax, cudaStream_t st,
+               bool* unsupported) {
     *unsupported = false;
     static int max_ck = 0;      // 16 where the device allows clusters beyond the portable 8
     if (max_ck == 0) {
@@ -1075,14 +1076,14 @@ int launch_tma(const __half* X, const float* s, const __half* LA, int M, int K, 
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, quant_act_tma_kernel, mx, mla, mq, s, M, K, kc, r, ck, a_scale, T, ldt);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, quant_act_tma_kernel, mx, mla, mq, s, M, K, kc, r, ck, a_scale, T, ldt, qmax);
     if (e != cudaSuccess) return record_cuda_error(e, "quant_act_tma_kernel");
     return check_launch("quant_act_tma_kernel");
 }
 
 template <int MAXT>
 int launch_large(const __half* X, const float* s, const __half* LA, int M, int K, int r,
-                 int8_t* Xq, float* a_scale, __nv_bfloat16* T, cudaStream_t st) {
+                 int8_t* Xq, float* a_scale, __nv_bfloat16* T, float qmax, cudaStream_t st) {
     size_t smem = 2 * (size_t)(kTileM + r) * kRowBytes;
     static size_t configured = 0;   // largest dynamic shared memory size opted into so far
     if (smem > configured) {
@@ -1092,14 +1093,16 @@ int launch_large(const __half* X, const float* s, const __half* LA, int M, int K
         configured = smem;
     }
     int grid = (M + kTileM - 1) / kTileM;
-    quant_act_large_kernel<MAXT><<<grid, kLargeThreads, smem, st>>>(X, s, LA, M, K, r, Xq, a_scale, T);
+    quant_act_large_kernel<MAXT><<<grid, kLargeThreads, smem, st>>>(X, s, LA, M, K, r, Xq, a_scale, T, qmax);
     return check_launch("quant_act_large_kernel");
 }
 
 }  // namespace
 
 int launch_quant_act(const __half* X, const float* s, const __half* LA, int M, int K, int r,
-                     int8_t* Xq, float* a_scale, __nv_bfloat16* T, cudaStream_t st) {
+                     int8_t* Xq, float* a_scale, __nv_bfloat16* T, cudaStream_t st, int act_bits) {
+    // symmetric codes of act_bits bits in the int8 container: +-127 for 8 bits, +-31 for 6
+    const float qmax = (float)((1 << (act_bits - 1)) - 1);
     if (M == 0) return ASER_OK;
     if (M <= 32) {
         size_t smem = (size_t)K * sizeof(float);
@@ -1111,7 +1114,7 @@ int launch_quant_act(const __half* X, const float* s, const __half* LA, int M, i
             configured = smem;
         }
         dim3 grid(1 + (r + kRowsPerCta - 1) / kRowsPerCta, M);
-        quant_act_small_kernel<<<grid, kSmallThreads, smem, st>>>(X, s, LA, M, K, r, Xq, a_scale, T);
+        quant_act_small_kernel<<<grid, kSmallThreads, smem, st>>>(X, s, LA, M, K, r, Xq, a_scale, T, qmax);
         return check_launch("quant_act_small_kernel");
     }
     bool unsupported = false;
@@ -1120,22 +1123,22 @@ int launch_quant_act(const __half* X, const float* s, const __half* LA, int M, i
         // columns of T.  Both write the same codes and scales (the arithmetic is deterministic),
         // which costs one extra sweep over X but keeps the projection on the tensor cores.
         const int r1 = r - kTMaxRank;
-        int rc = launch_tma(X, s, LA, M, K, kTMaxRank, Xq, a_scale, T, r, st, &unsupported);
+        int rc = launch_tma(X, s, LA, M, K, kTMaxRank, Xq, a_scale, T, r, qmax, st, &unsupported);
         if (!unsupported) {
             if (rc != ASER_OK) return rc;
-            rc = launch_tma(X, s, LA + (size_t)kTMaxRank * K, M, K, r1, Xq, a_scale, T + kTMaxRank, r, st,
+            rc = launch_tma(X, s, LA + (size_t)kTMaxRank * K, M, K, r1, Xq, a_scale, T + kTMaxRank, r, qmax, st,
                             &unsupported);
             // the shape test is the same for both halves, so the second cannot be refused alone
             if (!unsupported) return rc;
             return record_cuda_error(cudaErrorUnknown, "quant_act: second half refused");
         }
-        return launch_large<4>(X, s, LA, M, K, r, Xq, a_scale, T, st);
+        return launch_large<4>(X, s, LA, M, K, r, Xq, a_scale, T, qmax, st);
     }
-    const int rc = launch_tma(X, s, LA, M, K, r, Xq, a_scale, T, r, st, &unsupported);
+    const int rc = launch_tma(X, s, LA, M, K, r, Xq, a_scale, T, r, qmax, st, &unsupported);
     if (!unsupported) return rc;
-    if (r <= 64) return launch_large<1>(X, s, LA, M, K, r, Xq, a_scale, T, st);
-    if (r <= 128) return launch_large<2>(X, s, LA, M, K, r, Xq, a_scale, T, st);
-    return launch_large<4>(X, s, LA, M, K, r, Xq, a_scale, T, st);
+    if (r <= 64) return launch_large<1>(X, s, LA, M, K, r, Xq, a_scale, T, qmax, st);
+    if (r <= 128) return launch_large<2>(X, s, LA, M, K, r, Xq, a_scale, T, qmax, st);
+    return launch_large<4>(X, s, LA, M, K, r, Xq, a_scale, T, qmax, st);
 }
 
 }  // namespace aser

@@ -82,6 +82,67 @@ def test_int8_negative_extreme_not_minus_128():
 
 
 # ---------------------------------------------------------------------------
+# 6-bit activation codes (the W4A6 setting, Sec. 5.2)
+# ---------------------------------------------------------------------------
+
+def test_6bit_codes_by_hand():
+    # absmax 31 -> scale exactly 1 -> codes are rne(x), half to even
+    row = np.array([31.0, 0.5, 1.5, 2.5, -0.5, -1.5, -2.5, 3.5, 30.5, -30.5], np.float32)[None]
+    Xq, sc = F.quant_act(row, act_bits=6)
+    assert sc[0] == np.float32(1.0)
+    assert Xq[0].tolist() == [31, 0, 2, 2, 0, -2, -2, 4, 30, -30]
+    # the scale is one fp32 division by 31; the negative extreme maps to -31, never -32
+    row = np.array([[-5.0, 1.0, 0.1]], np.float32)
+    Xq, sc = F.quant_act(row, act_bits=6)
+    assert sc[0] == np.float32(5.0) / np.float32(31.0)
+    assert Xq[0].tolist() == [-31, 6, 1]     # 1/(5/31) = 6.2 -> 6, 0.1/(5/31) = 0.62 -> 1
+
+
+def test_6bit_range_error_bound_and_8bit_unchanged():
+    rng = np.random.default_rng(6)
+    xs = rng.standard_normal((4, 300)).astype(np.float32) * 3
+    xs[2] = 0.0
+    Xq, sc = F.quant_act(xs, act_bits=6)
+    assert sc[2] == 0.0 and not Xq[2].any()
+    assert Xq.min() >= -31 and Xq.max() <= 31
+    for m in (0, 1, 3):
+        k = np.argmax(np.abs(xs[m]))
+        assert abs(int(Xq[m, k])) == 31
+        err = np.abs(xs[m].astype(np.float64) - Xq[m].astype(np.float64) * float(sc[m]))
+        assert err.max() <= 0.5 * float(sc[m]) * (1 + 1e-6)
+    # 8 bits through the general routine is the W4A8 quantizer bit for bit
+    Xq8, sc8 = F.quant_act(xs)
+    Xq8b = np.empty_like(Xq8)
+    sc8b = np.empty_like(sc8)
+    F._lib.aser_oracle_quant_act_bits(F._ptr(xs), xs.shape[0], xs.shape[1], 8, F._ptr(Xq8b), F._ptr(sc8b))
+    assert np.array_equal(Xq8, Xq8b) and np.array_equal(sc8.view(np.uint32), sc8b.view(np.uint32))
+    # coarser codes, larger error: the 6-bit step is 127/31 of the 8-bit one
+    assert np.allclose(sc[[0, 1, 3]] / sc8[[0, 1, 3]], 127.0 / 31.0, rtol=1e-6)
+
+
+def test_6bit_forward_is_the_same_formula_with_coarser_codes():
+    rng = np.random.default_rng(7)
+    M, N, K = 3, 8, 64
+    X = rng.standard_normal((M, K)).astype(np.float16)
+    W = (rng.standard_normal((N, K)) * 0.05).astype(np.float16)
+    q, w_scale = F.quant_w4(W, None)
+    out = F.forward(X, None, F.pack_w4(q), w_scale, act_bits=6)
+    xq, sc = F.quant_act(X.astype(np.float32), act_bits=6)
+    brute = np.zeros((M, N))
+    for m in range(M):
+        for n in range(N):
+            acc = sum(int(xq[m, k]) * int(q[n, k]) for k in range(K))
+            brute[m, n] = acc * float(sc[m]) * float(w_scale[n])
+    assert np.allclose(out.y, brute, rtol=1e-12, atol=1e-12)
+    # against the product with the SAME int4 weights (so that only the activation codes differ)
+    # the 6-bit pass is the coarser approximation, by about the ratio of the steps
+    ref = X.astype(np.float64) @ (q.astype(np.float64) * w_scale.astype(np.float64)[:, None]).T
+    out8 = F.forward(X, None, F.pack_w4(q), w_scale)
+    e6, e8 = np.linalg.norm(out.y - ref), np.linalg.norm(out8.y - ref)
+    assert 2.0 * e8 < e6 < 8.0 * e8
+
+
+# ---------------------------------------------------------------------------
 # int4 per-output-channel quantizer
 # ---------------------------------------------------------------------------
 

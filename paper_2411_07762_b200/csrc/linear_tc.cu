@@ -244,7 +244,9 @@ __device__ __forceinline__ bool group_mbar_wait(uint32_t bar, uint32_t parity, c
 // ---------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------
-template <int BT>
+// MID: the mid-tile schedule for the low-rank chunks is compiled in (only useful, and only
+// instantiated, for 128-token tiles with r > 64; the other variants keep their loops free of it).
+template <int BT, bool MID>
 __global__ void __launch_bounds__(Cfg<BT>::Threads, 1)
 linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_lb,
                  const __grid_constant__ CUtensorMap map_t, const Params p) {
@@ -398,7 +400,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 // first, so they go out four stages before the end of the tile instead.
                 const int nst = (w.kb1 - w.kb0 + KS - 1) / KS;
                 const int lr_at = (C::NL == 1 && nst > 5) ? nst - 4 : 1;
-                const bool mid = lr_mid_tile(C::NL, w.has_lr, lr_chunks, nst);
+                const bool mid = MID && lr_mid_tile(C::NL, w.has_lr, lr_chunks, nst);
                 int mid_next = 0;          // mid-tile schedule: next chunk to load
                 int st_idx = 0;
                 for (int kb = w.kb0; kb < w.kb1 && ok; kb += KS, ++st_idx) {
@@ -451,7 +453,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 if (!ok) break;
                 tc_fence_after();
                 const int nst = (w.kb1 - w.kb0 + KS - 1) / KS;
-                const bool mid = issuer == 0 && lr_mid_tile(C::NL, w.has_lr, lr_chunks, nst);
+                const bool mid = MID && issuer == 0 && lr_mid_tile(C::NL, w.has_lr, lr_chunks, nst);
                 int lc = 0;                // low-rank chunks of this item multiplied so far
                 // one chunk: wait for its conversion, multiply, hand the slot back
                 auto lr_chunk = [&](int c) {
@@ -555,7 +557,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         };
         while (ok && next_work(cur, p, w)) {
             const int nst = (w.kb1 - w.kb0 + KS - 1) / KS;
-            const bool mid = group == 0 && lr_mid_tile(C::NL, w.has_lr, lr_chunks, nst);
+            const bool mid = MID && group == 0 && lr_mid_tile(C::NL, w.has_lr, lr_chunks, nst);
             int lc = 0;                    // low-rank chunks of this item converted so far
             int st_idx = 0;
             for (int kb = w.kb0; kb < w.kb1 && ok; kb += KS, ++st_idx) {
@@ -850,13 +852,13 @@ Layout make_layout(int M, int N, int K, int r) {
     return L;
 }
 
-template <int BT>
+template <int BT, bool MID>
 int launch_bt(const CUtensorMap& mx, const CUtensorMap& mlb, const CUtensorMap& mt, const Params& p,
               int grid, cudaStream_t st, bool overlap_prev) {
     using C = Cfg<BT>;
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(linear_tc_kernel<BT>,
+        cudaError_t e = cudaFuncSetAttribute(linear_tc_kernel<BT, MID>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, C::SmemBytes);
         if (e != cudaSuccess) return record_cuda_error(e, "linear_tc smem attribute");
         configured = true;
@@ -871,7 +873,7 @@ int launch_bt(const CUtensorMap& mx, const CUtensorMap& mlb, const CUtensorMap& 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = overlap_prev ? 1 : 0;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, linear_tc_kernel<BT>, mx, mlb, mt, p);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, linear_tc_kernel<BT, MID>, mx, mlb, mt, p);
     if (e != cudaSuccess) return record_cuda_error(e, "linear_tc_kernel");
     return check_launch("linear_tc_kernel");
 }
@@ -950,10 +952,12 @@ int launch_linear_tc(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
     p.tail_first = (L.KB >= 64) ? 1 : 0;
 
     switch (L.BT) {
-        case 16: return launch_bt<16>(mx, mlb, mt, p, grid, st, overlap_prev);
-        case 32: return launch_bt<32>(mx, mlb, mt, p, grid, st, overlap_prev);
-        case 64: return launch_bt<64>(mx, mlb, mt, p, grid, st, overlap_prev);
-        default: return launch_bt<128>(mx, mlb, mt, p, grid, st, overlap_prev);
+        case 16: return launch_bt<16, false>(mx, mlb, mt, p, grid, st, overlap_prev);
+        case 32: return launch_bt<32, false>(mx, mlb, mt, p, grid, st, overlap_prev);
+        case 64: return launch_bt<64, false>(mx, mlb, mt, p, grid, st, overlap_prev);
+        default:
+            if (r > 64) return launch_bt<128, true>(mx, mlb, mt, p, grid, st, overlap_prev);
+            return launch_bt<128, false>(mx, mlb, mt, p, grid, st, overlap_prev);
     }
 }
 

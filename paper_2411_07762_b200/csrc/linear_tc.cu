@@ -919,12 +919,26 @@ int launch_linear_tc(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
             if (L.units % g) continue;
             const long long share = L.units / g;
             if (share < KBl && KBl % share == 0) { grid = g; break; }
-            // ... and where a CTA's share is short, a grid that gives every CTA WHOLE tiles (no tile
-            // shared, no reduction through the workspace) beats one more busy SM in six.  Measured
-            // at 128 CTAs against 148: 2 tiles of 32 blocks -28 %, 8 x 32 -6 %, 14 x 32 -3 %,
-            // 4 x 64 -2 %; but 28 x 32 +6 %, 16 x 64 +3 %, 4 x 112 +6 % (long tiles hide the
-            // reduction, long shares make the idle SMs expensive).
-            if (share % KBl == 0 && share <= 512 && KBl <= 64) { grid = g; break; }
+        }
+        // 128-token tiles: a grid that gives every CTA WHOLE tiles has no shared tile at all.  A
+        // shared 128 x 128 tile costs a 128 KB partial (int32 + fp32) per contributor through the
+        // workspace and a serial tail in the last CTA while the accumulators wait; measured, a
+        // launch with shared tiles pays about as much as 64 more column blocks per CTA (20 us at
+        // K = 4096; about half of that where tiles are long and hide it).  So: the smallest
+        // whole-tile share among the grids down to a third of the SM count, taken if it beats the
+        // split share plus that fee.  Measured at 128 against 148 CTAs: 2 tiles of 32 blocks
+        // -28 %, 8 x 32 -6 %, 14 x 32 -3 %, 4 x 64 -2 %; at 112 CTAs 2 x 64 -27 %; 28 x 32,
+        // 16 x 64 and 4 x 112 are faster split and stay so.
+        if (L.BT == 128) {
+            const long long fee = (KBl <= 64) ? 64 : 32;
+            long long best = (L.units + grid - 1) / grid + fee;
+            int best_g = 0;
+            for (int g = num_sms < kMaxCtas ? num_sms : kMaxCtas; g >= num_sms / 3 && g >= 1; --g) {
+                if (L.units % ((long long)g * KBl)) continue;
+                const long long share = L.units / g;
+                if (share < best) { best = share; best_g = g; }
+            }
+            if (best_g) grid = best_g;
         }
     }
 

@@ -20,7 +20,9 @@
  * row-major and contiguous; pointers must be 16-byte aligned.  The library
  * allocates no memory, never synchronises (except aser_check_status), and
  * enqueues all work on the cudaStream_t passed as `stream` (NULL = the legacy
- * default stream).  NaN/Inf inputs give unspecified values but never a fault.
+ * default stream).  A process may use the library on several devices (the one current at the
+ * call is used; per-device set-up is done on first use).  NaN/Inf inputs give unspecified
+ * values but never a fault.
  * Shapes: M >= 0, K % 128 == 0, N % 8 == 0, r % 16 == 0, 0 <= r <= 256.
  * M == 0 is a no-op that returns ASER_OK.
  */
@@ -44,7 +46,7 @@ extern "C" {
 #define ASER_ERR_DEVICE         -7  /* current device is not compute capability 10.x */
 
 /*
- * aser_pack_w4 -- offline weight quantization (Sec. 4.2 Eq. 9/11: Q(W_s) of the
+ * aser_pack_w4 -- offline weight quantization (Sec. 4.2 Eq. 10/12: Q(W_s) of the
  * smoothed weight W M; Sec. 5.1: per-channel round-to-nearest).
  *   ws = fp32(W[n,k]) * s[k]            (one fp32 multiply; s == NULL means ones)
  *   w_scale[n] = max_k |ws| / 7         (fp32 division)
@@ -70,7 +72,7 @@ int aser_unrepack_w4(const void* Wk, int N, int K, uint8_t* Wq, void* stream);
 
 /*
  * aser_quant_act -- fused activation kernel: smoothing (Sec. 4.2, the M^-1 X
- * factor of Eq. 9), per-token int8 round-to-nearest (Sec. 5.1) and the down
+ * factor of Eq. 10), per-token int8 round-to-nearest (Sec. 5.1) and the down
  * projection of the reconstruction branch (Sec. 4.1, V_r^T S^-1 applied to X~).
  *   x~ = fp32(X[m,k]) / s[k]                       (fp32 division; s == NULL means ones)
  *   a_scale[m] = max_k |x~| / 127                  (fp32 division; zero row -> 0, codes 0)
@@ -97,6 +99,24 @@ int aser_quant_act_bits(const void* X_f16, const float* s, const void* LA_f16,
                         int8_t* Xq, float* a_scale, void* T_bf16, void* stream);
 
 /*
+ * aser_quant_act_ex -- aser_quant_act_bits with a choice of how T is stored (the paper fixes no
+ * storage precision for the intermediate of its low-rank branch, Sec. 4.1):
+ *   t_pair == 0: T [M, r] bf16, as above.
+ *   t_pair == 1: T [M, 2r] bf16 holds every entry as a pair, T[m,j] = bf16(t) and
+ *                T[m,r+j] = bf16(t - T[m,j]), i.e. 16 significant bits instead of 8.  The linear
+ *                kernels need no change: call them with rank 2r and the up projection written
+ *                twice, LB2 [N, 2r] = [L_B | L_B], so that L_B T_hi + L_B T_lo is what they add.
+ *                Needs 2r <= 256.  Meant for layers whose low-rank term is as large as the
+ *                output itself (the paper's outlier split of Sec. 4.2, Eq. 12, where whole
+ *                weight columns ride on the factors): there the 2^-9 rounding of a single bf16
+ *                is not small against the output tolerance.
+ * Everything else as aser_quant_act_bits.
+ */
+int aser_quant_act_ex(const void* X_f16, const float* s, const void* LA_f16,
+                      int M, int K, int r, int act_bits, int t_pair,
+                      int8_t* Xq, float* a_scale, void* T_bf16, void* stream);
+
+/*
  * aser_linear_w4a8_lr -- integer GEMM, dequantisation and up projection
  * (Sec. 4.2: W_q X + L_A L_B X in the paper's letters):
  *   acc[m,n] = sum_k Xq[m,k] * q[n,k]                               (exact int32)
@@ -104,8 +124,11 @@ int aser_quant_act_bits(const void* X_f16, const float* s, const void* LA_f16,
  * Wk is the repacked weight (aser_repack_w4).  acc_debug, when not NULL, receives the
  * int32 accumulators [M,N] (bit-exact); pass NULL in timed runs.  workspace must hold
  * aser_workspace_bytes(M,N,K,r) bytes, must have been zeroed once with
- * aser_workspace_init, and may be reused by later calls on the same stream; two calls
- * that overlap in time need separate workspaces.  With at most 16 tokens and at most 64 MB of
+ * aser_workspace_init, and may be reused by later calls on the same stream, of the same or of
+ * any other shape it is large enough for (the status word and the tile counters sit at fixed
+ * offsets and every launch leaves the counters at zero); two calls that overlap in time need
+ * separate workspaces.  Both kernels feed T to the tensor cores as fp16: finite entries of
+ * magnitude 65504 or more become infinite there, so |T| must stay below that.  With at most 16 tokens and at most 64 MB of
  * packed weights the call runs a streaming kernel that leaves the workspace untouched; the
  * argument is validated all the same, so callers need not know which kernel serves a shape.
  * aser_linear_w4a8 is the same without the low-rank term (the plain W4A8 control).
@@ -162,13 +185,14 @@ size_t aser_workspace_bytes(int M, int N, int K, int r);
 int aser_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
 /*
  * aser_check_status -- synchronises `stream`, reads the status word and returns
- * ASER_OK or ASER_ERR_DEVICE_TIMEOUT (a kernel's bounded wait gave up; its output is
- * invalid).  Clears the word.  Debugging aid, not part of the hot path.
+ * ASER_OK or ASER_ERR_DEVICE_TIMEOUT (a kernel's bounded wait, about 0.2 s, gave up; its output
+ * is invalid).  Clears the word and the tile counters that such a launch may have left
+ * behind, so the workspace is usable again.  Debugging aid, not part of the hot path.
  */
 int aser_check_status(void* workspace, void* stream);
 
 /*
- * aser_forward -- one whole forward pass of the layer (Sec. 4.2, Eq. 9 with the low-rank term
+ * aser_forward -- one whole forward pass of the layer (Sec. 4.2, Eq. 10 with the low-rank term
  * of Sec. 4.1) from DEVICE buffers: aser_quant_act followed by aser_linear_w4a8_lr (the plain
  * kernel when r == 0), enqueued on `stream`, no synchronisation.
  * Because the library knows that the quantization kernel is what precedes the linear kernel,
@@ -180,7 +204,8 @@ int aser_check_status(void* workspace, void* stream);
  * for aser_linear_w4a8_lr.  Xq [M,K], a_scale [M], T_bf16 [M,r] (NULL when r == 0) are the
  * caller's intermediates (written), Y_f16 [M,N] the result.  Wk, w_scale and LB_f16 must not
  * be written by work still in flight on `stream` when the call is made.
- * Errors: as the two calls; nothing is enqueued when an argument is rejected.
+ * Errors: as the two calls; every argument of both launches is checked first, so nothing is
+ * enqueued when one is rejected.
  */
 int aser_forward(const void* X_f16, const float* s, const void* LA_f16, const void* Wk,
                  const float* w_scale, const void* LB_f16, int M, int N, int K, int r,
@@ -191,7 +216,8 @@ int aser_forward(const void* X_f16, const float* s, const void* LA_f16, const vo
  * aser_forward_host -- one whole forward pass from HOST buffers: copies X (fp16 [M,K],
  * ideally pinned) to the device staging buffer X_dev, runs aser_forward, and copies Y back to Y_host,
  * all enqueued on `stream`; returns without synchronising.  Device-side operands and
- * staging buffers are the caller's.
+ * staging buffers are the caller's.  All arguments are checked before the first copy is
+ * enqueued.
  */
 int aser_forward_host(const void* X_host_f16, void* Y_host_f16,
                       void* X_dev, int8_t* Xq_dev, float* a_scale_dev, void* T_dev, void* Y_dev,

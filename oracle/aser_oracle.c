@@ -69,7 +69,7 @@ static float f16_to_f32(uint16_t h)
 }
 
 /* ---------------------------------------------------------------------------
- * Activation smoothing (Sec. 4.2, Eq. 9: W X = (W M)(M^-1 X)).
+ * Activation smoothing (Sec. 4.2, Eq. 10: W X = (W M)(M^-1 X)).
  * x~[m,k] = fp32(X[m,k]) / s[k], one fp32 division.  s == NULL means all ones.
  * ------------------------------------------------------------------------- */
 void aser_oracle_smooth_act(const uint16_t* X, const float* s, long M, long K, float* xs)
@@ -121,7 +121,7 @@ void aser_oracle_quant_act(const float* xs, long M, long K, int8_t* Xq, float* a
 
 /* ---------------------------------------------------------------------------
  * Per-output-channel symmetric int4 round-to-nearest of the smoothed weight
- * W diag(s) (Sec. 4.2 Eq. 9 and Eq. 11, Q(W_s); Sec. 5.1 "per-channel for
+ * W diag(s) (Sec. 4.2 Eq. 10 and Eq. 12, Q(W_s); Sec. 5.1 "per-channel for
  * weights").  ws = fp32(W) * s (one fp32 multiply); w_scale[n] = max_k|ws|/7;
  * code = rne(ws / w_scale) clamped to [-8, 7].  A zero row: scale 0, codes 0.
  * `ws_out` (optional) receives the smoothed fp32 weights.

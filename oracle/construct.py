@@ -1,7 +1,7 @@
 """Oracle construction of an ASER-quantized layer (test infrastructure, NumPy fp64).
 
 Follows the per-layer body of Algorithm 1 of the paper: smoothing vector
-(Sec. 4.2, Eq. 10), int4 round-to-nearest of the smoothed weight, whitening by
+(Sec. 4.2, Eq. 11), int4 round-to-nearest of the smoothed weight, whitening by
 Cholesky (Sec. 4.1, Eq. 5), SVD of the whitened error and truncation (Eq. 6),
 factor split (text below Eq. 8), rank threshold (Eq. 9 of Sec. 4.1).
 
@@ -16,7 +16,7 @@ Readings where the paper is silent (all recorded in the design notes):
     channels and an undamped Cholesky would not exist;
   * the Cholesky factor is the lower one, the Gram matrix is not normalised;
   * the SVD target with the outlier split is W diag(s) - Q(W_s), i.e.
-    E_q + W_o with E_q = W_s - Q(W_s) (Eq. 11), not the double-counted
+    E_q + W_o with E_q = W_s - Q(W_s) (Eq. 12), not the double-counted
     expression printed inside Algorithm 1.
 """
 from __future__ import annotations
@@ -46,7 +46,7 @@ def outlier_index_set(X_cal: np.ndarray, W: np.ndarray, f: int) -> np.ndarray:
 
 
 def smoothing_vector_paper(X_cal: np.ndarray, W: np.ndarray, f: int):
-    """Eq. 10: m_i = X-bar_i / min_{I_f} X-bar on the outlier set, 1 elsewhere."""
+    """Eq. 11: m_i = X-bar_i / min_{I_f} X-bar on the outlier set, 1 elsewhere."""
     idx = outlier_index_set(X_cal, W, f)
     xbar = channel_abs_mean(X_cal)
     m = np.ones(X_cal.shape[1], dtype=np.float64)
@@ -138,7 +138,7 @@ def construct_layer(W: np.ndarray, X_cal: np.ndarray, s: np.ndarray | None, r: i
     """Quantize W diag(s) to int4 and build rank-r factors from calibration tokens.
 
     `split_outliers`: index set I_f whose columns of W diag(s) are kept out of
-    the quantizer (W_o, Eq. 11) and carried by the low-rank term only.
+    the quantizer (W_o, Eq. 12) and carried by the low-rank term only.
     Exactly one of `r`, `alpha` selects the rank.
     """
     N, K = W.shape

@@ -60,7 +60,7 @@ def _f16_bits(a: np.ndarray) -> np.ndarray:
 
 
 def smooth_act(X: np.ndarray, s: np.ndarray | None) -> np.ndarray:
-    """x~ = fp32(X) / s  (Eq. 9, the M^-1 X factor).  X fp16 [M,K], s fp32 [K] or None."""
+    """x~ = fp32(X) / s  (Eq. 10, the M^-1 X factor).  X fp16 [M,K], s fp32 [K] or None."""
     Xb = _f16_bits(X)
     M, K = Xb.shape
     sv = None if s is None else _c(s, np.float32)

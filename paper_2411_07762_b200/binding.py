@@ -11,7 +11,7 @@ lib_path = os.path.join(_HERE, "libaser.so")
 
 EXPORTED_SYMBOLS = (
     "aser_pack_w4", "aser_repacked_bytes", "aser_repack_w4", "aser_unrepack_w4",
-    "aser_quant_act", "aser_quant_act_bits", "aser_linear_w4a8_lr", "aser_linear_w4a8", "aser_linear_w4a8_lr_simt", "aser_linear_w4a8_lr_static",
+    "aser_quant_act", "aser_quant_act_bits", "aser_quant_act_ex", "aser_linear_w4a8_lr", "aser_linear_w4a8", "aser_linear_w4a8_lr_simt", "aser_linear_w4a8_lr_static",
     "aser_workspace_bytes", "aser_workspace_init", "aser_check_status", "aser_forward",
     "aser_forward_host",
     "aser_last_error", "aser_version",
@@ -31,6 +31,7 @@ lib.aser_repack_w4.argtypes = [_P, _I, _I, _P, _P]
 lib.aser_unrepack_w4.argtypes = [_P, _I, _I, _P, _P]
 lib.aser_quant_act.argtypes = [_P, _P, _P, _I, _I, _I, _P, _P, _P, _P]
 lib.aser_quant_act_bits.argtypes = [_P, _P, _P, _I, _I, _I, _I, _P, _P, _P, _P]
+lib.aser_quant_act_ex.argtypes = [_P, _P, _P, _I, _I, _I, _I, _I, _P, _P, _P, _P]
 lib.aser_linear_w4a8_lr.argtypes = [_P, _P, _P, _P, _P, _P, _I, _I, _I, _I, _P, _P, _P, _Z, _P]
 lib.aser_linear_w4a8.argtypes = [_P, _P, _P, _P, _I, _I, _I, _P, _P, _P, _Z, _P]
 lib.aser_linear_w4a8_lr_simt.argtypes = [_P, _P, _P, _P, _P, _P, _I, _I, _I, _I, _P, _P, _P]
@@ -109,18 +110,24 @@ def unrepack_w4(Wk: torch.Tensor, N: int, K: int) -> torch.Tensor:
 
 
 def quant_act(X: torch.Tensor, s: torch.Tensor | None, L_A: torch.Tensor | None,
-              out=None, act_bits: int = 8):
+              out=None, act_bits: int = 8, t_pair: bool = False):
     """X fp16 [M,K] -> (Xq int8 [M,K], a_scale fp32 [M], T bf16 [M,r]).  act_bits != 8 goes
-    through aser_quant_act_bits (codes of that width in the int8 container)."""
+    through aser_quant_act_bits (codes of that width in the int8 container); t_pair through
+    aser_quant_act_ex (T [M,2r]: a bf16 value and its bf16 remainder per entry)."""
     _dev(X, torch.float16, "X")
     M, K = X.shape
     r = 0 if L_A is None else L_A.shape[0]
     if out is None:
         Xq = torch.empty((M, K), dtype=torch.int8, device=X.device)
         a_scale = torch.empty((M,), dtype=torch.float32, device=X.device)
-        T = torch.empty((M, r), dtype=torch.bfloat16, device=X.device)
+        T = torch.empty((M, 2 * r if t_pair else r), dtype=torch.bfloat16, device=X.device)
     else:
         Xq, a_scale, T = out
+    if t_pair:
+        _chk(lib.aser_quant_act_ex(_ptr(X), _ptr(s), _ptr(L_A) if r else None, M, K, r, act_bits, 1,
+                                   _ptr(Xq), _ptr(a_scale), _ptr(T) if r else None, _stream()),
+             "aser_quant_act_ex")
+        return Xq, a_scale, T
     if act_bits != 8:
         _chk(lib.aser_quant_act_bits(_ptr(X), _ptr(s), _ptr(L_A) if r else None, M, K, r, act_bits,
                                      _ptr(Xq), _ptr(a_scale), _ptr(T) if r else None, _stream()),
@@ -194,6 +201,11 @@ def linear_w4a8_lr_static(Xq, a_scale, Wk, w_scale, T, L_B, N: int, Y=None, acc_
                                         r, _ptr(Y), _ptr(acc_debug), _stream()),
          "aser_linear_w4a8_lr_static")
     return Y
+
+
+def pair_up_projection(L_B: torch.Tensor) -> torch.Tensor:
+    """[L_B | L_B]: the up projection a linear kernel needs beside a T stored as bf16 pairs."""
+    return torch.cat([L_B, L_B], dim=1).contiguous()
 
 
 def pad_rank(L_A: torch.Tensor, L_B: torch.Tensor, multiple: int = 16):

@@ -26,6 +26,29 @@ int check_launch(const char* where) {
     return ASER_OK;
 }
 
+int current_device(int* dev) {
+    cudaError_t e = cudaGetDevice(dev);
+    if (e != cudaSuccess) return record_cuda_error(e, "cudaGetDevice");
+    if (*dev < 0 || *dev >= kMaxDevices)
+        return record_error(ASER_ERR_DEVICE, "device ordinal beyond the per-device tables");
+    return ASER_OK;
+}
+
+int device_sm_count(int* num_sms) {
+    static int cached[kMaxDevices] = {0};
+    int dev = 0;
+    int rc = current_device(&dev);
+    if (rc != ASER_OK) return rc;
+    if (cached[dev] == 0) {
+        int n = 0;
+        cudaError_t e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess || n <= 0) return record_cuda_error(e, "query SM count");
+        cached[dev] = n;
+    }
+    *num_sms = cached[dev];
+    return ASER_OK;
+}
+
 namespace {
 
 int fail(int code, const char* msg) {
@@ -160,8 +183,16 @@ int aser_quant_act(const void* X_f16, const float* s, const void* LA_f16, int M,
 
 int aser_quant_act_bits(const void* X_f16, const float* s, const void* LA_f16, int M, int K, int r,
                         int act_bits, int8_t* Xq, float* a_scale, void* T_bf16, void* stream) {
+    return aser_quant_act_ex(X_f16, s, LA_f16, M, K, r, act_bits, 0, Xq, a_scale, T_bf16, stream);
+}
+
+int aser_quant_act_ex(const void* X_f16, const float* s, const void* LA_f16, int M, int K, int r,
+                      int act_bits, int t_pair, int8_t* Xq, float* a_scale, void* T_bf16,
+                      void* stream) {
     if (!shape_ok(M, 0, K, r)) return fail(ASER_ERR_SHAPE, "unsupported M, K or r");
     if (act_bits < 2 || act_bits > 8) return fail(ASER_ERR_SHAPE, "act_bits must be 2..8");
+    if (t_pair != 0 && t_pair != 1) return fail(ASER_ERR_SHAPE, "t_pair must be 0 or 1");
+    if (t_pair && 2 * r > 256) return fail(ASER_ERR_SHAPE, "t_pair needs 2 r <= 256");
     if (M == 0) return ASER_OK;
     ASER_REQUIRE_PTR(X_f16);
     ASER_OPTIONAL_PTR(s);
@@ -175,7 +206,7 @@ int aser_quant_act_bits(const void* X_f16, const float* s, const void* LA_f16, i
     if (rc != ASER_OK) return rc;
     return launch_quant_act(static_cast<const __half*>(X_f16), s, static_cast<const __half*>(LA_f16),
                             M, K, r, Xq, a_scale, static_cast<__nv_bfloat16*>(T_bf16),
-                            static_cast<cudaStream_t>(stream), act_bits);
+                            static_cast<cudaStream_t>(stream), act_bits, t_pair != 0);
 }
 
 int aser_linear_w4a8_lr(const int8_t* Xq, const float* a_scale, const void* Wk,
@@ -237,12 +268,40 @@ int aser_check_status(void* workspace, void* stream) {
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return record_cuda_error(e, "aser_check_status");
     if (word == 0) return ASER_OK;
-    e = cudaMemsetAsync(workspace, 0, sizeof(word), st);
+    // a launch that gave up may also have left tile counters behind: clear them with the word
+    e = cudaMemsetAsync(workspace, 0, kWsZeroedBytes, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return record_cuda_error(e, "aser_check_status clear");
     snprintf(g_last_error, sizeof(g_last_error),
              "a bounded device-side wait gave up (status word 0x%08x)", word);
     return ASER_ERR_DEVICE_TIMEOUT;
+}
+
+// Every check aser_forward makes, with nothing enqueued: the arguments of both launches and the
+// linear kernel's own range checks.
+static int forward_validate(const void* X_f16, const float* s, const void* LA_f16, const void* Wk,
+                            const float* w_scale, const void* LB_f16, int M, int N, int K, int r,
+                            const int8_t* Xq, const float* a_scale, const void* T_bf16,
+                            const void* Y_f16, const void* workspace, size_t workspace_bytes) {
+    ASER_REQUIRE_PTR(X_f16);
+    ASER_OPTIONAL_PTR(s);
+    ASER_REQUIRE_PTR(Xq);
+    ASER_REQUIRE_PTR(a_scale);
+    ASER_REQUIRE_PTR(Wk);
+    ASER_REQUIRE_PTR(w_scale);
+    ASER_REQUIRE_PTR(Y_f16);
+    if (r > 0) {
+        ASER_REQUIRE_PTR(LA_f16);
+        ASER_REQUIRE_PTR(T_bf16);
+        ASER_REQUIRE_PTR(LB_f16);
+    }
+    if (workspace == nullptr || misaligned16(workspace) ||
+        workspace_bytes < aser_workspace_bytes(M, N, K, r))
+        return fail(ASER_ERR_WORKSPACE, "workspace missing, misaligned or too small");
+    int rc = check_device();
+    if (rc != ASER_OK) return rc;
+    if (!linear_decode_prefers(M, N, K)) rc = linear_tc_check(M, N, K, r, workspace_bytes);
+    return rc;
 }
 
 int aser_forward(const void* X_f16, const float* s, const void* LA_f16, const void* Wk,
@@ -251,15 +310,10 @@ int aser_forward(const void* X_f16, const float* s, const void* LA_f16, const vo
                  size_t workspace_bytes, void* stream) {
     if (!shape_ok(M, N, K, r)) return fail(ASER_ERR_SHAPE, "unsupported M, N, K or r");
     if (M == 0 || N == 0) return ASER_OK;
-    // validate the second launch's arguments before the first is enqueued
-    ASER_REQUIRE_PTR(Wk);
-    ASER_REQUIRE_PTR(w_scale);
-    ASER_REQUIRE_PTR(Y_f16);
-    if (r > 0) ASER_REQUIRE_PTR(LB_f16);
-    if (workspace == nullptr || misaligned16(workspace) ||
-        workspace_bytes < aser_workspace_bytes(M, N, K, r))
-        return fail(ASER_ERR_WORKSPACE, "workspace missing, misaligned or too small");
-    int rc = aser_quant_act(X_f16, s, LA_f16, M, K, r, Xq, a_scale, T_bf16, stream);
+    int rc = forward_validate(X_f16, s, LA_f16, Wk, w_scale, LB_f16, M, N, K, r, Xq, a_scale, T_bf16,
+                              Y_f16, workspace, workspace_bytes);
+    if (rc != ASER_OK) return rc;
+    rc = aser_quant_act(X_f16, s, LA_f16, M, K, r, Xq, a_scale, T_bf16, stream);
     if (rc != ASER_OK) return rc;
     return linear_common(Xq, a_scale, Wk, w_scale, r > 0 ? T_bf16 : nullptr, r > 0 ? LB_f16 : nullptr,
                          M, N, K, r, Y_f16, nullptr, workspace, workspace_bytes, stream,
@@ -275,13 +329,15 @@ int aser_forward_host(const void* X_host_f16, void* Y_host_f16, void* X_dev, int
     if (M == 0 || N == 0) return ASER_OK;
     if (X_host_f16 == nullptr || Y_host_f16 == nullptr)
         return fail(ASER_ERR_NULL, "host buffer is NULL");
-    ASER_REQUIRE_PTR(X_dev);
-    ASER_REQUIRE_PTR(Y_dev);
+    // everything is checked before the first copy is enqueued
+    int rc = forward_validate(X_dev, s, LA_f16, Wk, w_scale, LB_f16, M, N, K, r, Xq_dev, a_scale_dev,
+                              T_dev, Y_dev, workspace, workspace_bytes);
+    if (rc != ASER_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = cudaMemcpyAsync(X_dev, X_host_f16, (size_t)M * K * 2, cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return record_cuda_error(e, "copy X to device");
-    int rc = aser_forward(X_dev, s, LA_f16, Wk, w_scale, LB_f16, M, N, K, r, Xq_dev, a_scale_dev,
-                          T_dev, Y_dev, workspace, workspace_bytes, stream);
+    rc = aser_forward(X_dev, s, LA_f16, Wk, w_scale, LB_f16, M, N, K, r, Xq_dev, a_scale_dev,
+                      T_dev, Y_dev, workspace, workspace_bytes, stream);
     if (rc != ASER_OK) return rc;
     e = cudaMemcpyAsync(Y_host_f16, Y_dev, (size_t)M * N * 2, cudaMemcpyDeviceToHost, st);
     if (e != cudaSuccess) return record_cuda_error(e, "copy Y to host");

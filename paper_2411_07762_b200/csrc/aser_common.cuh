@@ -18,6 +18,14 @@ int record_error(int code, const char* msg);
 // cudaGetLastError() after a launch -> ASER_OK or ASER_ERR_LAUNCH.
 int check_launch(const char* where);
 
+// Per-device caches (shared-memory opt-ins, SM counts, occupancy answers) are arrays indexed by
+// the CUDA device ordinal: a process may drive several GPUs, and function attributes belong to
+// a device's context.  current_device returns ASER_OK and the ordinal, or an error code.
+constexpr int kMaxDevices = 64;
+int current_device(int* dev);
+// Number of SMs of the current device.
+int device_sm_count(int* num_sms);
+
 inline bool misaligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 
 // Kernel launchers (one per .cu file); arguments are already validated.
@@ -25,8 +33,10 @@ int launch_pack_w4(const __half* W, const float* s, int N, int K, uint8_t* Wq, f
                    cudaStream_t st);
 int launch_repack_w4(const uint8_t* Wq, int N, int K, uint8_t* Wk, bool inverse, cudaStream_t st);
 // act_bits: width of the symmetric activation codes (2..8); they are stored in int8 either way.
+// t_pair: T is written as [M, 2r], a bf16 value and the bf16 remainder of each entry.
 int launch_quant_act(const __half* X, const float* s, const __half* LA, int M, int K, int r,
-                     int8_t* Xq, float* a_scale, __nv_bfloat16* T, cudaStream_t st, int act_bits = 8);
+                     int8_t* Xq, float* a_scale, __nv_bfloat16* T, cudaStream_t st, int act_bits = 8,
+                     bool t_pair = false);
 int launch_linear_simt(const int8_t* Xq, const float* a_scale, const uint8_t* Wq,
                        const float* w_scale, const __nv_bfloat16* T, const __half* LB,
                        int M, int N, int K, int r, __half* Y, int32_t* acc_debug, cudaStream_t st);
@@ -48,6 +58,9 @@ int launch_linear_decode(const int8_t* Xq, const float* a_scale, const uint8_t* 
                          int M, int N, int K, int r, __half* Y, int32_t* acc_debug,
                          cudaStream_t st, bool overlap_prev = false);
 size_t linear_tc_workspace_bytes(int M, int N, int K, int r);
+// The range checks launch_linear_tc makes before it launches (workspace size, index widths), for
+// callers that must reject a call before they enqueue anything else.  Records the error text.
+int linear_tc_check(int M, int N, int K, int r, size_t workspace_bytes);
 // Leading bytes of the workspace (status word + tile counters) that must be zero at launch.
 size_t linear_tc_zeroed_prefix_bytes(int M, int N, int K, int r);
 
@@ -62,8 +75,11 @@ constexpr int kWkRows = 128;
 constexpr int kWkCols = 128;
 constexpr int kWkBlockBytes = kWkRows * kWkCols / 2;  // 8192
 
-// Workspace header (first 256 bytes): word 0 = status, rest reserved.
+// Workspace header (first 256 bytes): word 0 = status, rest reserved.  The tile counters of the
+// tensor-core kernel follow; header and counters (kWsZeroedBytes in all) must read zero when a
+// kernel starts, everything behind them is written before it is read.
 constexpr size_t kWsHeaderBytes = 256;
+constexpr size_t kWsZeroedBytes = 1024;
 
 #ifdef __CUDACC__
 // ---- device side -----------------------------------------------------------

@@ -299,12 +299,10 @@ int launch_nt(const int8_t* Xq, const float* a_scale, const uint8_t* Wk, const f
               int32_t* acc_debug, cudaStream_t st, bool overlap_prev) {
     // Rows per CTA: 32 where that still gives every SM about one and a half CTAs (activation
     // fragments reused twice), else 16 (few output channels: latency matters, every SM gets work).
-    static int num_sms = 0;
-    if (num_sms == 0) {
-        int dev = 0;
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
-        if (e != cudaSuccess) { num_sms = 0; return record_cuda_error(e, "query SM count"); }
+    int num_sms = 0;
+    {
+        const int rc = device_sm_count(&num_sms);
+        if (rc != ASER_OK) return rc;
     }
     // (Four blocks in flight per warp at 32 rows, i.e. 256 bytes per thread and two CTAs per SM,
     // measured 7 % slower at 8192 x 8192 than two blocks and three CTAs per SM.)

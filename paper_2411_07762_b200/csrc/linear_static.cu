@@ -3,38 +3,41 @@
 // shared between CTAs) lives in a fixed array that is part of the library image.
 #include <stdio.h>
 
+#include <atomic>
+
 #include "aser_common.cuh"
 
 namespace aser {
 namespace {
 
 constexpr size_t kStaticScratchBytes = 8u << 20;  // 8 MiB: enough for up to 32 tokens per call
-constexpr int kMaxDevices = 64;
 
 // One copy per GPU that loads the library, resident until the process exits.
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 // Device address of g_static_scratch per CUDA device ordinal.  In host code the array's name
 // only identifies the symbol; the address a kernel can use comes from cudaGetSymbolAddress.
-void* g_scratch_addr[kMaxDevices] = {nullptr};
+// Threads may race to fill a slot; they store the same value, atomically.  An address stays
+// valid for the life of the device's primary context: after cudaDeviceReset it is stale.
+std::atomic<void*> g_scratch_addr[kMaxDevices];
 
 int scratch_for_current_device(void** out) {
     int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return record_cuda_error(e, "cudaGetDevice");
-    if (dev < 0 || dev >= kMaxDevices)
-        return record_error(ASER_ERR_DEVICE, "device ordinal beyond the static scratch table");
-    if (g_scratch_addr[dev] == nullptr) {
+    const int rc = current_device(&dev);
+    if (rc != ASER_OK) return rc;
+    void* addr = g_scratch_addr[dev].load(std::memory_order_acquire);
+    if (addr == nullptr) {
         int major = 0;
-        e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+        cudaError_t e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
         if (e != cudaSuccess) return record_cuda_error(e, "cudaDeviceGetAttribute");
         if (major != 10) return record_error(ASER_ERR_DEVICE, "device is not compute capability 10.x");
         void* ptr = nullptr;
         e = cudaGetSymbolAddress(&ptr, g_static_scratch);
         if (e != cudaSuccess) return record_cuda_error(e, "cudaGetSymbolAddress(static scratch)");
-        g_scratch_addr[dev] = ptr;
+        g_scratch_addr[dev].store(ptr, std::memory_order_release);
+        addr = ptr;
     }
-    *out = g_scratch_addr[dev];
+    *out = addr;
     return ASER_OK;
 }
 

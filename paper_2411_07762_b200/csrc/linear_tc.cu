@@ -31,7 +31,7 @@ namespace {
 
 constexpr int kMaxCtas = 160;     // upper bound on the persistent grid (workspace sizing)
 constexpr uint32_t kStatusTimeout = 1u;
-constexpr long long kWaitLimitClocks = 4000000000ll;  // about 2 s of SM clocks per wait
+constexpr long long kWaitLimitClocks = 400000000ll;  // about 0.2 s of SM clocks per wait
 
 // Per token-tile configuration.  A pipeline stage carries KS 128-column blocks: one bulk copy of
 // KS x 8 KiB of packed weights, one TMA box of KS activation tiles, KS x 32 tensor-memory columns
@@ -89,7 +89,7 @@ struct Params {
     __half* Y;
     int32_t* acc_debug;
     uint32_t* status;      // workspace word 0
-    int* counters;         // one per tile
+    int* counters;         // one per CTA: a shared tile's counter is that of the CTA owning its first unit
     int32_t* part_int;     // [grid][2][BT][128]
     float* part_lr;        // [grid][BT][128]
     int M, N, K, r;
@@ -715,15 +715,18 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 named_bar_sync(1, C::EpiThreads);            // every partial store of this CTA precedes ...
                 if (et == 0) {                     // ... this release; the last arriver acquires all
                     int old;
+                    // A CTA owns the first unit of at most one shared tile (the one cut off at the
+                    // end of its range), so c_first names the tile's counter: the counter array
+                    // has a fixed size and place whatever the problem's shape.
                     asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;"
-                                 : "=r"(old) : "l"(p.counters + w.tile) : "memory");
+                                 : "=r"(old) : "l"(p.counters + c_first) : "memory");
                     *last_flag = (old == c_last - c_first) ? 1 : 0;
                 }
                 named_bar_sync(1, C::EpiThreads);
                 const bool last = *last_flag != 0;
                 named_bar_sync(1, C::EpiThreads);           // everyone has read the flag before it is reused
                 if (last) {
-                    if (et == 0) p.counters[w.tile] = 0;   // ready for the next launch
+                    if (et == 0) p.counters[c_first] = 0;  // ready for the next launch
                     // Slot of every contributor, computed once (by one thread each) instead of
                     // per chunk: CTA c's items in order are a tile cut off at the start of its
                     // range (slot 0), whole tiles, a tile cut off at the end of its range.
@@ -816,17 +819,11 @@ int make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, int esize, const void*
 // tokens x 128 bytes, 128-byte swizzle.  In shared memory each block's BT x 128-byte tile is
 // contiguous, which is the K-major operand layout the MMA descriptor expects.
 int make_map_x(CUtensorMap* map, const void* base, uint64_t M, uint64_t K, uint32_t BT, uint32_t KS) {
-    EncodeTiledFn fn = get_encode_fn();
-    if (!fn) return record_cuda_error(cudaErrorUnknown, "cuTensorMapEncodeTiled unavailable");
-    cuuint64_t dims[3] = {128, M, K / 128};
-    cuuint64_t strides[2] = {K, 128};
-    cuuint32_t box[3] = {128, BT, KS};
-    cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(base), dims, strides, box,
-                    estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return record_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled (Xq)");
-    return ASER_OK;
+    MapKey k = make_key(base, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, CU_TENSOR_MAP_SWIZZLE_128B);
+    k.dims[0] = 128; k.dims[1] = M; k.dims[2] = K / 128;
+    k.strides[0] = K; k.strides[1] = 128;
+    k.box[0] = 128; k.box[1] = BT; k.box[2] = KS;
+    return encode_tiled(map, k, "cuTensorMapEncodeTiled (Xq)");
 }
 
 int pick_bt(int M) { return M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128; }
@@ -844,9 +841,11 @@ Layout make_layout(int M, int N, int K, int r) {
     L.TT = (M + L.BT - 1) / L.BT;
     L.KB = K / 128;
     L.units = (long long)L.NT * L.TT * L.KB;
-    size_t tiles = (size_t)L.NT * L.TT;
+    // Status word and counters sit at the same offsets for every shape, and a launch leaves the
+    // counters at zero again, so one workspace serves calls of different shapes in turn.
     L.off_counters = kWsHeaderBytes;
-    L.off_part_int = L.off_counters + ((tiles * 4 + 255) / 256) * 256;
+    L.off_part_int = kWsZeroedBytes;
+    static_assert(kWsHeaderBytes + kMaxCtas * 4 <= kWsZeroedBytes, "counter region");
     L.off_part_lr = L.off_part_int + (size_t)kMaxCtas * 2 * L.BT * 128 * 4;
     L.total = L.off_part_lr + (r > 0 ? (size_t)kMaxCtas * L.BT * 128 * 4 : 0);
     return L;
@@ -856,12 +855,15 @@ template <int BT, bool MID>
 int launch_bt(const CUtensorMap& mx, const CUtensorMap& mlb, const CUtensorMap& mt, const Params& p,
               int grid, cudaStream_t st, bool overlap_prev) {
     using C = Cfg<BT>;
-    static bool configured = false;
-    if (!configured) {
+    static bool configured[kMaxDevices] = {false};
+    int dev = 0;
+    const int drc = current_device(&dev);
+    if (drc != ASER_OK) return drc;
+    if (!configured[dev]) {
         cudaError_t e = cudaFuncSetAttribute(linear_tc_kernel<BT, MID>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, C::SmemBytes);
         if (e != cudaSuccess) return record_cuda_error(e, "linear_tc smem attribute");
-        configured = true;
+        configured[dev] = true;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid, 1, 1);
@@ -881,13 +883,20 @@ int launch_bt(const CUtensorMap& mx, const CUtensorMap& mlb, const CUtensorMap& 
 }  // namespace
 
 size_t linear_tc_workspace_bytes(int M, int N, int K, int r) {
-    if (M <= 0 || N <= 0) return 0;
+    if (M <= 0 || N <= 0) return kWsZeroedBytes - kWsHeaderBytes;
     return make_layout(M, N, K, r).total - kWsHeaderBytes;
 }
 
-size_t linear_tc_zeroed_prefix_bytes(int M, int N, int K, int r) {
-    if (M <= 0 || N <= 0) return kWsHeaderBytes;
-    return make_layout(M, N, K, r).off_part_int;
+size_t linear_tc_zeroed_prefix_bytes(int, int, int, int) { return kWsZeroedBytes; }
+
+int linear_tc_check(int M, int N, int K, int r, size_t workspace_bytes) {
+    const Layout L = make_layout(M, N, K, r);
+    if (workspace_bytes < L.total) return record_error(ASER_ERR_WORKSPACE, "workspace too small");
+    if (L.units >= (1ll << 31) / kMaxCtas * kMaxCtas)
+        return record_error(ASER_ERR_SHAPE, "M * N * K beyond the kernel's 31-bit work-unit count");
+    if ((long long)(M + 128) * N >= (1ll << 32))   // 32-bit element indices in the epilogue
+        return record_error(ASER_ERR_SHAPE, "M * N beyond the kernel's 32-bit output index");
+    return ASER_OK;
 }
 
 int launch_linear_tc(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
@@ -895,16 +904,13 @@ int launch_linear_tc(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
                      int M, int N, int K, int r, __half* Y, int32_t* acc_debug,
                      void* workspace, size_t workspace_bytes, cudaStream_t st, bool overlap_prev) {
     Layout L = make_layout(M, N, K, r);
-    if (workspace_bytes < L.total) return ASER_ERR_WORKSPACE;
-    if (L.units >= (1ll << 31) / kMaxCtas * kMaxCtas) return ASER_ERR_SHAPE;
-    if ((long long)(M + 128) * N >= (1ll << 32)) return ASER_ERR_SHAPE;   // 32-bit element indices in the epilogue
+    const int pre = linear_tc_check(M, N, K, r, workspace_bytes);
+    if (pre != ASER_OK) return pre;
 
-    static int num_sms = 0;
-    if (num_sms == 0) {
-        int dev = 0;
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
-        if (e != cudaSuccess) { num_sms = 0; return record_cuda_error(e, "query SM count"); }
+    int num_sms = 0;
+    {
+        const int rc = device_sm_count(&num_sms);
+        if (rc != ASER_OK) return rc;
     }
     int grid = num_sms < kMaxCtas ? num_sms : kMaxCtas;
     long long want = (L.units + 1) / 2;   // at least two units per CTA on tiny problems

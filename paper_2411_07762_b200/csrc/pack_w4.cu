@@ -1,5 +1,5 @@
 // Offline weight path: smoothing multiply, per-output-channel int4 round-to-nearest,
-// nibble packing (Sec. 4.2 Eq. 9/11 Q(W_s); Sec. 5.1 per-channel RTN), plus the
+// nibble packing (Sec. 4.2 Eq. 10/12 Q(W_s); Sec. 5.1 per-channel RTN), plus the
 // permutation between the canonical packed form and the tensor-core kernel's layout.
 #include "aser_common.cuh"
 

@@ -1,4 +1,4 @@
-// Fused activation kernel: smoothing divide (Sec. 4.2, the M^-1 X factor of Eq. 9),
+// Fused activation kernel: smoothing divide (Sec. 4.2, the M^-1 X factor of Eq. 10),
 // per-token int8 round-to-nearest (Sec. 5.1) and the down projection T = X~ L_A^T of the
 // error-reconstruction branch (Sec. 4.1).
 //
@@ -74,6 +74,22 @@ __device__ __forceinline__ uint2 quant8(const float (&v)[8], float sc, bool nonz
     return make_uint2(w[0], w[1]);
 }
 
+// T element(s) -> memory.  `lo_off` == 0: T[j] = bf16(t).  Otherwise T is stored as a PAIR of
+// bf16 numbers, T[j] = bf16(t) and T[j + lo_off] = bf16(t - T[j]), whose sum carries 16
+// significant bits; a linear kernel given the up projection twice, [L_B | L_B], then adds both.
+__device__ __forceinline__ void store_t(__nv_bfloat16* row, int j, float t, int lo_off) {
+    const __nv_bfloat16 hi = __float2bfloat16_rn(t);
+    row[j] = hi;
+    if (lo_off) row[j + lo_off] = __float2bfloat16_rn(t - __bfloat162float(hi));
+}
+__device__ __forceinline__ void store_t2(__nv_bfloat16* row, int j, float t0, float t1, int lo_off) {
+    const __nv_bfloat162 hi = __floats2bfloat162_rn(t0, t1);
+    *reinterpret_cast<__nv_bfloat162*>(row + j) = hi;
+    if (lo_off)
+        *reinterpret_cast<__nv_bfloat162*>(row + j + lo_off) =
+            __floats2bfloat162_rn(t0 - __low2float(hi), t1 - __high2float(hi));
+}
+
 // ---------------------------------------------------------------------------
 // few tokens
 // ---------------------------------------------------------------------------
@@ -87,7 +103,7 @@ __global__ void __launch_bounds__(kSmallThreads)
 quant_act_small_kernel(const __half* __restrict__ X, const float* __restrict__ s,
                        const __half* __restrict__ LA, int M, int K, int r,
                        int8_t* __restrict__ Xq, float* __restrict__ a_scale,
-                       __nv_bfloat16* __restrict__ T, float qmax) {
+                       __nv_bfloat16* __restrict__ T, int ldt, int lo_off, float qmax) {
     extern __shared__ __align__(16) float xs[];
     grid_dep_launch();      // a dependent linear kernel may start streaming its weights
     __shared__ float red[kRowsPerCta][kSmallThreads / 32];
@@ -165,7 +181,7 @@ quant_act_small_kernel(const __half* __restrict__ X, const float* __restrict__ s
         float t = 0.f;
 #pragma unroll
         for (int i = 0; i < kSmallThreads / 32; ++i) t += red[threadIdx.x][i];
-        T[(size_t)m * r + j0 + threadIdx.x] = __float2bfloat16_rn(t);
+        store_t(T + (size_t)m * ldt, j0 + threadIdx.x, t, lo_off);
     }
 }
 
@@ -208,7 +224,7 @@ __global__ void __launch_bounds__(kLargeThreads)
 quant_act_large_kernel(const __half* __restrict__ X, const float* __restrict__ s,
                        const __half* __restrict__ LA, int M, int K, int r,
                        int8_t* __restrict__ Xq, float* __restrict__ a_scale,
-                       __nv_bfloat16* __restrict__ T, float qmax) {
+                       __nv_bfloat16* __restrict__ T, int ldt, int lo_off, float qmax) {
     extern __shared__ __align__(16) uint8_t smem[];
     grid_dep_launch();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -306,12 +322,8 @@ quant_act_large_kernel(const __half* __restrict__ X, const float* __restrict__ s
             int nt = warp + t * 8;
             if (nt < ntiles) {
                 int j = nt * 8 + tq * 2;
-                if (m0 + g < M)
-                    *reinterpret_cast<__nv_bfloat162*>(T + (size_t)(m0 + g) * r + j) =
-                        __floats2bfloat162_rn(acc[t][0], acc[t][1]);
-                if (m0 + g + 8 < M)
-                    *reinterpret_cast<__nv_bfloat162*>(T + (size_t)(m0 + g + 8) * r + j) =
-                        __floats2bfloat162_rn(acc[t][2], acc[t][3]);
+                if (m0 + g < M) store_t2(T + (size_t)(m0 + g) * ldt, j, acc[t][0], acc[t][1], lo_off);
+                if (m0 + g + 8 < M) store_t2(T + (size_t)(m0 + g + 8) * ldt, j, acc[t][2], acc[t][3], lo_off);
             }
         }
     }
@@ -368,7 +380,7 @@ constexpr int kTMaxRank = 128;              // larger r takes the mma.sync kerne
 constexpr int kXAtomBytes = kTTok * 128;    // 64 rows x 64 fp16
 constexpr int kXStageBytes = 2 * kXAtomBytes;
 constexpr int kOutTileBytes = kTTok * kTCols;   // 64 rows x 128 int8
-constexpr long long kQaWaitLimitClocks = 4000000000ll;   // about 2 s of SM clocks per wait
+constexpr long long kQaWaitLimitClocks = 400000000ll;   // about 0.2 s of SM clocks per wait
 
 // Ring depth: as many stages (activation tile + L_A tile) as fit beside the exchange buffers.
 // A stage takes about 3 k cycles to go round (HBM latency plus the hand-overs between TMA,
@@ -575,7 +587,7 @@ __global__ void __launch_bounds__(kTThreads, 1)
 quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_la,
                      const __grid_constant__ CUtensorMap map_q, const float* __restrict__ s,
                      int M, int K, int Kc, int r, int CK, float* __restrict__ a_scale,
-                     __nv_bfloat16* __restrict__ T, int ldt, float qmax) {
+                     __nv_bfloat16* __restrict__ T, int ldt, int lo_off, float qmax) {
     extern __shared__ uint8_t smem_raw[];
     grid_dep_launch();      // a dependent linear kernel may start streaming its weights
     const uint32_t sraw = smem_u32(smem_raw);
@@ -849,7 +861,7 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                     for (int e = 0; e < 16; ++e) {
                         const int t = t0 + e;
                         if (CK > 1) t_stage[t * r + j] = __uint_as_float(v[e]);
-                        else if (m0 + t < M) T[(size_t)(m0 + t) * ldt + j] = __float2bfloat16_rn(__uint_as_float(v[e]));
+                        else if (m0 + t < M) store_t(T + (size_t)(m0 + t) * ldt, j, __uint_as_float(v[e]), lo_off);
                     }
                 }
             }
@@ -945,8 +957,7 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                     const float2 pv = *reinterpret_cast<const float2*>(t_slots + (qq * rows_owned + tl) * r + col);
                     s0 += pv.x; s1 += pv.y;
                 }
-                if (m0 + t < M)
-                    *reinterpret_cast<__nv_bfloat162*>(T + (size_t)(m0 + t) * ldt + col) = __floats2bfloat162_rn(s0, s1);
+                if (m0 + t < M) store_t2(T + (size_t)(m0 + t) * ldt, col, s0, s1, lo_off);
             }
         }
         if (*abort_flag && warp == 0) {     // a wait gave up: poison the rows
@@ -970,14 +981,17 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
 // Opts the kernel in to `smem` bytes of dynamic shared memory (the one place that does it, so
 // that the value last set is known).
 int tma_set_smem(size_t smem) {
-    static size_t current = 0;
-    if (smem == current) return ASER_OK;
+    static size_t current[kMaxDevices] = {0};
+    int dev = 0;
+    const int rc = current_device(&dev);
+    if (rc != ASER_OK) return rc;
+    if (smem == current[dev]) return ASER_OK;
     cudaError_t e = cudaFuncSetAttribute(quant_act_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) {
-        current = 0;
+        current[dev] = 0;
         return record_cuda_error(e, "quant_act_tma smem attribute");
     }
-    current = smem;
+    current[dev] = smem;
     return ASER_OK;
 }
 
@@ -985,8 +999,12 @@ int tma_set_smem(size_t smem) {
 // schedule that size).  Queried once per (size, shared memory) pair.  The query counts with
 // the kernel's opted-in maximum of dynamic shared memory, so that is set to the size asked for.
 int tma_active_clusters(int ck, size_t smem) {
-    static int cached[17];
-    static size_t cached_smem[17];
+    static int cached_all[kMaxDevices][17];
+    static size_t cached_smem_all[kMaxDevices][17];
+    int dev = 0;
+    if (current_device(&dev) != ASER_OK) return 0;
+    int* cached = cached_all[dev];
+    size_t* cached_smem = cached_smem_all[dev];
     if (cached_smem[ck] == smem && smem != 0) return cached[ck];
     if (tma_set_smem(smem) != ASER_OK) {
         (void)cudaGetLastError();
@@ -1034,15 +1052,21 @@ int pick_tma_cluster(int M, int K, int r, int max_ck) {
 }
 
 int launch_tma(const __half* X, const float* s, const __half* LA, int M, int K, int r,
-               int8_t* Xq, float* a_scale, __nv_bfloat16* T, int ldt, float qmax, cudaStream_t st,
-               bool* unsupported) {
+               int8_t* Xq, float* a_scale, __nv_bfloat16* T, int ldt, int lo_off, float qmax,
+               cudaStream_t st, bool* unsupported) {
     *unsupported = false;
-    static int max_ck = 0;      // 16 where the device allows clusters beyond the portable 8
-    if (max_ck == 0) {
+    static int max_ck_all[kMaxDevices] = {0};   // 16 where the device allows clusters beyond the portable 8
+    int dev = 0;
+    {
+        const int rc = current_device(&dev);
+        if (rc != ASER_OK) return rc;
+    }
+    if (max_ck_all[dev] == 0) {
         cudaError_t e = cudaFuncSetAttribute(quant_act_tma_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-        max_ck = (e == cudaSuccess) ? 16 : 8;
+        max_ck_all[dev] = (e == cudaSuccess) ? 16 : 8;
         if (e != cudaSuccess) (void)cudaGetLastError();
     }
+    const int max_ck = max_ck_all[dev];
     if ((M + kTTok - 1) / kTTok > 65535 || r > kTMaxRank) { *unsupported = true; return ASER_OK; }
     const int ck = pick_tma_cluster(M, K, r, max_ck);
     if (ck == 0) { *unsupported = true; return ASER_OK; }
@@ -1076,45 +1100,54 @@ int launch_tma(const __half* X, const float* s, const __half* LA, int M, int K, 
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, quant_act_tma_kernel, mx, mla, mq, s, M, K, kc, r, ck, a_scale, T, ldt, qmax);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, quant_act_tma_kernel, mx, mla, mq, s, M, K, kc, r, ck, a_scale, T, ldt, lo_off, qmax);
     if (e != cudaSuccess) return record_cuda_error(e, "quant_act_tma_kernel");
     return check_launch("quant_act_tma_kernel");
 }
 
 template <int MAXT>
 int launch_large(const __half* X, const float* s, const __half* LA, int M, int K, int r,
-                 int8_t* Xq, float* a_scale, __nv_bfloat16* T, float qmax, cudaStream_t st) {
+                 int8_t* Xq, float* a_scale, __nv_bfloat16* T, int ldt, int lo_off, float qmax,
+                 cudaStream_t st) {
     size_t smem = 2 * (size_t)(kTileM + r) * kRowBytes;
-    static size_t configured = 0;   // largest dynamic shared memory size opted into so far
-    if (smem > configured) {
+    static size_t configured[kMaxDevices] = {0};   // largest dynamic shared memory size opted into so far
+    int dev = 0;
+    const int drc = current_device(&dev);
+    if (drc != ASER_OK) return drc;
+    if (smem > configured[dev]) {
         cudaError_t e = cudaFuncSetAttribute(quant_act_large_kernel<MAXT>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return record_cuda_error(e, "quant_act_large smem attribute");
-        configured = smem;
+        configured[dev] = smem;
     }
     int grid = (M + kTileM - 1) / kTileM;
-    quant_act_large_kernel<MAXT><<<grid, kLargeThreads, smem, st>>>(X, s, LA, M, K, r, Xq, a_scale, T, qmax);
+    quant_act_large_kernel<MAXT><<<grid, kLargeThreads, smem, st>>>(X, s, LA, M, K, r, Xq, a_scale, T, ldt, lo_off, qmax);
     return check_launch("quant_act_large_kernel");
 }
 
 }  // namespace
 
 int launch_quant_act(const __half* X, const float* s, const __half* LA, int M, int K, int r,
-                     int8_t* Xq, float* a_scale, __nv_bfloat16* T, cudaStream_t st, int act_bits) {
+                     int8_t* Xq, float* a_scale, __nv_bfloat16* T, cudaStream_t st, int act_bits,
+                     bool t_pair) {
     // symmetric codes of act_bits bits in the int8 container: +-127 for 8 bits, +-31 for 6
     const float qmax = (float)((1 << (act_bits - 1)) - 1);
     if (M == 0) return ASER_OK;
+    const int ldt = t_pair ? 2 * r : r, lo_off = t_pair ? r : 0;
     if (M <= 32) {
         size_t smem = (size_t)K * sizeof(float);
-        static size_t configured = 48 * 1024;
-        if (smem > configured) {
+        static size_t configured[kMaxDevices] = {0};   // beyond the 48 KiB every kernel may use
+        int dev = 0;
+        const int drc = current_device(&dev);
+        if (drc != ASER_OK) return drc;
+        if (smem > 48 * 1024 && smem > configured[dev]) {
             cudaError_t e = cudaFuncSetAttribute(quant_act_small_kernel,
                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return record_cuda_error(e, "quant_act_small smem attribute");
-            configured = smem;
+            configured[dev] = smem;
         }
         dim3 grid(1 + (r + kRowsPerCta - 1) / kRowsPerCta, M);
-        quant_act_small_kernel<<<grid, kSmallThreads, smem, st>>>(X, s, LA, M, K, r, Xq, a_scale, T, qmax);
+        quant_act_small_kernel<<<grid, kSmallThreads, smem, st>>>(X, s, LA, M, K, r, Xq, a_scale, T, ldt, lo_off, qmax);
         return check_launch("quant_act_small_kernel");
     }
     bool unsupported = false;
@@ -1123,22 +1156,22 @@ int launch_quant_act(const __half* X, const float* s, const __half* LA, int M, i
         // columns of T.  Both write the same codes and scales (the arithmetic is deterministic),
         // which costs one extra sweep over X but keeps the projection on the tensor cores.
         const int r1 = r - kTMaxRank;
-        int rc = launch_tma(X, s, LA, M, K, kTMaxRank, Xq, a_scale, T, r, qmax, st, &unsupported);
+        int rc = launch_tma(X, s, LA, M, K, kTMaxRank, Xq, a_scale, T, ldt, lo_off, qmax, st, &unsupported);
         if (!unsupported) {
             if (rc != ASER_OK) return rc;
-            rc = launch_tma(X, s, LA + (size_t)kTMaxRank * K, M, K, r1, Xq, a_scale, T + kTMaxRank, r, qmax, st,
-                            &unsupported);
+            rc = launch_tma(X, s, LA + (size_t)kTMaxRank * K, M, K, r1, Xq, a_scale, T + kTMaxRank, ldt, lo_off,
+                            qmax, st, &unsupported);
             // the shape test is the same for both halves, so the second cannot be refused alone
             if (!unsupported) return rc;
             return record_cuda_error(cudaErrorUnknown, "quant_act: second half refused");
         }
-        return launch_large<4>(X, s, LA, M, K, r, Xq, a_scale, T, qmax, st);
+        return launch_large<4>(X, s, LA, M, K, r, Xq, a_scale, T, ldt, lo_off, qmax, st);
     }
-    const int rc = launch_tma(X, s, LA, M, K, r, Xq, a_scale, T, r, qmax, st, &unsupported);
+    const int rc = launch_tma(X, s, LA, M, K, r, Xq, a_scale, T, ldt, lo_off, qmax, st, &unsupported);
     if (!unsupported) return rc;
-    if (r <= 64) return launch_large<1>(X, s, LA, M, K, r, Xq, a_scale, T, qmax, st);
-    if (r <= 128) return launch_large<2>(X, s, LA, M, K, r, Xq, a_scale, T, qmax, st);
-    return launch_large<4>(X, s, LA, M, K, r, Xq, a_scale, T, qmax, st);
+    if (r <= 64) return launch_large<1>(X, s, LA, M, K, r, Xq, a_scale, T, ldt, lo_off, qmax, st);
+    if (r <= 128) return launch_large<2>(X, s, LA, M, K, r, Xq, a_scale, T, ldt, lo_off, qmax, st);
+    return launch_large<4>(X, s, LA, M, K, r, Xq, a_scale, T, ldt, lo_off, qmax, st);
 }
 
 }  // namespace aser

@@ -3,6 +3,7 @@
 // Shared by the kernels that use them; everything here is inline.
 #pragma once
 #include <cuda.h>
+#include <string.h>
 
 #include "aser_common.cuh"
 
@@ -191,22 +192,67 @@ inline EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
-// 2-D row-major tensor [rows, cols] of `esize`-byte elements, box = [box_rows, box_cols] with
-// the given shared-memory swizzle; out-of-range elements read as zero and are not written.
+// A tensor map depends only on the address, shape, strides, box and modes it was encoded for,
+// never on the tensor's contents, so a map encoded once can serve every later launch with the
+// same arguments.  encode_tiled keeps the most recent maps of the calling thread in a small
+// direct-mapped table (a layer's buffers come back call after call) and spares the hot path the
+// driver's encoder.
+struct MapKey {
+    const void* base;
+    uint64_t dims[3];
+    uint64_t strides[2];
+    uint32_t box[3];
+    uint32_t dtype, rank, swizzle;
+};
+
+inline int encode_tiled(CUtensorMap* map, const MapKey& key, const char* what) {
+    struct Entry { MapKey key; CUtensorMap map; bool used; };
+    constexpr int kEntries = 256;
+    static thread_local Entry table[kEntries];
+    uint64_t h = 1469598103934665603ull;
+    const unsigned char* kb = reinterpret_cast<const unsigned char*>(&key);
+    for (size_t i = 0; i < sizeof(MapKey); ++i) h = (h ^ kb[i]) * 1099511628211ull;
+    Entry& e = table[(h ^ (h >> 32)) % kEntries];
+    if (e.used && memcmp(&e.key, &key, sizeof(MapKey)) == 0) { *map = e.map; return ASER_OK; }
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return record_cuda_error(cudaErrorUnknown, "cuTensorMapEncodeTiled unavailable");
+    cuuint64_t dims[3] = {key.dims[0], key.dims[1], key.dims[2]};
+    cuuint64_t strides[2] = {key.strides[0], key.strides[1]};
+    cuuint32_t box[3] = {key.box[0], key.box[1], key.box[2]};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(map, (CUtensorMapDataType)key.dtype, key.rank, const_cast<void*>(key.base), dims,
+                    strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, (CUtensorMapSwizzle)key.swizzle,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return record_cuda_error(cudaErrorInvalidValue, what);
+    e.key = key; e.map = *map; e.used = true;
+    return ASER_OK;
+}
+
+inline MapKey make_key(const void* base, CUtensorMapDataType dt, uint32_t rank, CUtensorMapSwizzle sw) {
+    MapKey k;
+    memset(&k, 0, sizeof(k));       // padding bytes take part in the comparison
+    k.base = base; k.dtype = (uint32_t)dt; k.rank = rank; k.swizzle = (uint32_t)sw;
+    return k;
+}
+
+// 2-D row-major tensor [rows, cols] of `esize`-byte elements whose rows are `ld` elements apart
+// (a column range of a wider matrix), box = [box_rows, box_cols] with the given shared-memory
+// swizzle; out-of-range elements read as zero and are not written.
+inline int encode_map_2d_ld(CUtensorMap* map, CUtensorMapDataType dt, int esize, const void* base,
+                            uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows,
+                            uint32_t box_cols, CUtensorMapSwizzle swizzle) {
+    MapKey k = make_key(base, dt, 2, swizzle);
+    k.dims[0] = cols; k.dims[1] = rows;
+    k.strides[0] = ld * (uint64_t)esize;
+    k.box[0] = box_cols; k.box[1] = box_rows;
+    return encode_tiled(map, k, "cuTensorMapEncodeTiled");
+}
+
+// The same with contiguous rows.
 inline int encode_map_2d(CUtensorMap* map, CUtensorMapDataType dt, int esize, const void* base,
                          uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t box_cols,
                          CUtensorMapSwizzle swizzle) {
-    EncodeTiledFn fn = get_encode_fn();
-    if (!fn) return record_cuda_error(cudaErrorUnknown, "cuTensorMapEncodeTiled unavailable");
-    cuuint64_t dims[2] = {cols, rows};
-    cuuint64_t strides[1] = {cols * (uint64_t)esize};
-    cuuint32_t box[2] = {box_cols, box_rows};
-    cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return record_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
-    return ASER_OK;
+    return encode_map_2d_ld(map, dt, esize, base, rows, cols, cols, box_rows, box_cols, swizzle);
 }
 
 // Row-major tensor [rows, cols] of `esize`-byte elements viewed as 128-byte column blocks:
@@ -215,18 +261,12 @@ inline int encode_map_2d(CUtensorMap* map, CUtensorMapDataType dt, int esize, co
 // of the MMA descriptors).  Coordinates: (0, row, block).
 inline int encode_map_blocks(CUtensorMap* map, CUtensorMapDataType dt, int esize, const void* base,
                              uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t box_blocks) {
-    EncodeTiledFn fn = get_encode_fn();
-    if (!fn) return record_cuda_error(cudaErrorUnknown, "cuTensorMapEncodeTiled unavailable");
     const uint64_t per_block = 128 / (uint64_t)esize;
-    cuuint64_t dims[3] = {per_block, rows, cols / per_block};
-    cuuint64_t strides[2] = {cols * (uint64_t)esize, 128};
-    cuuint32_t box[3] = {(cuuint32_t)per_block, box_rows, box_blocks};
-    cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = fn(map, dt, 3, const_cast<void*>(base), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return record_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled (blocks)");
-    return ASER_OK;
+    MapKey k = make_key(base, dt, 3, CU_TENSOR_MAP_SWIZZLE_128B);
+    k.dims[0] = per_block; k.dims[1] = rows; k.dims[2] = cols / per_block;
+    k.strides[0] = cols * (uint64_t)esize; k.strides[1] = 128;
+    k.box[0] = (uint32_t)per_block; k.box[1] = box_rows; k.box[2] = box_blocks;
+    return encode_tiled(map, k, "cuTensorMapEncodeTiled (blocks)");
 }
 
 }  // namespace aser

@@ -13,8 +13,12 @@ pytestmark = pytest.mark.gpu
 
 @pytest.fixture(scope="module")
 def aser(cuda_device):
+    import os
     import paper_2411_07762_b200 as aser
-    return aser
+    # the oracle's row loops are independent: all host cores for the full-size cases
+    F.set_threads(len(os.sched_getaffinity(0)))
+    yield aser
+    F.set_threads(1)
 
 
 def bits(a):
@@ -92,7 +96,7 @@ def test_quant_act_parity(aser, M, K, r):
     assert np.array_equal(bits(sc.cpu().numpy()), bits(sc_ref))
     if r:
         T_ref = F.down_proj(xs, L_A)
-        assert_T_close(T.float().cpu().numpy(), T_ref)
+        assert_T_close(T.float().cpu().numpy(), T_ref, xs, L_A)
 
 
 @pytest.mark.parametrize("M,K,r", [(8, 1024, 16), (300, 1024, 64), (2048, 512, 32)])
@@ -109,7 +113,7 @@ def test_quant_act_dense_smoothing_vector(aser, M, K, r):
     Xq, sc, T = aser.quant_act(to_dev(lay.X), to_dev(s), to_dev(L_A))
     assert np.array_equal(Xq.cpu().numpy(), Xq_ref)
     assert np.array_equal(bits(sc.cpu().numpy()), bits(sc_ref))
-    assert_T_close(T.float().cpu().numpy(), F.down_proj(xs, L_A))
+    assert_T_close(T.float().cpu().numpy(), F.down_proj(xs, L_A), xs, L_A)
 
 
 def test_quant_act_without_smoothing_vector(aser):
@@ -123,7 +127,13 @@ def test_quant_act_without_smoothing_vector(aser):
 # whole path: quant_act -> linear
 # ---------------------------------------------------------------------------
 def run_path(aser, lay, s, Wq_ref, w_scale_ref, L_A, L_B, impl, rows=None, use_dgemm=False,
-             large_lowrank_term=False):
+             t_pair=False, timed_config=False, ws=None, ref=None):
+    """Pack, quantize and multiply on the GPU, run the oracle on the same arrays, compare every
+    stage.  `rows`: the oracle's products cover these token rows only (None = all).
+    `t_pair`: T as bf16 pairs with the up projection written twice.  `timed_config`: the linear
+    kernel runs once more without the accumulator dump (the configuration that is timed) and
+    that output is compared with the oracle as well.  `ws`: a caller-owned workspace (reuse
+    across calls).  `ref`: a precomputed oracle result for these inputs."""
     M, K = lay.X.shape
     N = lay.W.shape[0]
     r = 0 if L_A is None else L_A.shape[0]
@@ -131,45 +141,48 @@ def run_path(aser, lay, s, Wq_ref, w_scale_ref, L_A, L_B, impl, rows=None, use_d
     Wq, wsc = aser.pack_w4(dW, ds)
     assert np.array_equal(Wq.cpu().numpy(), Wq_ref)
     assert np.array_equal(bits(wsc.cpu().numpy()), bits(w_scale_ref))
+    del dW
     dLA = None if r == 0 else to_dev(L_A)
     dLB = None if r == 0 else to_dev(L_B)
-    Xq, sc, T = aser.quant_act(to_dev(lay.X), ds, dLA)
+    Xq, sc, T = aser.quant_act(to_dev(lay.X), ds, dLA, t_pair=t_pair)
+    if t_pair:
+        dLB = aser.pair_up_projection(dLB)
+    r_lin = 2 * r if t_pair else r
     acc = torch.full((M, N), -7, dtype=torch.int32, device="cuda")
+    Y_timed = None
     if impl == "simt":
         Y = aser.linear_w4a8_lr_simt(Xq, sc, Wq, wsc, T, dLB, acc_debug=acc)
     else:
         Wk = aser.repack_w4(Wq)
-        ws = aser.new_workspace(M, N, K, r)
-        if r:
-            Y = aser.linear_w4a8_lr(Xq, sc, Wk, wsc, T, dLB, N, ws, acc_debug=acc)
-        else:
-            Y = aser.linear_w4a8(Xq, sc, Wk, wsc, N, ws, acc_debug=acc)
+        if ws is None:
+            ws = aser.new_workspace(M, N, K, r_lin)
+
+        def call(acc_debug):
+            if r:
+                return aser.linear_w4a8_lr(Xq, sc, Wk, wsc, T, dLB, N, ws, acc_debug=acc_debug)
+            return aser.linear_w4a8(Xq, sc, Wk, wsc, N, ws, acc_debug=acc_debug)
+        Y = call(acc)
+        if timed_config:
+            Y_timed = call(None)
         aser.check_status(ws)
     torch.cuda.synchronize()
-    ref = F.forward(lay.X, s, Wq_ref, w_scale_ref, L_A, L_B, rows=rows, use_dgemm=use_dgemm)
+    if ref is None:
+        ref = F.forward(lay.X, s, Wq_ref, w_scale_ref, L_A, L_B, rows=rows, use_dgemm=use_dgemm)
     assert np.array_equal(Xq.cpu().numpy(), ref.Xq)
     assert np.array_equal(bits(sc.cpu().numpy()), bits(ref.a_scale))
     acc_h = acc.cpu().numpy()
     assert np.array_equal(acc_h if rows is None else acc_h[rows], ref.acc)
-    if large_lowrank_term:
-        # The bound 2e-3 * max|y_ref| budgets the bf16 rounding of T (2^-9 relative) for a low-rank
-        # term that is a few per cent of y.  Where the factors carry whole weight columns that no
-        # longer holds; the rounding of T then adds up to 2^-9 * sum_j |L_B[n,j]| |T[m,j]| (2^-8
-        # with the fp16 rounding of x~ in the tensor-core projection), which is allowed on top.
-        y_gpu = Y.cpu().numpy().astype(np.float64)
-        if rows is not None:
-            y_gpu = y_gpu[rows]
-        slack = 2.0 ** -8 * (np.abs(ref.T) @ np.abs(L_B.astype(np.float64)).T)
-        bound = 2e-3 * np.abs(ref.y).max(axis=1, keepdims=True) + slack
-        assert np.all(np.abs(y_gpu - ref.y) <= bound)
-    else:
-        assert_rows_close(Y.cpu().numpy(), ref.y, rows)
+    assert_rows_close(Y.cpu().numpy(), ref.y, rows)
+    if Y_timed is not None:
+        assert_rows_close(Y_timed.cpu().numpy(), ref.y, rows)
     return Y
 
 
 PATH_CASES = [  # M, N, K, r
     (16, 512, 512, 16), (1, 256, 512, 16), (7, 136, 1024, 32), (33, 264, 512, 0),
     (130, 384, 1024, 64), (257, 520, 2048, 128), (40, 128, 384, 256),
+    # 17..32 tokens: the 32-token tile of the tensor-core kernel
+    (19, 264, 1024, 32), (32, 384, 512, 16), (17, 1152, 2048, 64),
 ]
 
 
@@ -181,7 +194,7 @@ def test_path_parity_small(aser, impl, M, N, K, r):
     s, Wq, w_scale, L_A, L_B = oracle_layer(lay, r, construct=(K <= 1024 and r > 0))
     if r == 0:
         L_A = L_B = None
-    run_path(aser, lay, s, Wq, w_scale, L_A, L_B, impl)
+    run_path(aser, lay, s, Wq, w_scale, L_A, L_B, impl, timed_config=(impl == "tc"))
 
 
 @pytest.mark.parametrize("impl", ["simt", "tc"])
@@ -202,16 +215,17 @@ def test_config1_tiny_with_constructed_factors(aser, impl):
 def test_config2_decode_full_size(aser, impl, M):
     lay, r = synth.config2_decode(M)
     s, Wq, w_scale, L_A, L_B = oracle_layer(lay, r, construct=(M == 8))
-    run_path(aser, lay, s, Wq, w_scale, L_A, L_B, impl, use_dgemm=True)
+    run_path(aser, lay, s, Wq, w_scale, L_A, L_B, impl, use_dgemm=True, timed_config=True)
 
 
 @pytest.mark.parametrize("impl", ["tc"])
 @pytest.mark.parametrize("which", ["gate_up", "down"])
-def test_config3_prefill_full_size_sampled_rows(aser, impl, which):
+def test_config3_prefill_full_size_all_rows(aser, impl, which):
+    """Both prefill layers at full size: every accumulator bit-exact and every output element
+    within the bound, with and without the accumulator dump (the timed configuration)."""
     lay, r = synth.config3_prefill(which)
     s, Wq, w_scale, L_A, L_B = oracle_layer(lay, r, construct=False)
-    rows = np.array([0, 1, 127, 128, 1000, 1023, 1024, 2046, 2047])
-    run_path(aser, lay, s, Wq, w_scale, L_A, L_B, impl, rows=rows, use_dgemm=True)
+    run_path(aser, lay, s, Wq, w_scale, L_A, L_B, impl, use_dgemm=True, timed_config=True)
 
 
 FORWARD_CASES = [  # M, N, K, r
@@ -249,27 +263,53 @@ def test_forward_overlapped_is_bit_identical_to_separate_calls(aser, M, N, K, r)
     aser.check_status(layer.ws)
 
 
-@pytest.mark.parametrize("name", ["k", "gate", "down"])
-def test_config4_block_linears_full_size_sampled_rows(aser, name):
-    """Decoder-block linears at 4096 tokens, rank 128 (the GQA projection, the widest and the
-    deepest layer): every int8 code and scale, and Y on sampled token rows."""
+@pytest.mark.parametrize("name", ["q", "k", "gate", "down"])
+def test_config4_block_linears_full_size_all_rows(aser, name):
+    """Decoder-block linears at 4096 tokens, rank 128 (the square projection with eight whole
+    tiles per CTA, the GQA projection, the widest and the deepest layer): every code, scale,
+    accumulator and output element.  The widest layer also runs a 32-token call first on the
+    workspace sized for 4096 tokens: one workspace serves calls of different shapes in turn."""
     lay, r = synth.config4_block_layer(name)
     s, Wq, w_scale, L_A, L_B = oracle_layer(lay, r, construct=False)
-    rows = np.array([0, 63, 64, 2047, 2048, 4031, 4095])
-    run_path(aser, lay, s, Wq, w_scale, L_A, L_B, "tc", rows=rows, use_dgemm=True)
+    ref = F.forward(lay.X, s, Wq, w_scale, L_A, L_B, use_dgemm=True)
+    M, K = lay.X.shape
+    N = lay.W.shape[0]
+    ws = aser.new_workspace(M, N, K, r)
+    if name == "gate":
+        m = 32
+        small = synth.LayerInputs(X=lay.X[:m], W=lay.W, X_cal=lay.X_cal, outlier_idx=lay.outlier_idx,
+                                  outlier_gain=lay.outlier_gain, meta=lay.meta)
+        ref_small = F.ForwardResult(xs=ref.xs[:m], Xq=ref.Xq[:m], a_scale=ref.a_scale[:m],
+                                    acc=ref.acc[:m], T=ref.T[:m], y=ref.y[:m], rows=None)
+        run_path(aser, small, s, Wq, w_scale, L_A, L_B, "tc", ws=ws, ref=ref_small)
+    run_path(aser, lay, s, Wq, w_scale, L_A, L_B, "tc", ws=ws, ref=ref, timed_config=True)
+    if name == "gate":     # and back to the small shape on the same workspace
+        run_path(aser, small, s, Wq, w_scale, L_A, L_B, "tc", ws=ws, ref=ref_small)
 
 
-@pytest.mark.parametrize("M,N,r", [(16, 8192, 32), (16, 28672, 64), (128, 28672, 256), (1024, 8192, 128), (4096, 8192, 0)])
-def test_config5_sweep_points_sampled_rows(aser, M, N, r):
-    """Points of the 70B-class sweep (K = 8192): 16 tokens on both few-token paths (streaming
-    kernel up to 64 MB of packed weights, tensor-core kernel above), rank 256 (two launches of the
-    quantization cluster kernel) and rank 0 (plain W4A8)."""
+C5_POINTS = [  # M, N, r, all rows?
+    (1, 8192, 64, True), (16, 8192, 32, True), (16, 28672, 64, True), (128, 8192, 0, True),
+    (128, 28672, 256, True), (1024, 8192, 128, True), (1024, 28672, 32, False),
+    (4096, 8192, 128, True), (4096, 8192, 0, False), (4096, 28672, 64, True),
+]
+
+
+@pytest.mark.parametrize("M,N,r,full", C5_POINTS)
+def test_config5_sweep_points(aser, M, N, r, full):
+    """Points of the 70B-class sweep (K = 8192): few tokens on both few-token paths (streaming
+    kernel up to 64 MB of packed weights, tensor-core kernel above), rank 256 (two launches of
+    the quantization cluster kernel), rank 0 (plain W4A8), and 4096 tokens at both widths
+    compared on every row (the remaining points on token rows spread over every 128-token tile)."""
     lay = synth.config5_point(M, N)
     s, Wq, w_scale, L_A, L_B = oracle_layer(lay, r, construct=False)
     if r == 0:
         L_A = L_B = None
-    rows = np.unique(np.array([0, 1, M // 2, M - 2, M - 1]).clip(0, M - 1))
-    run_path(aser, lay, s, Wq, w_scale, L_A, L_B, "tc", rows=rows, use_dgemm=True)
+    rows = None
+    if not full:
+        base = np.arange(0, M, 128)
+        rows = np.unique(np.concatenate([base, base + 127, base + 61]).clip(0, M - 1))
+    run_path(aser, lay, s, Wq, w_scale, L_A, L_B, "tc", rows=rows, use_dgemm=True,
+             timed_config=(M == 4096))
 
 
 @pytest.mark.gpu
@@ -297,15 +337,21 @@ def test_rank_not_a_multiple_of_16_is_padded_with_zeros(aser, M, N, K, r):
 
 
 @pytest.mark.gpu
-def test_paper_smoothing_rule_with_outlier_split_runs_through_the_same_path(aser):
-    """The paper's own variant (Sec. 4.2): m_i = X-bar_i / min over the f outlier channels, and the
-    outlier columns W_o kept out of the int4 matrix and carried by the low-rank factors.  For the
-    GPU this is the same path with different inputs: the caller zeroes the outlier columns of W
-    before packing.  Packed weights and accumulators bit-exact; the output within the bound plus
-    the bf16 rounding of T, whose term is now as large as the outlier columns' contribution; and
-    the split layer's output is closer to the fp product than plain W4A8 on the same codes."""
+@pytest.mark.parametrize("M", [16, 200])
+def test_paper_smoothing_rule_with_outlier_split_runs_through_the_same_path(aser, M):
+    """The paper's own variant (Sec. 4.2): m_i = X-bar_i / min over the f outlier channels
+    (Eq. 11), and the outlier columns W_o kept out of the int4 matrix and carried by the low-rank
+    factors (Eq. 12).  For the GPU this is the same path with different inputs: the caller zeroes
+    the outlier columns of W before packing.  The low-rank term is then as large as the output,
+    so T is stored as bf16 pairs (aser_quant_act_ex); with that the output meets the same
+    2e-3 * max|y_ref| bound as everywhere else.  Packed weights and accumulators bit-exact; and
+    the split layer's output is closer to the fp product than plain W4A8 on the same codes.
+    M = 16 takes the few-token kernels, M = 200 the tensor-core kernels."""
     from oracle import construct as Cn
     lay, r = synth.config1_tiny()
+    if M != 16:
+        lay = synth.make_layer(M, 512, 512, seed=synth.seed_for(1, M), n_out=4, outlier_gain=40.0,
+                               sigma_w=0.02, n_cal=128)
     s, idx = Cn.smoothing_vector_paper(lay.X_cal, lay.W, f=4)
     assert np.array_equal(idx, lay.outlier_idx)
     L = Cn.construct_layer(lay.W, lay.X_cal, s, r=r, split_outliers=idx)
@@ -313,12 +359,85 @@ def test_paper_smoothing_rule_with_outlier_split_runs_through_the_same_path(aser
     W_split[:, idx] = 0
     lay_split = synth.LayerInputs(X=lay.X, W=W_split, X_cal=lay.X_cal, outlier_idx=lay.outlier_idx,
                                   outlier_gain=lay.outlier_gain, meta=lay.meta)
-    Y = run_path(aser, lay_split, s, L.Wq, L.w_scale, L.L_A, L.L_B, "tc", large_lowrank_term=True)
+    Y = run_path(aser, lay_split, s, L.Wq, L.w_scale, L.L_A, L.L_B, "tc", t_pair=True,
+                 timed_config=True)
     plain = run_path(aser, lay_split, s, L.Wq, L.w_scale, None, None, "tc")
     ref = lay.X.astype(np.float64) @ lay.W.astype(np.float64).T
     e_lr = np.linalg.norm(Y.cpu().numpy().astype(np.float64) - ref)
     e_plain = np.linalg.norm(plain.cpu().numpy().astype(np.float64) - ref)
     assert e_lr < 0.5 * e_plain        # without the factors the outlier columns are simply missing
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("M,K,r", [(8, 1024, 16), (300, 2048, 64), (129, 4096, 128), (40, 512, 48)])
+def test_quant_act_pair_storage_of_T(aser, M, K, r):
+    """aser_quant_act_ex with t_pair: hi + lo reproduces the fp64 projection to 2^-16 of each
+    entry (plus the fp16 rounding of x~ inside the tensor-core product), codes and scales are
+    those of the plain call, and hi is the plain call's T."""
+    lay = synth.make_layer(M, 8, K, seed=800 + M + K + r, n_cal=8)
+    s = synth.standin_smoothing_vector(K, lay.outlier_idx, 13.0)
+    L_A = synth.standin_factors(8, K, r, seed=M, scale_a=0.05)[0]
+    dX, ds, dLA = to_dev(lay.X), to_dev(s), to_dev(L_A)
+    Xq0, sc0, T0 = aser.quant_act(dX, ds, dLA)
+    Xq, sc, T = aser.quant_act(dX, ds, dLA, t_pair=True)
+    assert T.shape == (M, 2 * r)
+    assert torch.equal(Xq, Xq0) and torch.equal(sc, sc0)
+    assert torch.equal(T[:, :r].contiguous().view(torch.int16), T0.view(torch.int16))
+    xs = F.smooth_act(lay.X, s)
+    T_ref = F.down_proj(xs, L_A)
+    T_sum = T[:, :r].double().cpu().numpy() + T[:, r:].double().cpu().numpy()
+    xs64, la64 = xs.astype(np.float64), L_A.astype(np.float64)
+    rms = np.sqrt((xs64 ** 2) @ (la64 ** 2).T)
+    l1 = np.abs(xs64) @ np.abs(la64).T
+    tol = 2.0 ** -16 * np.abs(T_ref) + 2.0 ** -9.2 * rms * (M > 32) + 2.0 ** -20 * l1 + 1e-30
+    assert np.all(np.abs(T_sum - T_ref) <= tol)
+    with pytest.raises(aser.AserError) as err:      # 2 r beyond the kernels' 256
+        aser.quant_act(dX, ds, to_dev(synth.standin_factors(8, K, 144, seed=1)[0]), t_pair=True)
+    assert err.value.code == -3
+
+
+@pytest.mark.gpu
+def test_rank_from_threshold_end_to_end(aser):
+    """Sec. 4.1 Eq. 9 end to end: the oracle picks the rank from the singular-value threshold
+    alpha (any integer, here not a multiple of 16), pad_rank brings the factors to the kernels'
+    granularity, and the GPU output matches the oracle run on the UNPADDED factors."""
+    from oracle import construct as Cn
+    lay = synth.make_layer(48, 384, 512, seed=synth.seed_for(1, 77), n_out=5, outlier_gain=40.0, n_cal=256)
+    s = Cn.smoothing_vector_config(lay.X_cal, lay.W, lay.outlier_idx)
+    seen = set()
+    for alpha in (0.05, 0.12, 0.3):
+        L = Cn.construct_layer(lay.W, lay.X_cal, s, r=None, alpha=alpha)
+        r = L.L_A.shape[0]
+        assert r == Cn.rank_from_alpha(L.sigma, alpha) and 0 < r < 256
+        seen.add(r % 16 != 0)
+        dLA, dLB = aser.pad_rank(to_dev(L.L_A), to_dev(L.L_B))
+        ds = to_dev(s)
+        Wq, wsc = aser.pack_w4(to_dev(lay.W), ds)
+        assert np.array_equal(Wq.cpu().numpy(), L.Wq)
+        Xq, sc, T = aser.quant_act(to_dev(lay.X), ds, dLA)
+        ws = aser.new_workspace(48, 384, 512, dLA.shape[0])
+        acc = torch.zeros((48, 384), dtype=torch.int32, device="cuda")
+        Y = aser.linear_w4a8_lr(Xq, sc, aser.repack_w4(Wq), wsc, T, dLB, 384, ws, acc_debug=acc)
+        aser.check_status(ws)
+        ref = F.forward(lay.X, s, L.Wq, L.w_scale, L.L_A, L.L_B)
+        assert np.array_equal(acc.cpu().numpy(), ref.acc)
+        assert_rows_close(Y.cpu().numpy(), ref.y)
+    assert True in seen                 # at least one rank that needed padding
+
+
+@pytest.mark.gpu
+def test_status_word_reports_a_timeout_and_clears(aser):
+    """aser_check_status without any kernel timing out: a status word planted by a memset must
+    come back as ASER_ERR_DEVICE_TIMEOUT once, then the workspace is clean (word and counters)."""
+    ws = aser.new_workspace(64, 256, 512, 16)
+    aser.check_status(ws)
+    ws[0] = 1
+    ws[256:260] = 3                     # a tile counter left behind by the same launch
+    with pytest.raises(aser.AserError) as err:
+        aser.check_status(ws)
+    assert err.value.code == -6 and "status word" in str(err.value)
+    aser.check_status(ws)
+    assert int(ws[:1024].to(torch.int32).sum()) == 0
 
 
 # ---------------------------------------------------------------------------
@@ -342,7 +461,7 @@ def test_quant_act_6bit_parity(aser, M, K, r):
     assert np.array_equal(bits(sc.cpu().numpy()), bits(sc_ref))
     assert int(Xq.abs().max()) == 31
     if r:
-        assert_T_close(T.float().cpu().numpy(), F.down_proj(xs, L_A))
+        assert_T_close(T.float().cpu().numpy(), F.down_proj(xs, L_A), xs, L_A)
 
 
 @pytest.mark.gpu

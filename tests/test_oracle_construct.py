@@ -221,7 +221,7 @@ def test_smoothing_shrinks_activation_range():
 
 
 def test_outlier_split_variant(small_layer):
-    """W M = W_s + W_o (Eq. 11): the outlier columns are not quantized and move into the
+    """W M = W_s + W_o (Eq. 12): the outlier columns are not quantized and move into the
     SVD target, which then equals W diag(s) - Q(W_s)."""
     lay, s = small_layer
     idx = lay.outlier_idx

@@ -27,7 +27,7 @@ def test_smoothing_divides_each_channel():
 
 
 def test_smoothing_identity_fp64():
-    """W diag(s) diag(s)^-1 X = W X  (Eq. 9 of Sec. 4.2)."""
+    """W diag(s) diag(s)^-1 X = W X  (Eq. 10 of Sec. 4.2)."""
     rng = np.random.default_rng(1)
     X = rng.standard_normal((8, 64)).astype(np.float16)
     W = (rng.standard_normal((32, 64)) * 0.02).astype(np.float16)

@@ -409,11 +409,13 @@ class Model:
         torch.cuda.synchronize()
         return graphs
 
-    def time_region(self, fn, calls, repeats=REPEATS, barrier=None):
+    def time_region(self, fn, calls, repeats=REPEATS, barrier=None, label=""):
         """Median device time of `calls` calls of fn, as ms per call, with the spread.  One
         repeat replays the captured region (back to back, as often as it takes to last
         MIN_REGION_MS) between two CUDA events on the replaying stream."""
         torch = self.torch
+        if os.environ.get("ASER_BENCH_TRACE"):
+            print("region %s %s calls=%d" % (self.name, label, calls), file=sys.stderr, flush=True)
         if self.n_sets > 1:      # a region cycles through every operand set: no set returns early
             calls = -(-calls // self.n_sets) * self.n_sets
         graphs = self.capture(fn, calls)
@@ -499,13 +501,13 @@ def roofline_of(w, name, us_linear, peaks, lib_int8, li=None):
 def measure(m, steps, peaks, lib_int8, barrier=None, max_over_ranks=lambda x: x, per_layer=True):
     """All timed quantities of one workload (ms / us per step or call)."""
     w = m.w
-    t_step = m.time_region(m.step, steps, barrier=barrier)
+    t_step = m.time_region(m.step, steps, barrier=barrier, label="step")
     ms_step = max_over_ranks(t_step["median"])
     calls = max(1, min(steps, 64))
-    t_step_plain = m.time_region(lambda i: m.step(i, False), calls) if m.r else t_step
-    t_lin = m.time_region(m.linear_only, calls)
-    t_lin_plain = m.time_region(lambda i: m.linear_only(i, None, False), calls) if m.r else t_lin
-    t_act = m.time_region(m.quant_only, calls)
+    t_step_plain = m.time_region(lambda i: m.step(i, False), calls, label="step_plain") if m.r else t_step
+    t_lin = m.time_region(m.linear_only, calls, label="linear")
+    t_lin_plain = m.time_region(lambda i: m.linear_only(i, None, False), calls, label="linear_plain") if m.r else t_lin
+    t_act = m.time_region(m.quant_only, calls, label="quant")
     out = dict(ms_step=ms_step, step=t_step,
                us=dict(step=ms_step * 1e3, step_plain=t_step_plain["median"] * 1e3,
                        quant_act=t_act["median"] * 1e3, linear_lr=t_lin["median"] * 1e3,
@@ -519,11 +521,11 @@ def measure(m, steps, peaks, lib_int8, barrier=None, max_over_ranks=lambda x: x,
     if per_layer and len(w["layers"]) > 1:
         rows = []
         for li, (nm, K, N, _) in enumerate(w["layers"]):
-            tl = m.time_region(lambda i: m.linear_only(i, li), calls)
-            tp = m.time_region(lambda i: m.linear_only(i, li, False), calls) if m.r else tl
-            ta = m.time_region(lambda i: m.quant_only(i, li), calls)
-            ts = m.time_region(lambda i: m.layer_step(i, li), calls)
-            tsp = m.time_region(lambda i: m.layer_step(i, li, False), calls) if m.r else ts
+            tl = m.time_region(lambda i: m.linear_only(i, li), calls, label=nm + " linear")
+            tp = m.time_region(lambda i: m.linear_only(i, li, False), calls, label=nm + " linear_plain") if m.r else tl
+            ta = m.time_region(lambda i: m.quant_only(i, li), calls, label=nm + " quant")
+            ts = m.time_region(lambda i: m.layer_step(i, li), calls, label=nm + " step")
+            tsp = m.time_region(lambda i: m.layer_step(i, li, False), calls, label=nm + " step_plain") if m.r else ts
             ops = 2.0 * w["M"] * N * K
             roof = roofline_of(w, m.name, tl["median"] * 1e3, peaks, lib_int8, li)
             rows.append(dict(layer=nm, K=K, N=N, us_step=ts["median"] * 1e3, us_linear_lr=tl["median"] * 1e3,

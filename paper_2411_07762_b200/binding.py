@@ -271,11 +271,7 @@ class AserLinear:
         """One forward pass through aser_forward (quantization and linear kernel overlapped)."""
         M = X.shape[0]
         assert M <= self.max_tokens
-        if not lowrank and self.r:
-            self.quant(X)
-            self.linear(M, False)
-            return self.Y[:M]
-        r = self.r
+        r = self.r if lowrank else 0       # the plain W4A8 control: the same entry point at rank 0
         _chk(lib.aser_forward(_ptr(X), _ptr(self.s), _ptr(self.L_A) if r else None, _ptr(self.Wk),
                               _ptr(self.w_scale), _ptr(self.L_B) if r else None, M, self.N, self.K, r,
                               _ptr(self.Xq), _ptr(self.a_scale), _ptr(self.T) if r else None,

@@ -186,6 +186,17 @@ struct Abort {
     uint32_t* status;     // global
 };
 
+// Debugging aid: a role of the CTA whose wait gave up first leaves its progress counters in the
+// workspace header (words 8 + 8 * role ...), read by the host after aser_check_status reports
+// the time-out.
+__device__ __noinline__ void dump_role(uint32_t* status, int role, uint32_t a, uint32_t b, uint32_t c,
+                                       uint32_t d, uint32_t e) {
+    for (int spin = 0; spin < 100000 && ((volatile uint32_t*)status)[5] == 0u; ++spin) {}
+    if (((volatile uint32_t*)status)[2] != blockIdx.x) return;
+    uint32_t* w = status + 8 + 6 * role;
+    w[0] = 0xD0000000u | threadIdx.x; w[1] = a; w[2] = b; w[3] = c; w[4] = d; w[5] = e;
+}
+
 // Slow path of a bounded wait, kept out of line so that the role loops stay small (the kernel
 // runs six different instruction streams per SM and lives or dies by its instruction cache).
 __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* flag,
@@ -200,6 +211,14 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volat
             } else if (clock64() - t0 > kWaitLimitClocks) {
                 *flag = 1;
                 atomicOr(status, kStatusTimeout);
+                // where the first wait gave up (debugging aid): header words 1..5
+                if (atomicCAS(status + 1, 0u, 0x80000000u | threadIdx.x) == 0u) {
+                    status[2] = blockIdx.x;
+                    status[3] = (bar & 1023u) >> 3;     // index of the barrier
+                    status[4] = parity;
+                    __threadfence();
+                    status[5] = 1u;                     // record complete
+                }
                 return false;
             }
         }
@@ -357,6 +376,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             while (w_ok && w_issue_one()) {}
             const uint32_t cw = wcw;
             const bool ok = w_ok;
+            if (*abort_flag) dump_role(p.status, 0, cw, (uint32_t)wkb, (uint32_t)ww.tile, (uint32_t)ww.kb0, (uint32_t)ww.kb1);
             if (!ok || *abort_flag) {
                 // let copies already issued land before the CTA's shared memory goes away
                 for (uint32_t i = (cw > (uint32_t)C::NW ? cw - C::NW : 0); i < cw; ++i)
@@ -426,6 +446,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     for (int c = early; c < lr_chunks && ok; ++c) ok = issue_lr(c);
                 }
             }
+            if (*abort_flag) dump_role(p.status, 1, cx, cl, (uint32_t)w.tile, (uint32_t)w.kb0, (uint32_t)w.kb1);
             if (!ok || *abort_flag) {
                 // let copies already issued land before the CTA's shared memory goes away
                 for (uint32_t i = (cl > (uint32_t)C::NL ? cl - C::NL : 0); i < cl; ++i)
@@ -518,6 +539,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 if (ok) tc_commit(bar(B_ACC_FULL + buf));
                 ++ci;
             }
+            if (*abort_flag) dump_role(p.status, 2 + issuer, ca, cl, ci, (uint32_t)w.tile, ((uint32_t)w.kb0 << 16) | (uint32_t)w.kb1);
         }
     } else if (warp < 10) {
         // =================== unpack warps: int4 -> int8 (x16) into tensor memory ===================
@@ -613,6 +635,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             if (ok && w.has_lr && group == 0)
                 for (int c = lc; c < lr_chunks && ok; ++c) ok = convert_chunk();
         }
+        if (leader && *abort_flag) dump_role(p.status, 4 + group, cw, cl, 0u, (uint32_t)w.tile, ((uint32_t)w.kb0 << 16) | (uint32_t)w.kb1);
     } else if (warp < 10 + C::EW) {
         // =================== epilogue warps ===================
         const int q = warp & 3;
@@ -791,6 +814,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 }
             }
         }
+        if (et == 0 && *abort_flag) dump_role(p.status, 6, ci, (uint32_t)partial_idx, 0u, (uint32_t)w.tile, ((uint32_t)w.kb0 << 16) | (uint32_t)w.kb1);
     }
 
     // =================== teardown ===================

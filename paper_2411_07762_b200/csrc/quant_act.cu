@@ -619,6 +619,17 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     const uint32_t bar_amax = bar_acc + 8;      // the peers' row maxima have landed
     const uint32_t bar_t = bar_acc + 16;        // the peers' partial T have landed
     constexpr uint32_t kTmemCols = 64;                      // D[j, token]: 64 token columns
+    // The two consumer groups take alternate uses of the ring.  A wait on a phase PARITY is only
+    // sound for a waiter that observes every phase of its barrier.  With an even ring a stage
+    // always comes back to the same group, which therefore sees each of its phases.  With an odd
+    // ring the groups alternate on a stage; a warp that only waited for its own uses could find
+    // the barrier one phase behind (the other group's load still in flight), read that as "my
+    // phase is complete", work on a stage that has not landed and arrive on a barrier out of
+    // turn.  So with an odd ring every consumer warp waits for EVERY use of the ring and the
+    // warps of the idle group hand the stage on at once: the hand-over barriers then count all
+    // sixteen warps.
+    const bool all_observe = (NS & 1) != 0;
+    const uint32_t ring_arrivals = all_observe ? kTConsumerWarps : kTGroupWarps;
 
     // Use i of the ring: i < nst is sweep 1 (X and L_A tiles), the rest sweep 2 (X only).
     // A stage's previous use was released by the MMAs (sweep 1) or the consumers (sweep 2).
@@ -655,9 +666,9 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         if (lane == 0) {
             for (int st = 0; st < kTMaxStages; ++st) {
                 mbar_init(bar_full(st), 1);                     // the producer's expect_tx arrival
-                mbar_init(bar_ready(st), kTGroupWarps);         // the stage's consumer group is done with it
+                mbar_init(bar_ready(st), ring_arrivals);        // the consumers are done with the stage
                 mbar_init(bar_free1(st), 1);                    // sweep 1: the MMAs have read it
-                mbar_init(bar_free2(st), kTGroupWarps);         // sweep 2: the group has read it
+                mbar_init(bar_free2(st), ring_arrivals);        // sweep 2: the consumers have read it
             }
             for (int o = 0; o < kTOut; ++o) {
                 mbar_init(bar_out_full(o), kTGroupWarps);       // an output tile is written
@@ -779,10 +790,14 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         float amax0 = 0.f, amax1 = 0.f;
         __half2 hamax0 = __float2half2_rn(0.f), hamax1 = hamax0;
         bool ok = true;
-        for (int i = grp; i < nst; i += 2) {
+        for (int i = all_observe ? 0 : grp; i < nst; i += all_observe ? 1 : 2) {
             const int st = i % NS;
             ok = qa_warp_wait(bar_full(st), (uint32_t)(i / NS) & 1u, abort_flag, lane);
             if (!ok) break;
+            if ((i & 1) != grp) {           // the other group's use: observed, handed on
+                if (lane == 0) mbar_arrive(bar_ready(st));
+                continue;
+            }
             const uint32_t a0 = sb + L.x_ring + st * kXStageBytes + x_off, a1 = a0 ^ 16u;
             const uint4 v0 = lds128(a0), v1 = lds128(a1);
             const uint4 w0 = lds128(a0 + kRow32), w1 = lds128(a1 + kRow32);
@@ -902,10 +917,14 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         // the wait on the accumulator above says the MMAs are done reading it) ----
         const float rcp0 = (sc0 > 0.f) ? __frcp_rn(sc0) : 0.f;
         const float rcp1 = (sc1 > 0.f) ? __frcp_rn(sc1) : 0.f;
-        for (int jj = grp; jj < nst && ok; jj += 2) {
+        for (int jj = all_observe ? 0 : grp; jj < nst && ok; jj += all_observe ? 1 : 2) {
             const int i = nst + jj, st = i % NS, o = jj % kTOut;
             ok = qa_warp_wait(bar_full(st), (uint32_t)(i / NS) & 1u, abort_flag, lane);
             if (!ok) break;
+            if ((jj & 1) != grp) {          // the other group's use: observed, handed on
+                if (lane == 0) mbar_arrive(bar_free2(st));
+                continue;
+            }
             const uint32_t a0 = sb + L.x_ring + st * kXStageBytes + x_off, a1 = a0 ^ 16u;
             const uint4 v0 = lds128(a0), v1 = lds128(a1);
             const uint4 w0 = lds128(a0 + kRow32), w1 = lds128(a1 + kRow32);

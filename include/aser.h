@@ -117,6 +117,29 @@ int aser_quant_act_ex(const void* X_f16, const float* s, const void* LA_f16,
                       int8_t* Xq, float* a_scale, void* T_bf16, void* stream);
 
 /*
+ * aser_quant_act_ws -- aser_quant_act_ex for callers that can spare scratch memory (same
+ * passages of the paper; the scratch is an implementation matter).  With more than 32 tokens it
+ * runs two kernels instead of one: the first reads X once, takes the row maxima and the
+ * projection T on the tensor cores and leaves per-slice partial results in the scratch; the
+ * second writes the scales, the codes and T.  Results are those of aser_quant_act_ex (Xq and
+ * a_scale bit-exact; T may differ in its last bf16 bit because the fp32 sums are formed in a
+ * different order), at several times the throughput.  Two extensions:
+ *   - r may go up to 512 (a multiple of 16): L_A may be the STACKED down projections of
+ *     several layers that read the same X and share s (query/key/value, gate/up), so that X is
+ *     read and quantized once; T [M, r] then holds the layers' T side by side and each layer's
+ *     linear kernel is given its column range (aser_linear_w4a8_lr_ld);
+ *   - with t_pair, 2 r <= 512.
+ * workspace: aser_quant_workspace_bytes(M, K, r) bytes, 16-byte aligned, contents irrelevant
+ * (the first 1024 bytes are not touched, so a linear kernel's workspace may be lent).  Work on
+ * `stream` that still uses the workspace when the call is made must precede it on `stream`.
+ */
+size_t aser_quant_workspace_bytes(int M, int K, int r);
+int aser_quant_act_ws(const void* X_f16, const float* s, const void* LA_f16,
+                      int M, int K, int r, int act_bits, int t_pair,
+                      int8_t* Xq, float* a_scale, void* T_bf16,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * aser_linear_w4a8_lr -- integer GEMM, dequantisation and up projection
  * (Sec. 4.2: W_q X + L_A L_B X in the paper's letters):
  *   acc[m,n] = sum_k Xq[m,k] * q[n,k]                               (exact int32)
@@ -140,6 +163,16 @@ int aser_linear_w4a8_lr(const int8_t* Xq, const float* a_scale, const void* Wk,
 int aser_linear_w4a8(const int8_t* Xq, const float* a_scale, const void* Wk,
                      const float* w_scale, int M, int N, int K, void* Y_f16,
                      int32_t* acc_debug, void* workspace, size_t workspace_bytes, void* stream);
+/*
+ * aser_linear_w4a8_lr_ld -- aser_linear_w4a8_lr with T given as a column range of a wider
+ * matrix: T_bf16 points at the layer's first column and consecutive rows are ldt elements apart
+ * (ldt >= r, a multiple of 8; 0 means r).  This is how the layers of a shared-input group read
+ * their part of a stacked T.
+ */
+int aser_linear_w4a8_lr_ld(const int8_t* Xq, const float* a_scale, const void* Wk,
+                           const float* w_scale, const void* T_bf16, int ldt, const void* LB_f16,
+                           int M, int N, int K, int r, void* Y_f16, int32_t* acc_debug,
+                           void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * aser_linear_w4a8_lr_simt -- the same operation on CUDA cores (dp4a) from the
@@ -198,8 +231,9 @@ int aser_check_status(void* workspace, void* stream);
  * Because the library knows that the quantization kernel is what precedes the linear kernel,
  * it launches the latter as a programmatic dependent: the linear kernel starts while the
  * quantization still runs, streams the weights (which that kernel does not write) and waits
- * for its completion before it reads Xq, a_scale or T.  Results are bit-identical to the two
- * separate calls.
+ * for its completion before it reads Xq, a_scale or T.  With more than 32 tokens the
+ * activation step is aser_quant_act_ws on the same workspace.  Results are those of the separate
+ * calls.
  * X_f16 [M,K], s [K] or NULL, LA_f16 [r,K] / LB_f16 [N,r] (NULL when r == 0), Wk and w_scale as
  * for aser_linear_w4a8_lr.  Xq [M,K], a_scale [M], T_bf16 [M,r] (NULL when r == 0) are the
  * caller's intermediates (written), Y_f16 [M,N] the result.  Wk, w_scale and LB_f16 must not
@@ -211,6 +245,25 @@ int aser_forward(const void* X_f16, const float* s, const void* LA_f16, const vo
                  const float* w_scale, const void* LB_f16, int M, int N, int K, int r,
                  int8_t* Xq, float* a_scale, void* T_bf16, void* Y_f16,
                  void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * aser_forward_shared -- the forward pass of n_layers layers that read the SAME activation X
+ * and share the smoothing vector s (Algorithm 1 builds each layer's factors on its own; where
+ * the layers' inputs and s coincide their activation work is identical): X is smoothed and
+ * quantized once, one pass computes every layer's T from the stacked down projections
+ * LA_stacked [sum r, K] (layer l's rows follow layer l-1's), then each layer's linear kernel runs
+ * on the shared codes.  Per layer l: Wk[l], w_scale[l], LB_f16[l] [N[l], r[l]], Y_f16[l] [M, N[l]].
+ * Xq [M, K], a_scale [M], T_bf16 [M, sum r] are the caller's intermediates.  sum r <= 512.
+ * workspace: aser_forward_shared_workspace_bytes(...) bytes, zeroed once with
+ * aser_workspace_init.  Each layer's output equals that of aser_forward on that layer alone up
+ * to the last bf16 bit of T.  Errors: every argument is checked before anything is enqueued.
+ */
+size_t aser_forward_shared_workspace_bytes(int n_layers, const int* N, const int* r, int M, int K);
+int aser_forward_shared(const void* X_f16, const float* s, const void* LA_stacked_f16, int n_layers,
+                        const void* const* Wk, const float* const* w_scale,
+                        const void* const* LB_f16, const int* N, const int* r, int M, int K,
+                        int8_t* Xq, float* a_scale, void* T_bf16, void* const* Y_f16,
+                        void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * aser_forward_host -- one whole forward pass from HOST buffers: copies X (fp16 [M,K],

@@ -11,7 +11,9 @@ lib_path = os.path.join(_HERE, "libaser.so")
 
 EXPORTED_SYMBOLS = (
     "aser_pack_w4", "aser_repacked_bytes", "aser_repack_w4", "aser_unrepack_w4",
-    "aser_quant_act", "aser_quant_act_bits", "aser_quant_act_ex", "aser_linear_w4a8_lr", "aser_linear_w4a8", "aser_linear_w4a8_lr_simt", "aser_linear_w4a8_lr_static",
+    "aser_quant_act", "aser_quant_act_bits", "aser_quant_act_ex", "aser_quant_act_ws",
+    "aser_quant_workspace_bytes", "aser_linear_w4a8_lr_ld", "aser_forward_shared",
+    "aser_forward_shared_workspace_bytes", "aser_linear_w4a8_lr", "aser_linear_w4a8", "aser_linear_w4a8_lr_simt", "aser_linear_w4a8_lr_static",
     "aser_workspace_bytes", "aser_workspace_init", "aser_check_status", "aser_forward",
     "aser_forward_host",
     "aser_last_error", "aser_version",
@@ -32,6 +34,13 @@ lib.aser_unrepack_w4.argtypes = [_P, _I, _I, _P, _P]
 lib.aser_quant_act.argtypes = [_P, _P, _P, _I, _I, _I, _P, _P, _P, _P]
 lib.aser_quant_act_bits.argtypes = [_P, _P, _P, _I, _I, _I, _I, _P, _P, _P, _P]
 lib.aser_quant_act_ex.argtypes = [_P, _P, _P, _I, _I, _I, _I, _I, _P, _P, _P, _P]
+lib.aser_quant_workspace_bytes.argtypes = [_I, _I, _I]
+lib.aser_quant_workspace_bytes.restype = _Z
+lib.aser_quant_act_ws.argtypes = [_P, _P, _P, _I, _I, _I, _I, _I, _P, _P, _P, _P, _Z, _P]
+lib.aser_linear_w4a8_lr_ld.argtypes = [_P, _P, _P, _P, _P, _I, _P, _I, _I, _I, _I, _P, _P, _P, _Z, _P]
+lib.aser_forward_shared_workspace_bytes.argtypes = [_I, _P, _P, _I, _I]
+lib.aser_forward_shared_workspace_bytes.restype = _Z
+lib.aser_forward_shared.argtypes = [_P, _P, _P, _I, _P, _P, _P, _P, _P, _I, _I, _P, _P, _P, _P, _P, _Z, _P]
 lib.aser_linear_w4a8_lr.argtypes = [_P, _P, _P, _P, _P, _P, _I, _I, _I, _I, _P, _P, _P, _Z, _P]
 lib.aser_linear_w4a8.argtypes = [_P, _P, _P, _P, _I, _I, _I, _P, _P, _P, _Z, _P]
 lib.aser_linear_w4a8_lr_simt.argtypes = [_P, _P, _P, _P, _P, _P, _I, _I, _I, _I, _P, _P, _P]
@@ -138,6 +147,31 @@ def quant_act(X: torch.Tensor, s: torch.Tensor | None, L_A: torch.Tensor | None,
     return Xq, a_scale, T
 
 
+def quant_workspace_bytes(M: int, K: int, r: int) -> int:
+    return int(lib.aser_quant_workspace_bytes(M, K, r))
+
+
+def quant_act_ws(X: torch.Tensor, s, L_A, ws: torch.Tensor | None = None, out=None,
+                 act_bits: int = 8, t_pair: bool = False):
+    """aser_quant_act_ws: quant_act with scratch memory (allocated here with torch when `ws` is
+    None); L_A may be the stacked down projections of several layers, up to 512 rows."""
+    _dev(X, torch.float16, "X")
+    M, K = X.shape
+    r = 0 if L_A is None else L_A.shape[0]
+    if ws is None:
+        ws = torch.empty((max(1024, quant_workspace_bytes(M, K, r)),), dtype=torch.uint8, device=X.device)
+    if out is None:
+        Xq = torch.empty((M, K), dtype=torch.int8, device=X.device)
+        a_scale = torch.empty((M,), dtype=torch.float32, device=X.device)
+        T = torch.empty((M, 2 * r if t_pair else r), dtype=torch.bfloat16, device=X.device)
+    else:
+        Xq, a_scale, T = out
+    _chk(lib.aser_quant_act_ws(_ptr(X), _ptr(s), _ptr(L_A) if r else None, M, K, r, act_bits,
+                               1 if t_pair else 0, _ptr(Xq), _ptr(a_scale), _ptr(T) if r else None,
+                               _ptr(ws), ws.numel(), _stream()), "aser_quant_act_ws")
+    return Xq, a_scale, T
+
+
 def workspace_bytes(M: int, N: int, K: int, r: int) -> int:
     return int(lib.aser_workspace_bytes(M, N, K, r))
 
@@ -164,6 +198,20 @@ def linear_w4a8_lr(Xq, a_scale, Wk, w_scale, T, L_B, N: int, ws: torch.Tensor,
                                  _ptr(T) if r else None, _ptr(L_B) if r else None, M, N, K, r,
                                  _ptr(Y), _ptr(acc_debug), _ptr(ws), ws.numel(), _stream()),
          "aser_linear_w4a8_lr")
+    return Y
+
+
+def linear_w4a8_lr_ld(Xq, a_scale, Wk, w_scale, T_wide, col0: int, L_B, N: int, ws: torch.Tensor,
+                      Y=None, acc_debug=None):
+    """aser_linear_w4a8_lr_ld: the layer's T is columns [col0, col0 + r) of T_wide [M, R]."""
+    M, K = Xq.shape
+    r = L_B.shape[1]
+    if Y is None:
+        Y = torch.empty((M, N), dtype=torch.float16, device=Xq.device)
+    t_ptr = C.c_void_p(T_wide.data_ptr() + 2 * col0)
+    _chk(lib.aser_linear_w4a8_lr_ld(_ptr(Xq), _ptr(a_scale), _ptr(Wk), _ptr(w_scale), t_ptr,
+                                    T_wide.shape[1], _ptr(L_B), M, N, K, r, _ptr(Y), _ptr(acc_debug),
+                                    _ptr(ws), ws.numel(), _stream()), "aser_linear_w4a8_lr_ld")
     return Y
 
 
@@ -248,11 +296,13 @@ class AserLinear:
         self.ws = new_workspace(max_tokens, self.N, self.K, self.r, dev)
 
     def quant(self, X: torch.Tensor):
+        """The activation step alone, as aser_forward runs it (aser_quant_act_ws on the layer's
+        workspace)."""
         M = X.shape[0]
         r = self.r
-        _chk(lib.aser_quant_act(_ptr(X), _ptr(self.s), _ptr(self.L_A) if r else None, M, self.K, r,
-                                _ptr(self.Xq), _ptr(self.a_scale), _ptr(self.T) if r else None,
-                                _stream()), "aser_quant_act")
+        _chk(lib.aser_quant_act_ws(_ptr(X), _ptr(self.s), _ptr(self.L_A) if r else None, M, self.K, r,
+                                   8, 0, _ptr(self.Xq), _ptr(self.a_scale), _ptr(self.T) if r else None,
+                                   _ptr(self.ws), self.ws.numel(), _stream()), "aser_quant_act_ws")
 
     def linear(self, M: int, lowrank: bool = True, acc_debug=None):
         r = self.r if lowrank else 0
@@ -281,6 +331,54 @@ class AserLinear:
     def forward_host(self, X_host: torch.Tensor, Y_host: torch.Tensor):
         """Host fp16 X [M,K] (pinned) -> host fp16 Y [M,N] through aser_forward_host."""
         forward_host(self, X_host, Y_host)
+
+
+class AserSharedInput:
+    """Layers that read the same activation and share the smoothing vector (query/key/value, or
+    gate/up): one activation pass for all of them through aser_forward_shared.  Built from
+    AserLinear objects; their packed weights and factors are used in place."""
+
+    def __init__(self, layers, max_tokens: int):
+        self.layers = list(layers)
+        first = self.layers[0]
+        self.K, self.s = first.K, first.s
+        for L in self.layers:
+            if L.K != self.K or (L.s is not first.s and not torch.equal(L.s, first.s)):
+                raise ValueError("layers of a shared-input group need the same K and smoothing vector")
+        dev = first.Wk.device
+        self.n = len(self.layers)
+        self.r = [L.r for L in self.layers]
+        self.N = [L.N for L in self.layers]
+        self.r_total = sum(self.r)
+        self.L_A = torch.cat([L.L_A for L in self.layers if L.r], dim=0).contiguous() if self.r_total else None
+        self.max_tokens = max_tokens
+        self.Xq = torch.empty((max_tokens, self.K), dtype=torch.int8, device=dev)
+        self.a_scale = torch.empty((max_tokens,), dtype=torch.float32, device=dev)
+        self.T = torch.empty((max_tokens, max(self.r_total, 1)), dtype=torch.bfloat16, device=dev)
+        self.Y = [torch.empty((max_tokens, n), dtype=torch.float16, device=dev) for n in self.N]
+        arr_i = C.c_int * self.n
+        arr_p = C.c_void_p * self.n
+        self._N, self._r = arr_i(*self.N), arr_i(*self.r)
+        self._Wk = arr_p(*[L.Wk.data_ptr() for L in self.layers])
+        self._ws = arr_p(*[L.w_scale.data_ptr() for L in self.layers])
+        self._LB = arr_p(*[(L.L_B.data_ptr() if L.r else None) for L in self.layers])
+        self._Y = arr_p(*[y.data_ptr() for y in self.Y])
+        nbytes = int(lib.aser_forward_shared_workspace_bytes(self.n, self._N, self._r, max_tokens, self.K))
+        if nbytes == 0:
+            raise ValueError("unsupported shapes for a shared-input group")
+        self.ws = torch.empty((nbytes,), dtype=torch.uint8, device=dev)
+        _chk(lib.aser_workspace_init(_ptr(self.ws), nbytes, _stream()), "aser_workspace_init")
+
+    def __call__(self, X: torch.Tensor):
+        """Returns the layers' outputs [M, N_l] (views of preallocated buffers)."""
+        M = X.shape[0]
+        assert M <= self.max_tokens
+        T = self.T if M == self.max_tokens else self.T[:M]
+        _chk(lib.aser_forward_shared(_ptr(X), _ptr(self.s), _ptr(self.L_A), self.n, self._Wk, self._ws,
+                                     self._LB, self._N, self._r, M, self.K, _ptr(self.Xq),
+                                     _ptr(self.a_scale), _ptr(self.T) if self.r_total else None, self._Y,
+                                     _ptr(self.ws), self.ws.numel(), _stream()), "aser_forward_shared")
+        return [y[:M] for y in self.Y]
 
 
 def forward_host(layer: AserLinear, X_host: torch.Tensor, Y_host: torch.Tensor):

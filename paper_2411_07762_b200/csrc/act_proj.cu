@@ -1,0 +1,452 @@
+// Activation path for many tokens when the caller provides scratch memory: two kernels.
+//
+//   act_proj_kernel    reads X once from HBM.  A CTA owns 128 tokens and one slice of K; TMA
+//                      streams the slice through a shared-memory ring together with the matching
+//                      columns of L_A.  The consumer warps take the row maxima of |x / s| (and
+//                      write x / s back as fp16 where s != 1), one thread issues tcgen05.mma
+//                      (kind::f16) with L_A on the M side (up to four groups of 128 rows, so the
+//                      down projections of several layers that share X are computed in one pass)
+//                      and the 128 tokens on the N side; the partial T of the slice goes to the
+//                      scratch as fp32 and the partial row maxima beside it.
+//   act_quant_kernel   per token row: the scale from the slices' maxima, the int8 codes (X comes
+//                      from L2 where the chunk of tokens was sized to stay there), and T as the
+//                      sum of the slices' partials in a fixed order, rounded to bf16.
+//
+// (Sec. 4.2 smoothing M^-1 X of Eq. 10, Sec. 5.1 per-token round-to-nearest, Sec. 4.1 projection
+// V_r^T S^-1 of the reconstruction branch.)  Both kernels are deterministic: no atomics.
+// Long inputs are processed in chunks of tokens small enough for the second kernel to find X in
+// L2.  Every mbarrier wait is bounded; a CTA that gives up poisons its row maxima with NaN.
+#include "act_math.cuh"
+#include "aser_common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace aser {
+
+namespace {
+
+constexpr int kPTok = 128;                  // tokens per CTA (the MMA's N)
+constexpr int kPCols = 64;                  // columns per stage: one 128-byte swizzled tile row
+constexpr int kPConsumerWarps = 8;
+constexpr int kPThreads = (2 + kPConsumerWarps) * 32;   // producer, MMA issuer, consumers
+constexpr int kPTileBytes = kPTok * 128;    // 128 rows x 64 fp16 (an X tile or one L_A group tile)
+constexpr int kPMaxGroups = 4;              // 128-row groups of L_A: r <= 512
+constexpr int kProjPlanSms = 148;           // chunks and slices are planned for this many SMs (the
+                                            // scratch size must not depend on the device)
+constexpr long long kPWaitLimitClocks = 400000000ll;   // about 0.2 s of SM clocks per wait
+
+__host__ __device__ constexpr int proj_stages(int groups) {
+    const int per_stage = kPTileBytes * (1 + groups);
+    const int ns = (220 * 1024) / per_stage;
+    return ns > 8 ? 8 : ns;                 // 8, 6, 4, 3, 2 stages for 0..4 groups
+}
+
+__device__ __noinline__ bool pj_wait_slow(uint32_t bar, uint32_t parity, volatile int* flag) {
+    uint32_t spins = 0;
+    long long t0 = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 255u) == 0) {
+            if (*flag) return false;
+            if (t0 == 0) {
+                t0 = clock64();
+            } else if (clock64() - t0 > kPWaitLimitClocks) {
+                *flag = 1;
+                return false;
+            }
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ bool pj_wait(uint32_t bar, uint32_t parity, volatile int* flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return pj_wait_slow(bar, parity, flag);
+}
+__device__ __forceinline__ bool pj_warp_wait(uint32_t bar, uint32_t parity, volatile int* flag, int lane) {
+    int ok = 1;
+    if (lane == 0) ok = pj_wait(bar, parity, flag) ? 1 : 0;
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+__device__ __forceinline__ uint4 pj_lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void pj_sts128(uint32_t addr, uint4 v) {
+    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+// grid = (KS slices, token tiles of the chunk).  Scratch of the chunk:
+//   amax_part [KS][Mc]      fp32   row maxima of |x~| over the slice (NaN: the CTA gave up)
+//   t_part    [KS][Mc][Rp]  fp32   partial T, Rp = r rounded up to 32
+// map_x: X as fp16 [K / 64 blocks][M][64], box 1 block x 128 rows, 128-byte swizzle (rows past
+// M read as zero).  map_la: L_A as fp16 [K / 64 blocks][r][64], box 1 block x 128 rows (rows past
+// r read as zero, so every group tile is a full 128 x 64 operand).
+__global__ void __launch_bounds__(kPThreads, 1)
+act_proj_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_la,
+                const float* __restrict__ s, int m_first, int Mc, int K, int Kc, int r, int Rp,
+                float* __restrict__ amax_part, float* __restrict__ t_part) {
+    // bytes one L_A box delivers: 128 rows (rows past r are zero-filled), r rows when r < 128
+    // (the MMA then also reads the stale rows behind them; their accumulator rows are never read)
+    const uint32_t la_box_bytes = (uint32_t)(r < 128 ? r : 128) * 128u;
+    extern __shared__ uint8_t smem_raw[];
+    grid_dep_launch();
+    const uint32_t sraw = smem_u32(smem_raw);
+    const uint32_t sb = (sraw + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (sb - sraw);
+    const int groups = (r + 127) / 128;
+    const int NS = proj_stages(groups);
+    const int stage_bytes = kPTileBytes * (1 + groups);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int ks = blockIdx.x, tile = blockIdx.y;
+    const int k0 = ks * Kc;
+    const int nst = Kc / kPCols;
+    const int row0 = tile * kPTok;                  // first token of the tile inside the chunk
+    // after the ring: barriers, flags, the per-warp row maxima
+    uint8_t* tail = smem + NS * stage_bytes;
+    const uint32_t bars = sb + NS * stage_bytes;
+    auto bar_full = [&](int st) { return bars + st * 8; };
+    auto bar_ready = [&](int st) { return bars + (8 + st) * 8; };
+    auto bar_free = [&](int st) { return bars + (16 + st) * 8; };
+    const uint32_t bar_acc = bars + 24 * 8;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 25 * 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 25 * 8 + 8);
+    volatile int* never_flag = abort_flag + 1;                      // stays 0: waits of the wind-down
+    uint8_t* ones_sm = tail + 256;                                  // per 8 columns of the slice: all divisors are 1
+    float* amax_w = reinterpret_cast<float*>(tail + 256 + ((Kc / 8 + 15) & ~15));   // [8 warps][128 rows]
+    const uint32_t tmem_cols = groups <= 1 ? 128u : groups == 2 ? 256u : 512u;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int st = 0; st < 8; ++st) {
+                mbar_init(bar_full(st), 1);
+                mbar_init(bar_ready(st), kPConsumerWarps);
+                mbar_init(bar_free(st), 1);
+            }
+            mbar_init(bar_acc, 1);
+            *abort_flag = 0;
+            *never_flag = 0;
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            fence_proxy_async_smem();
+            prefetch_tensormap(&map_x);
+            if (r > 0) prefetch_tensormap(&map_la);
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (r > 0) {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(tmem_slot)), "r"(tmem_cols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
+    } else {
+        for (int g = tid - 64; g < Kc / 8; g += kPConsumerWarps * 32) {
+            bool one = true;
+            if (s) {
+                const float4 a = __ldg(reinterpret_cast<const float4*>(s + k0 + g * 8));
+                const float4 b = __ldg(reinterpret_cast<const float4*>(s + k0 + g * 8) + 1);
+                one = a.x == 1.f && a.y == 1.f && a.z == 1.f && a.w == 1.f &&
+                      b.x == 1.f && b.y == 1.f && b.z == 1.f && b.w == 1.f;
+            }
+            ones_sm[g] = one ? 1 : 0;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = (r > 0) ? *tmem_slot : 0u;
+
+    if (warp == 0) {
+        // ================= TMA producer =================
+        if (lane == 0) {
+            grid_dep_wait();        // X may come from the kernel before; the scratch may still be read by it
+            bool ok = true;
+            int issued = 0;
+            for (int i = 0; i < nst && ok; ++i) {
+                const int st = i % NS;
+                if (i >= NS) ok = pj_wait(bar_free(st), (uint32_t)(i / NS - 1) & 1u, abort_flag);
+                if (!ok) break;
+                const uint32_t dst = sb + st * stage_bytes;
+                const int kblk = (k0 + i * kPCols) / kPCols;
+                mbar_arrive_expect_tx(bar_full(st), (uint32_t)kPTileBytes + (uint32_t)groups * la_box_bytes);
+                tma_load_3d(dst, &map_x, 0, m_first + row0, kblk, bar_full(st));
+                for (int g = 0; g < groups; ++g)
+                    tma_load_3d(dst + (1 + g) * kPTileBytes, &map_la, 0, g * 128, kblk, bar_full(st));
+                ++issued;
+            }
+            if (*abort_flag) {      // let copies already issued land before the shared memory goes away
+                for (int i = (issued > NS ? issued - NS : 0); i < issued; ++i)
+                    pj_wait(bar_full(i % NS), (uint32_t)(i / NS) & 1u, never_flag);
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer =================
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc(1u, 0u, 128u, (uint32_t)kPTok);
+            bool ok = true;
+            for (int i = 0; i < nst && ok; ++i) {
+                const int st = i % NS;
+                ok = pj_wait(bar_ready(st), (uint32_t)(i / NS) & 1u, abort_flag);
+                if (!ok) break;
+                if (r > 0) {
+                    tc_fence_after();
+                    const uint64_t bdesc = smem_desc_sw128(sb + st * stage_bytes);
+                    for (int g = 0; g < groups; ++g) {
+                        const uint64_t adesc = smem_desc_sw128(sb + st * stage_bytes + (1 + g) * kPTileBytes);
+#pragma unroll
+                        for (int kk = 0; kk < kPCols / 16; ++kk)
+                            mma_f16_ss(tmem + g * 128, adesc + 2 * kk, bdesc + 2 * kk, idesc, (i != 0 || kk != 0) ? 1u : 0u);
+                    }
+                    tc_commit(bar_free(st));
+                } else {
+                    mbar_arrive(bar_free(st));
+                }
+            }
+            if (r > 0) {
+                tc_commit(bar_acc);     // arrives when every MMA issued above has completed
+                if (!ok) pj_wait(bar_acc, 0u, never_flag);      // giving up: let them finish before leaving
+            }
+        }
+    } else {
+        // ================= consumers =================
+        // Warp cw owns the 16-byte piece cw (8 columns) of every row; lane = rows lane, +32, +64, +96.
+        const int cw = warp - 2;
+        float amax[4] = {0.f, 0.f, 0.f, 0.f};
+        __half2 hmax[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) hmax[q] = __float2half2_rn(0.f);
+        bool ok = true;
+        for (int i = 0; i < nst; ++i) {
+            const int st = i % NS;
+            ok = pj_warp_wait(bar_full(st), (uint32_t)(i / NS) & 1u, abort_flag, lane);
+            if (!ok) break;
+            const uint32_t base = sb + st * stage_bytes;
+            uint32_t addr[4];
+            uint4 v[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int row = lane + 32 * q;
+                addr[q] = base + (uint32_t)row * 128u + (uint32_t)((cw ^ (row & 7)) << 4);
+                v[q] = pj_lds128(addr[q]);
+            }
+            if (ones_sm[i * 8 + cw]) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const __half2* h = reinterpret_cast<const __half2*>(&v[q]);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) hmax[q] = __hmax2(hmax[q], __habs2(h[e]));
+                }
+            } else {
+                const float4* sp = reinterpret_cast<const float4*>(s + k0 + i * kPCols + cw * 8);
+                const float4 s0 = __ldg(sp), s1 = __ldg(sp + 1);
+                const float sv[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const __half* h = reinterpret_cast<const __half*>(&v[q]);
+                    float f[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        f[e] = __half2float(h[e]);
+                        if (sv[e] != 1.f) f[e] = __fdiv_rn(f[e], sv[e]);
+                        amax[q] = fmaxf(amax[q], fabsf(f[e]));
+                    }
+                    __half2 p0 = __floats2half2_rn(f[0], f[1]), p1 = __floats2half2_rn(f[2], f[3]);
+                    __half2 p2 = __floats2half2_rn(f[4], f[5]), p3 = __floats2half2_rn(f[6], f[7]);
+                    uint4 pk;
+                    pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
+                    pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
+                    pj_sts128(addr[q], pk);
+                }
+                fence_proxy_async_smem();       // the MMA reads these through the async proxy
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_ready(st));
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const float a = fmaxf(amax[q], fmaxf(__low2float(hmax[q]), __high2float(hmax[q])));
+            amax_w[cw * kPTok + lane + 32 * q] = a;
+        }
+        named_bar_sync(1, kPConsumerWarps * 32);
+        if (tid - 64 < kPTok) {
+            const int row = tid - 64;
+            float a = amax_w[row];
+#pragma unroll
+            for (int w = 1; w < kPConsumerWarps; ++w) a = fmaxf(a, amax_w[w * kPTok + row]);
+            if (*abort_flag) a = __int_as_float(0x7fc00000);
+            if (row0 + row < Mc) amax_part[(size_t)ks * Mc + row0 + row] = a;
+        }
+        // ---- partial T: tensor memory -> scratch (fp32).  A warp reaches the 32 lanes (rows j of a
+        // group) of its quarter, warp % 4; the two warps of a quarter take 64 tokens each. ----
+        if (r > 0) {
+            if (ok) ok = pj_warp_wait(bar_acc, 0u, abort_flag, lane);
+            tc_fence_after();
+            const int q = warp & 3, half = cw >> 2;
+            float* tp = t_part + ((size_t)ks * Mc + row0) * Rp;
+            for (int g = 0; g < groups; ++g) {
+                const int j = g * 128 + q * 32 + lane;
+                if (g * 128 + q * 32 >= r) break;
+#pragma unroll 1
+                for (int c0 = half * 64; c0 < half * 64 + 64; c0 += 16) {
+                    uint32_t v[16];
+                    tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(g * 128 + c0), v);
+                    tmem_wait_ld(v);
+                    if (ok && j < Rp) {
+#pragma unroll
+                        for (int e = 0; e < 16; ++e)
+                            if (row0 + c0 + e < Mc) tp[(size_t)(c0 + e) * Rp + j] = __uint_as_float(v[e]);
+                    }
+                }
+            }
+            tc_fence_before();
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1 && r > 0) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols) : "memory");
+    }
+}
+
+// grid = rows of the chunk, 256 threads.  Launched as a programmatic dependent of act_proj_kernel.
+__global__ void __launch_bounds__(256)
+act_quant_kernel(const __half* __restrict__ X, const float* __restrict__ s, int m_first, int Mc, int K,
+                 int r, int Rp, int KS, const float* amax_part, const float* t_part,
+                 int8_t* __restrict__ Xq, float* __restrict__ a_scale, __nv_bfloat16* __restrict__ T,
+                 int ldt, int lo_off, float qmax) {
+    grid_dep_launch();      // a dependent linear kernel may start streaming its weights
+    grid_dep_wait();        // the partial maxima and the partial T come from act_proj_kernel
+    const int row = blockIdx.x, m = m_first + row;
+    float a = 0.f;
+    bool bad = false;
+    for (int ks = 0; ks < KS; ++ks) {
+        const float v = amax_part[(size_t)ks * Mc + row];
+        bad = bad || (v != v);
+        a = fmaxf(a, v);
+    }
+    if (bad) a = __int_as_float(0x7fc00000);
+    const float sc = __fdiv_rn(a, qmax);
+    if (threadIdx.x == 0) a_scale[m] = sc;
+    const float rcp = (sc > 0.f) ? __frcp_rn(sc) : 0.f;
+    const __half* xrow = X + (size_t)m * K;
+    int8_t* out = Xq + (size_t)m * K;
+    const int chunks = K / 8;
+    for (int c = threadIdx.x; c < chunks; c += 256) {
+        const RawChunk rc = load_raw(xrow, s, c * 8, true);
+        float v[8];
+        smooth8(rc, v);
+        uint2 q = make_uint2(0u, 0u);
+        if (sc > 0.f) q = quant8_pairs(v, sc, rcp, qmax);
+        *reinterpret_cast<uint2*>(out + c * 8) = q;
+    }
+    for (int j = threadIdx.x; j < r; j += 256) {
+        float t = 0.f;
+        for (int ks = 0; ks < KS; ++ks) t += t_part[((size_t)ks * Mc + row) * Rp + j];
+        store_t(T + (size_t)m * ldt, j, t, lo_off);
+    }
+}
+
+struct ProjPlan {
+    int Mc;         // tokens per chunk (a multiple of 128 unless it is all of M)
+    int KS;         // slices of K
+};
+
+// Chunk and slice sizes.  A chunk's X (2 Mc K bytes) should stay in L2 between the two kernels;
+// within that, take the chunk and the slice count that fill the SMs best in one wave (a slice
+// has at least four 64-column stages), preferring fewer chunks.
+ProjPlan proj_plan(int M, int K, int num_sms) {
+    const long long l2_budget = 48ll << 20;
+    const int blocks = K / kPCols;
+    int max_tiles = (int)(l2_budget / (2ll * K * kPTok));
+    if (max_tiles < 1) max_tiles = 1;
+    const int all_tiles = (M + kPTok - 1) / kPTok;
+    ProjPlan best{M, 1};
+    double best_score = -1.0;
+    for (int tiles = (all_tiles <= max_tiles ? all_tiles : max_tiles); tiles >= 1; --tiles) {
+        const int n_chunks = (all_tiles + tiles - 1) / tiles;
+        int ks_best = 1;
+        for (int ks = 1; ks <= blocks / 4 && tiles * ks <= num_sms; ++ks)
+            if (blocks % ks == 0) ks_best = ks;
+        // SM-time of the whole call in units of (one SM busy for one full-K tile)
+        const double per_chunk = 1.0 / ks_best + 0.15;          // streaming share plus fixed cost
+        const double score = 1.0 / (n_chunks * per_chunk);
+        if (score > best_score * 1.02) { best_score = score; best = ProjPlan{tiles * kPTok, ks_best}; }
+        if (tiles == all_tiles && tiles * ks_best * 10 >= num_sms * 8) break;   // one chunk fills the SMs
+    }
+    if (best.Mc > M) best.Mc = M;
+    return best;
+}
+
+size_t proj_scratch_bytes(int M, int K, int r, int num_sms) {
+    const ProjPlan p = proj_plan(M, K, num_sms);
+    const int Rp = (r + 31) / 32 * 32;
+    return (size_t)p.KS * p.Mc * (1 + Rp) * sizeof(float);
+}
+
+}  // namespace
+
+size_t quant_act_ws_scratch_bytes(int M, int K, int r) {
+    if (M <= 32) return 0;
+    return proj_scratch_bytes(M, K, r, kProjPlanSms);
+}
+
+int launch_quant_act_ws(const __half* X, const float* s, const __half* LA, int M, int K, int r,
+                        int8_t* Xq, float* a_scale, __nv_bfloat16* T, void* scratch, size_t scratch_bytes,
+                        cudaStream_t st, int act_bits, bool t_pair) {
+    const float qmax = (float)((1 << (act_bits - 1)) - 1);
+    const int ldt = t_pair ? 2 * r : r, lo_off = t_pair ? r : 0;
+    const int groups = (r + 127) / 128;
+    if (groups > kPMaxGroups) return record_error(ASER_ERR_SHAPE, "quant_act: r beyond 512");
+    const ProjPlan plan = proj_plan(M, K, kProjPlanSms);
+    const int Rp = (r + 31) / 32 * 32;
+    if (scratch == nullptr || scratch_bytes < (size_t)plan.KS * plan.Mc * (1 + Rp) * sizeof(float))
+        return record_error(ASER_ERR_WORKSPACE, "quant_act: scratch missing or too small");
+    float* amax_part = static_cast<float*>(scratch);
+    float* t_part = amax_part + (size_t)plan.KS * plan.Mc;
+    const int Kc = K / plan.KS;
+    const int NS = proj_stages(groups);
+    const size_t smem = (size_t)NS * kPTileBytes * (1 + groups) + 256 + ((Kc / 8 + 15) & ~15) +
+                        kPConsumerWarps * kPTok * sizeof(float) + 1024;
+    static size_t configured[kMaxDevices] = {0};
+    int dev = 0;
+    {
+        const int rc = current_device(&dev);
+        if (rc != ASER_OK) return rc;
+    }
+    if (smem > configured[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(act_proj_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return record_cuda_error(e, "act_proj smem attribute");
+        configured[dev] = smem;
+    }
+    CUtensorMap mx, mla;
+    int rc = encode_map_blocks(&mx, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, X, M, K, kPTok, 1);
+    if (rc != ASER_OK) return rc;
+    if (r > 0) {
+        rc = encode_map_blocks(&mla, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, LA, r, K, r < 128 ? r : 128, 1);
+        if (rc != ASER_OK) return rc;
+    } else {
+        mla = mx;
+    }
+    for (int m_first = 0; m_first < M; m_first += plan.Mc) {
+        const int Mc = (M - m_first < plan.Mc) ? (M - m_first) : plan.Mc;
+        const int tiles = (Mc + kPTok - 1) / kPTok;
+        act_proj_kernel<<<dim3(plan.KS, tiles, 1), kPThreads, smem, st>>>(mx, mla, s, m_first, Mc, K, Kc, r, Rp,
+                                                                          amax_part, t_part);
+        rc = check_launch("act_proj_kernel");
+        if (rc != ASER_OK) return rc;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(Mc, 1, 1);
+        cfg.blockDim = dim3(256, 1, 1);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cudaError_t e = cudaLaunchKernelEx(&cfg, act_quant_kernel, X, s, m_first, Mc, K, r, Rp, plan.KS,
+                                           (const float*)amax_part, (const float*)t_part, Xq, a_scale, T, ldt,
+                                           lo_off, qmax);
+        if (e != cudaSuccess) return record_cuda_error(e, "act_quant_kernel");
+    }
+    return ASER_OK;
+}
+
+}  // namespace aser

@@ -92,8 +92,10 @@ int check_device() {
 int linear_common(const int8_t* Xq, const float* a_scale, const void* Wk, const float* w_scale,
                   const void* T_bf16, const void* LB_f16, int M, int N, int K, int r, void* Y_f16,
                   int32_t* acc_debug, void* workspace, size_t workspace_bytes, void* stream,
-                  bool overlap_prev = false) {
+                  bool overlap_prev = false, int ldt = 0) {
     if (!shape_ok(M, N, K, r)) return fail(ASER_ERR_SHAPE, "unsupported M, N, K or r");
+    if (r > 0 && ldt != 0 && (ldt < r || ldt % 8 != 0))
+        return fail(ASER_ERR_SHAPE, "ldt must be a multiple of 8 and at least r");
     if (M == 0 || N == 0) return ASER_OK;
     ASER_REQUIRE_PTR(Xq);
     ASER_REQUIRE_PTR(a_scale);
@@ -106,7 +108,7 @@ int linear_common(const int8_t* Xq, const float* a_scale, const void* Wk, const 
         ASER_REQUIRE_PTR(LB_f16);
     }
     if (workspace == nullptr || misaligned16(workspace) ||
-        workspace_bytes < aser_workspace_bytes(M, N, K, r))
+        workspace_bytes < kWsHeaderBytes + linear_tc_workspace_bytes(M, N, K, r))
         return fail(ASER_ERR_WORKSPACE, "workspace missing, misaligned or too small");
     int rc = check_device();
     if (rc != ASER_OK) return rc;
@@ -115,12 +117,33 @@ int linear_common(const int8_t* Xq, const float* a_scale, const void* Wk, const 
                                     static_cast<const __nv_bfloat16*>(T_bf16),
                                     static_cast<const __half*>(LB_f16), M, N, K, r,
                                     static_cast<__half*>(Y_f16), acc_debug,
-                                    static_cast<cudaStream_t>(stream), overlap_prev);
+                                    static_cast<cudaStream_t>(stream), overlap_prev, ldt);
     return launch_linear_tc(Xq, a_scale, static_cast<const uint8_t*>(Wk), w_scale,
                             static_cast<const __nv_bfloat16*>(T_bf16),
                             static_cast<const __half*>(LB_f16), M, N, K, r,
                             static_cast<__half*>(Y_f16), acc_debug, workspace, workspace_bytes,
-                            static_cast<cudaStream_t>(stream), overlap_prev);
+                            static_cast<cudaStream_t>(stream), overlap_prev, ldt);
+}
+
+// Stacked ranks (several layers' down projections in one pass) go up to 512.
+bool act_shape_ok(int M, int K, int r) {
+    return M >= 0 && K > 0 && K % 128 == 0 && K <= 32768 && r >= 0 && r <= 512 && r % 16 == 0;
+}
+
+// Activation kernels with scratch: more than 32 tokens take the two-kernel path (its scratch
+// sits behind the workspace's zeroed prefix, where the linear kernel later keeps its partial
+// sums), fewer the few-token kernel.
+int quant_with_workspace(const void* X_f16, const float* s, const void* LA_f16, int M, int K, int r,
+                         int act_bits, bool t_pair, int8_t* Xq, float* a_scale, void* T_bf16,
+                         void* workspace, size_t workspace_bytes, void* stream) {
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (M <= 32)
+        return launch_quant_act(static_cast<const __half*>(X_f16), s, static_cast<const __half*>(LA_f16), M, K, r,
+                                Xq, a_scale, static_cast<__nv_bfloat16*>(T_bf16), st, act_bits, t_pair);
+    return launch_quant_act_ws(static_cast<const __half*>(X_f16), s, static_cast<const __half*>(LA_f16), M, K, r,
+                               Xq, a_scale, static_cast<__nv_bfloat16*>(T_bf16),
+                               static_cast<uint8_t*>(workspace) + kWsZeroedBytes,
+                               workspace_bytes - kWsZeroedBytes, st, act_bits, t_pair);
 }
 
 }  // namespace
@@ -249,7 +272,116 @@ int aser_linear_w4a8_lr_simt(const int8_t* Xq, const float* a_scale, const uint8
 
 size_t aser_workspace_bytes(int M, int N, int K, int r) {
     if (!shape_ok(M, N, K, r)) return 0;
-    return kWsHeaderBytes + linear_tc_workspace_bytes(M, N, K, r);
+    const size_t lin = kWsHeaderBytes + linear_tc_workspace_bytes(M, N, K, r);
+    const size_t act = aser_quant_workspace_bytes(M, K, r);
+    return lin > act ? lin : act;
+}
+
+size_t aser_quant_workspace_bytes(int M, int K, int r) {
+    if (!act_shape_ok(M, K, r)) return 0;
+    return kWsZeroedBytes + quant_act_ws_scratch_bytes(M, K, r);
+}
+
+int aser_quant_act_ws(const void* X_f16, const float* s, const void* LA_f16, int M, int K, int r,
+                      int act_bits, int t_pair, int8_t* Xq, float* a_scale, void* T_bf16,
+                      void* workspace, size_t workspace_bytes, void* stream) {
+    if (!act_shape_ok(M, K, r)) return fail(ASER_ERR_SHAPE, "unsupported M, K or r");
+    if (act_bits < 2 || act_bits > 8) return fail(ASER_ERR_SHAPE, "act_bits must be 2..8");
+    if (t_pair != 0 && t_pair != 1) return fail(ASER_ERR_SHAPE, "t_pair must be 0 or 1");
+    if (t_pair && 2 * r > 512) return fail(ASER_ERR_SHAPE, "t_pair needs 2 r <= 512");
+    if (M == 0) return ASER_OK;
+    ASER_REQUIRE_PTR(X_f16);
+    ASER_OPTIONAL_PTR(s);
+    ASER_REQUIRE_PTR(Xq);
+    ASER_REQUIRE_PTR(a_scale);
+    if (r > 0) {
+        ASER_REQUIRE_PTR(LA_f16);
+        ASER_REQUIRE_PTR(T_bf16);
+    }
+    if (workspace == nullptr || misaligned16(workspace) ||
+        workspace_bytes < aser_quant_workspace_bytes(M, K, r))
+        return fail(ASER_ERR_WORKSPACE, "workspace missing, misaligned or too small");
+    int rc = check_device();
+    if (rc != ASER_OK) return rc;
+    return quant_with_workspace(X_f16, s, LA_f16, M, K, r, act_bits, t_pair != 0, Xq, a_scale, T_bf16,
+                                workspace, workspace_bytes, stream);
+}
+
+int aser_linear_w4a8_lr_ld(const int8_t* Xq, const float* a_scale, const void* Wk,
+                           const float* w_scale, const void* T_bf16, int ldt, const void* LB_f16,
+                           int M, int N, int K, int r, void* Y_f16, int32_t* acc_debug,
+                           void* workspace, size_t workspace_bytes, void* stream) {
+    return linear_common(Xq, a_scale, Wk, w_scale, T_bf16, LB_f16, M, N, K, r, Y_f16, acc_debug,
+                         workspace, workspace_bytes, stream, false, ldt);
+}
+
+size_t aser_forward_shared_workspace_bytes(int n_layers, const int* N, const int* r, int M, int K) {
+    if (n_layers < 1 || N == nullptr || r == nullptr) return 0;
+    int r_total = 0;
+    size_t need = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        if (!shape_ok(M, N[l], K, r[l])) return 0;
+        r_total += r[l];
+        const size_t lin = kWsHeaderBytes + linear_tc_workspace_bytes(M, N[l], K, r[l]);
+        if (lin > need) need = lin;
+    }
+    const size_t act = aser_quant_workspace_bytes(M, K, r_total);
+    if (act == 0) return 0;
+    return act > need ? act : need;
+}
+
+int aser_forward_shared(const void* X_f16, const float* s, const void* LA_stacked_f16, int n_layers,
+                        const void* const* Wk, const float* const* w_scale, const void* const* LB_f16,
+                        const int* N, const int* r, int M, int K, int8_t* Xq, float* a_scale,
+                        void* T_bf16, void* const* Y_f16, void* workspace, size_t workspace_bytes,
+                        void* stream) {
+    if (n_layers < 1 || n_layers > 16) return fail(ASER_ERR_SHAPE, "n_layers must be 1..16");
+    if (Wk == nullptr || w_scale == nullptr || LB_f16 == nullptr || N == nullptr || r == nullptr ||
+        Y_f16 == nullptr)
+        return fail(ASER_ERR_NULL, "a per-layer array is NULL");
+    const size_t need = aser_forward_shared_workspace_bytes(n_layers, N, r, M, K);
+    if (need == 0) return fail(ASER_ERR_SHAPE, "unsupported M, N, K or r (stacked ranks go up to 512)");
+    if (M == 0) return ASER_OK;
+    int r_total = 0;
+    for (int l = 0; l < n_layers; ++l) r_total += r[l];
+    // every argument of every launch is checked before the first one is enqueued
+    ASER_REQUIRE_PTR(X_f16);
+    ASER_OPTIONAL_PTR(s);
+    ASER_REQUIRE_PTR(Xq);
+    ASER_REQUIRE_PTR(a_scale);
+    if (r_total > 0) {
+        ASER_REQUIRE_PTR(LA_stacked_f16);
+        ASER_REQUIRE_PTR(T_bf16);
+    }
+    for (int l = 0; l < n_layers; ++l) {
+        if (N[l] == 0) continue;
+        ASER_REQUIRE_PTR(Wk[l]);
+        ASER_REQUIRE_PTR(w_scale[l]);
+        ASER_REQUIRE_PTR(Y_f16[l]);
+        if (r[l] > 0) ASER_REQUIRE_PTR(LB_f16[l]);
+    }
+    if (workspace == nullptr || misaligned16(workspace) || workspace_bytes < need)
+        return fail(ASER_ERR_WORKSPACE, "workspace missing, misaligned or too small");
+    int rc = check_device();
+    if (rc != ASER_OK) return rc;
+    for (int l = 0; l < n_layers; ++l)
+        if (N[l] > 0 && !linear_decode_prefers(M, N[l], K)) {
+            rc = linear_tc_check(M, N[l], K, r[l], workspace_bytes);
+            if (rc != ASER_OK) return rc;
+        }
+    rc = quant_with_workspace(X_f16, s, LA_stacked_f16, M, K, r_total, 8, false, Xq, a_scale, T_bf16,
+                              workspace, workspace_bytes, stream);
+    if (rc != ASER_OK) return rc;
+    int col = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        const void* Tl = r[l] > 0 ? static_cast<const void*>(static_cast<const __nv_bfloat16*>(T_bf16) + col) : nullptr;
+        rc = linear_common(Xq, a_scale, Wk[l], w_scale[l], Tl, r[l] > 0 ? LB_f16[l] : nullptr, M, N[l], K,
+                           r[l], Y_f16[l], nullptr, workspace, workspace_bytes, stream,
+                           /*overlap_prev=*/l == 0, r_total);
+        if (rc != ASER_OK) return rc;
+        col += r[l];
+    }
+    return ASER_OK;
 }
 
 int aser_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
@@ -313,7 +445,8 @@ int aser_forward(const void* X_f16, const float* s, const void* LA_f16, const vo
     int rc = forward_validate(X_f16, s, LA_f16, Wk, w_scale, LB_f16, M, N, K, r, Xq, a_scale, T_bf16,
                               Y_f16, workspace, workspace_bytes);
     if (rc != ASER_OK) return rc;
-    rc = aser_quant_act(X_f16, s, LA_f16, M, K, r, Xq, a_scale, T_bf16, stream);
+    rc = quant_with_workspace(X_f16, s, LA_f16, M, K, r, 8, false, Xq, a_scale, T_bf16, workspace,
+                              workspace_bytes, stream);
     if (rc != ASER_OK) return rc;
     return linear_common(Xq, a_scale, Wk, w_scale, r > 0 ? T_bf16 : nullptr, r > 0 ? LB_f16 : nullptr,
                          M, N, K, r, Y_f16, nullptr, workspace, workspace_bytes, stream,

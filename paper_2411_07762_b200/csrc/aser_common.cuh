@@ -37,9 +37,16 @@ int launch_repack_w4(const uint8_t* Wq, int N, int K, uint8_t* Wk, bool inverse,
 int launch_quant_act(const __half* X, const float* s, const __half* LA, int M, int K, int r,
                      int8_t* Xq, float* a_scale, __nv_bfloat16* T, cudaStream_t st, int act_bits = 8,
                      bool t_pair = false);
+// The same with caller-provided scratch (quant_act_ws_scratch_bytes): the two-kernel path for more
+// than 32 tokens, ranks up to 512 (stacked down projections of layers that share X).
+size_t quant_act_ws_scratch_bytes(int M, int K, int r);
+int launch_quant_act_ws(const __half* X, const float* s, const __half* LA, int M, int K, int r,
+                        int8_t* Xq, float* a_scale, __nv_bfloat16* T, void* scratch, size_t scratch_bytes,
+                        cudaStream_t st, int act_bits = 8, bool t_pair = false);
 int launch_linear_simt(const int8_t* Xq, const float* a_scale, const uint8_t* Wq,
                        const float* w_scale, const __nv_bfloat16* T, const __half* LB,
                        int M, int N, int K, int r, __half* Y, int32_t* acc_debug, cudaStream_t st);
+// `ldt`: elements between rows of T (0 = r; larger when T is a column range of a wider matrix).
 // `overlap_prev`: the kernel launched before this one on `st` is this library's quant_act for
 // the same step.  The linear kernel may then start while that one still runs: it streams the
 // weights (which that kernel does not write) and waits for its completion before it touches
@@ -48,7 +55,7 @@ int launch_linear_tc(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
                      const float* w_scale, const __nv_bfloat16* T, const __half* LB,
                      int M, int N, int K, int r, __half* Y, int32_t* acc_debug,
                      void* workspace, size_t workspace_bytes, cudaStream_t st,
-                     bool overlap_prev = false);
+                     bool overlap_prev = false, int ldt = 0);
 // Few-token kernel (M <= kLinearDecodeMaxTokens): streams the weights once, no workspace.
 // linear_decode_prefers: the shapes for which it is faster than the tensor-core kernel.
 constexpr int kLinearDecodeMaxTokens = 16;
@@ -56,7 +63,7 @@ bool linear_decode_prefers(int M, int N, int K);
 int launch_linear_decode(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
                          const float* w_scale, const __nv_bfloat16* T, const __half* LB,
                          int M, int N, int K, int r, __half* Y, int32_t* acc_debug,
-                         cudaStream_t st, bool overlap_prev = false);
+                         cudaStream_t st, bool overlap_prev = false, int ldt = 0);
 size_t linear_tc_workspace_bytes(int M, int N, int K, int r);
 // The range checks launch_linear_tc makes before it launches (workspace size, index widths), for
 // callers that must reject a call before they enqueue anything else.  Records the error text.

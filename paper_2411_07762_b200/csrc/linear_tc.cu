@@ -926,7 +926,7 @@ int linear_tc_check(int M, int N, int K, int r, size_t workspace_bytes) {
 int launch_linear_tc(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
                      const float* w_scale, const __nv_bfloat16* T, const __half* LB,
                      int M, int N, int K, int r, __half* Y, int32_t* acc_debug,
-                     void* workspace, size_t workspace_bytes, cudaStream_t st, bool overlap_prev) {
+                     void* workspace, size_t workspace_bytes, cudaStream_t st, bool overlap_prev, int ldt) {
     Layout L = make_layout(M, N, K, r);
     const int pre = linear_tc_check(M, N, K, r, workspace_bytes);
     if (pre != ASER_OK) return pre;
@@ -979,7 +979,8 @@ int launch_linear_tc(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
     if (r > 0) {
         rc = make_map_2d(&mlb, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, LB, N, r, 128, 64);
         if (rc != ASER_OK) return rc;
-        rc = make_map_2d(&mt, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, T, M, r, L.BT, 64);
+        rc = encode_map_2d_ld(&mt, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, T, M, r, ldt > 0 ? ldt : r, L.BT, 64,
+                              CU_TENSOR_MAP_SWIZZLE_128B);
         if (rc != ASER_OK) return rc;
     } else {
         mlb = mx;

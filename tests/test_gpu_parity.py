@@ -123,6 +123,62 @@ def test_quant_act_without_smoothing_vector(aser):
     assert np.array_equal(Xq.cpu().numpy(), Xq_ref) and np.array_equal(bits(sc.cpu().numpy()), bits(sc_ref))
 
 
+WS_ACT_CASES = [  # M, K, r, t_pair
+    (33, 512, 16, False), (127, 1024, 64, False), (129, 4096, 128, False), (300, 2048, 256, False),
+    (64, 14336, 64, False), (200, 128, 48, False), (65, 256, 0, False), (1000, 2048, 112, False),
+    (2049, 512, 16, False), (40, 28672, 64, False),
+    # stacked down projections of several layers (more than 256 rows), the pair storage of T,
+    # and enough tokens at K = 14336 for the pass to be cut into chunks
+    (700, 4096, 384, False), (260, 1024, 512, False), (300, 2048, 96, True), (4096, 14336, 128, False),
+]
+
+
+@pytest.mark.parametrize("M,K,r,t_pair", WS_ACT_CASES)
+def test_quant_act_ws_parity(aser, M, K, r, t_pair):
+    """aser_quant_act_ws (two kernels, caller's scratch): codes and scales bit-exact against the
+    oracle, T within the derived bound, on ragged token tiles, zero rows and exact ties."""
+    lay = synth.make_layer(M, 8, K, seed=250 + M + K + r, n_cal=8)
+    s = synth.standin_smoothing_vector(K, lay.outlier_idx, 13.0)
+    X = lay.X.copy()
+    X[1] = 0
+    X[2, :] = 0
+    X[2, :6] = np.array([127, .5, 1.5, 2.5, -2.5, -126.5], np.float16)
+    L_A = synth.standin_factors(8, K, r, seed=M, scale_a=0.05)[0] if r else None
+    xs = F.smooth_act(X, s)
+    Xq_ref, sc_ref = F.quant_act(xs)
+    Xq, sc, T = aser.quant_act_ws(to_dev(X), to_dev(s), None if L_A is None else to_dev(L_A), t_pair=t_pair)
+    assert np.array_equal(Xq.cpu().numpy(), Xq_ref)
+    assert np.array_equal(bits(sc.cpu().numpy()), bits(sc_ref))
+    if r:
+        T_ref = F.down_proj(xs, L_A)
+        if t_pair:
+            assert_T_close(T[:, :r].float().cpu().numpy(), T_ref, xs, L_A)
+            T_sum = T[:, :r].double().cpu().numpy() + T[:, r:].double().cpu().numpy()
+            xs64, la64 = xs.astype(np.float64), L_A.astype(np.float64)
+            tol = 2.0 ** -16 * np.abs(T_ref) + 2.0 ** -9.2 * np.sqrt((xs64 ** 2) @ (la64 ** 2).T) + \
+                2.0 ** -20 * (np.abs(xs64) @ np.abs(la64).T) + 1e-30
+            assert np.all(np.abs(T_sum - T_ref) <= tol)
+        else:
+            assert_T_close(T.float().cpu().numpy(), T_ref, xs, L_A)
+
+
+def test_quant_act_ws_dense_smoothing_and_6_bits(aser):
+    """Every divisor differs from 1, and 6-bit codes, through the two-kernel path."""
+    M, K, r = 300, 1024, 64
+    lay = synth.make_layer(M, 8, K, seed=471, n_cal=8)
+    rng = np.random.default_rng(M + K)
+    s = rng.uniform(0.25, 6.0, size=K).astype(np.float32)
+    s[::7] = 1.0
+    L_A = synth.standin_factors(8, K, r, seed=M, scale_a=0.05)[0]
+    xs = F.smooth_act(lay.X, s)
+    for bits_ in (8, 6):
+        Xq_ref, sc_ref = F.quant_act(xs, act_bits=bits_)
+        Xq, sc, T = aser.quant_act_ws(to_dev(lay.X), to_dev(s), to_dev(L_A), act_bits=bits_)
+        assert np.array_equal(Xq.cpu().numpy(), Xq_ref)
+        assert np.array_equal(bits(sc.cpu().numpy()), bits(sc_ref))
+        assert_T_close(T.float().cpu().numpy(), F.down_proj(xs, L_A), xs, L_A)
+
+
 # ---------------------------------------------------------------------------
 # whole path: quant_act -> linear
 # ---------------------------------------------------------------------------
@@ -438,6 +494,64 @@ def test_status_word_reports_a_timeout_and_clears(aser):
     assert err.value.code == -6 and "status word" in str(err.value)
     aser.check_status(ws)
     assert int(ws[:1024].to(torch.int32).sum()) == 0
+
+
+SHARED_CASES = [  # M, K, [(N, r), ...]
+    (8, 1024, [(256, 32), (128, 16), (128, 16)]),
+    (200, 1024, [(384, 64), (136, 48), (128, 0)]),
+    (300, 2048, [(512, 128), (256, 128), (256, 128)]),
+]
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("M,K,spec", SHARED_CASES)
+def test_forward_shared_matches_oracle_per_layer(aser, M, K, spec):
+    """aser_forward_shared: one activation pass for layers that read the same X.  Codes and
+    scales bit-exact; every layer's output within the bound of the oracle run on that layer
+    alone; and the stacked T equals the per-layer T of separate aser_quant_act_ws calls."""
+    check_shared_group(aser, M, K, spec, seed0=1200 + M + K, construct=False)
+
+
+def check_shared_group(aser, M, K, spec, seed0, construct, gain=30.0):
+    base = synth.make_layer(M, spec[0][0], K, seed=seed0, n_cal=64, n_out=max(1, K // 100), outlier_gain=gain)
+    s = synth.standin_smoothing_vector(K, base.outlier_idx, 11.0)
+    ds = to_dev(s)
+    layers, refs = [], []
+    for li, (N, r) in enumerate(spec):
+        rng = np.random.default_rng(seed0 + 17 * li + 1)
+        W = (rng.standard_normal((N, K), dtype=np.float32) * np.float32(0.02)).astype(np.float16)
+        q, w_scale = F.quant_w4(W, s)
+        L_A, L_B = synth.standin_factors(N, K, max(r, 16), seed=seed0 + li, scale_a=0.01, scale_b=0.01)
+        L_A, L_B = (L_A[:r], np.ascontiguousarray(L_B[:, :r])) if r else (None, None)
+        lay = aser.AserLinear(to_dev(W), ds, None if r == 0 else to_dev(L_A), None if r == 0 else to_dev(L_B), M)
+        assert np.array_equal(lay.Wq.cpu().numpy(), F.pack_w4(q))
+        layers.append(lay)
+        refs.append(F.forward(base.X, s, F.pack_w4(q), w_scale, L_A, L_B, use_dgemm=True))
+    group = aser.AserSharedInput(layers, M)
+    X = to_dev(base.X)
+    for rep in range(2):                    # twice: the workspace is reused
+        Ys = group(X)
+        aser.check_status(group.ws)
+        torch.cuda.synchronize()
+        assert np.array_equal(group.Xq[:M].cpu().numpy(), refs[0].Xq)
+        assert np.array_equal(bits(group.a_scale[:M].cpu().numpy()), bits(refs[0].a_scale))
+        col = 0
+        for lay, ref, Y in zip(layers, refs, Ys):
+            assert_rows_close(Y.cpu().numpy(), ref.y)
+            if lay.r:
+                lay.quant(X)
+                assert torch.equal(group.T[:M, col:col + lay.r].contiguous().view(torch.int16),
+                                   lay.T[:M].view(torch.int16))
+                col += lay.r
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("which", ["qkv", "gate_up"])
+def test_forward_shared_decoder_block_groups_full_size(aser, which):
+    """The two shared-input groups of the decoder block at 4096 tokens, rank 128: query/key/value
+    (384 stacked rows) and gate/up (256)."""
+    spec = [(4096, 128), (1024, 128), (1024, 128)] if which == "qkv" else [(14336, 128), (14336, 128)]
+    check_shared_group(aser, 4096, 4096, spec, seed0=synth.seed_for(4, 50 + len(spec)), construct=False)
 
 
 # ---------------------------------------------------------------------------

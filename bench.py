@@ -317,7 +317,9 @@ def summarize(samples_ms):
 class Model:
     """Device-resident operands of a workload: one AserLinear per layer and one activation
     tensor per input group, in as many distinct operand sets as it takes for a step never to
-    find its operands in L2 (one set where a single step already exceeds twice the L2 size)."""
+    find its operands in L2 (one set where a single step already exceeds twice the L2 size).
+    Layers of one input group run through aser_forward_shared (one activation pass for the
+    group), a layer alone in its group through aser_forward."""
 
     def __init__(self, name, device):
         import torch
@@ -329,15 +331,20 @@ class Model:
         per_set = step_bytes(w)
         self.n_sets = 1 if per_set > 2 * L2_BYTES else int(np.ceil(2.2 * L2_BYTES / per_set))
         t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(device)
-        base_layers, base_x = [], {}
+        self.group_ids = [g for _, _, _, g in w["layers"]]
+        self.members = {}                       # input group -> layer indices
+        for li, g in enumerate(self.group_ids):
+            self.members.setdefault(g, []).append(li)
+        base_layers, base_x, group_s = [], {}, {}
         for li, (nm, K, N, g) in enumerate(w["layers"]):
             lay, s, L_A, L_B = make_layer_inputs(w, li)
-            base_layers.append(aser.AserLinear(t(lay.W), t(s), t(L_A) if self.r else None,
-                                               t(L_B) if self.r else None, self.M))
             if g not in base_x:
                 base_x[g] = t(lay.X)
+                group_s[g] = t(s)               # the layers of a group share the smoothing vector
+            base_layers.append(aser.AserLinear(t(lay.W), group_s[g], t(L_A) if self.r else None,
+                                               t(L_B) if self.r else None, self.M))
             del lay
-        self.sets = [(base_layers, base_x)]
+        self.sets = [self._make_set(base_layers, base_x)]
         for i in range(1, self.n_sets):
             # further operand sets: same shapes and value ranges; packed weights are the base
             # set's bytes rolled by a set-dependent offset (contents do not affect timing)
@@ -354,47 +361,83 @@ class Model:
                 L.T, L.Y = torch.empty_like(b.T), torch.empty_like(b.Y)
                 layers.append(L)
             xs = {g: torch.roll(x, shifts=i, dims=1).contiguous() for g, x in base_x.items()}
-            self.sets.append((layers, xs))
-        self.groups = [g for _, _, _, g in w["layers"]]
+            self.sets.append(self._make_set(layers, xs))
         torch.cuda.synchronize()
 
-    # one whole pass through the public entry point (aser_forward per layer)
+    def _make_set(self, layers, xs):
+        """(layers, inputs, shared-input groups with and without the low-rank term)."""
+        aser = self.aser
+        shared, shared_plain = {}, {}
+        for g, idx in self.members.items():
+            if len(idx) > 1:
+                shared[g] = aser.AserSharedInput([layers[i] for i in idx], self.M)
+                if self.r:
+                    plain = []
+                    for i in idx:
+                        P = object.__new__(aser.AserLinear)
+                        P.__dict__.update(layers[i].__dict__)
+                        P.r, P.L_A, P.L_B = 0, None, None
+                        plain.append(P)
+                    shared_plain[g] = aser.AserSharedInput(plain, self.M)
+                else:
+                    shared_plain[g] = shared[g]
+        return dict(layers=layers, xs=xs, shared=shared, shared_plain=shared_plain)
+
+    # one whole pass through the public entry points
     def step(self, i, lowrank=True):
-        layers, xs = self.sets[i % self.n_sets]
-        for L, g in zip(layers, self.groups):
-            L(xs[g], lowrank)
+        S = self.sets[i % self.n_sets]
+        for g, idx in self.members.items():
+            if len(idx) > 1:
+                (S["shared"] if lowrank else S["shared_plain"])[g](S["xs"][g])
+            else:
+                S["layers"][idx[0]](S["xs"][g], lowrank)
 
     def linear_only(self, i, li=None, lowrank=True):
-        layers, _ = self.sets[i % self.n_sets]
-        for j, L in enumerate(layers):
+        S = self.sets[i % self.n_sets]
+        for j, L in enumerate(S["layers"]):
             if li is None or li == j:
                 L.linear(self.M, lowrank)
 
-    def quant_only(self, i, li=None):
-        layers, xs = self.sets[i % self.n_sets]
-        for j, (L, g) in enumerate(zip(layers, self.groups)):
-            if li is None or li == j:
-                L.quant(xs[g])
+    def quant_only(self, i, g_only=None):
+        """The activation passes of a step (one per input group), or of one group."""
+        S = self.sets[i % self.n_sets]
+        for g, idx in self.members.items():
+            if g_only is not None and g != g_only:
+                continue
+            if len(idx) > 1:
+                S["shared"][g].quant(S["xs"][g])
+            else:
+                S["layers"][idx[0]].quant(S["xs"][g])
 
-    def layer_step(self, i, li, lowrank=True):
-        layers, xs = self.sets[i % self.n_sets]
-        layers[li](xs[self.groups[li]], lowrank)
+    def group_step(self, i, g, lowrank=True):
+        S = self.sets[i % self.n_sets]
+        idx = self.members[g]
+        if len(idx) > 1:
+            (S["shared"] if lowrank else S["shared_plain"])[g](S["xs"][g])
+        else:
+            S["layers"][idx[0]](S["xs"][g], lowrank)
 
     def launches_per_step(self):
-        """Kernels of this library launched by one step (two quantization launches above rank 128)."""
-        per_quant = 2 if (self.r > 128 and self.M > 32) else 1
-        return len(self.groups) * (per_quant + 1)
+        """Kernels of this library launched by one step: per input group the activation pass
+        (two kernels per chunk of tokens above 32 tokens, one below) and one linear kernel per layer."""
+        n = 0
+        for g, idx in self.members.items():
+            K = self.w["layers"][idx[0]][1]
+            n += self.aser.quant_act_ws_launches(self.M, K) + len(idx)
+        return n
 
     def check(self):
-        for layers, _ in self.sets:
-            for L in layers:
+        for S in self.sets:
+            for L in S["layers"]:
                 self.aser.check_status(L.ws)
+            for G in list(S["shared"].values()) + list(S["shared_plain"].values()):
+                self.aser.check_status(G.ws)
 
     # ---- timing ----
     def capture(self, fn, calls):
         """CUDA graphs that together make exactly `calls` calls fn(0) .. fn(calls - 1)."""
         torch = self.torch
-        chunk = max(1, min(calls, max(self.n_sets * 2, 4096 // max(1, 3 * len(self.groups)))))
+        chunk = max(1, min(calls, max(self.n_sets * 2, 4096 // max(1, 3 * len(self.group_ids)))))
         sizes = [chunk] * (calls // chunk) + ([calls % chunk] if calls % chunk else [])
         side = torch.cuda.Stream()
         graphs, start = [], 0
@@ -516,25 +559,36 @@ def measure(m, steps, peaks, lib_int8, barrier=None, max_over_ranks=lambda x: x,
                overhead=dict(linear=t_lin["median"] / t_lin_plain["median"] - 1.0,
                              step=t_step["median"] / t_step_plain["median"] - 1.0),
                roofline=roofline_of(w, m.name, t_lin["median"] * 1e3, peaks, lib_int8))
-    act_bytes = sum(algorithmic_bytes_act(w["M"], K, w["r"]) for _, K, _, _ in w["layers"])
+    act_bytes = sum(algorithmic_bytes_act(w["M"], w["layers"][idx[0]][1], w["r"] * len(idx))
+                    for idx in m.members.values())
     out["quant_act_gbs"] = act_bytes / (t_act["median"] * 1e-3) / 1e9
     if per_layer and len(w["layers"]) > 1:
         rows = []
         for li, (nm, K, N, _) in enumerate(w["layers"]):
             tl = m.time_region(lambda i: m.linear_only(i, li), calls, label=nm + " linear")
             tp = m.time_region(lambda i: m.linear_only(i, li, False), calls, label=nm + " linear_plain") if m.r else tl
-            ta = m.time_region(lambda i: m.quant_only(i, li), calls, label=nm + " quant")
-            ts = m.time_region(lambda i: m.layer_step(i, li), calls, label=nm + " step")
-            tsp = m.time_region(lambda i: m.layer_step(i, li, False), calls, label=nm + " step_plain") if m.r else ts
             ops = 2.0 * w["M"] * N * K
             roof = roofline_of(w, m.name, tl["median"] * 1e3, peaks, lib_int8, li)
-            rows.append(dict(layer=nm, K=K, N=N, us_step=ts["median"] * 1e3, us_linear_lr=tl["median"] * 1e3,
-                             us_linear_plain=tp["median"] * 1e3, us_quant_act=ta["median"] * 1e3,
+            rows.append(dict(layer=nm, K=K, N=N, us_linear_lr=tl["median"] * 1e3,
+                             us_linear_plain=tp["median"] * 1e3,
                              tops_linear=ops / (tl["median"] * 1e-3) / 1e12, frac=roof["frac"],
-                             lowrank_overhead_linear=tl["median"] / tp["median"] - 1.0,
-                             lowrank_overhead_step=ts["median"] / tsp["median"] - 1.0,
-                             quant_act_gbs=algorithmic_bytes_act(w["M"], K, w["r"]) / (ta["median"] * 1e-3) / 1e9))
+                             lowrank_overhead_linear=tl["median"] / tp["median"] - 1.0))
         out["layers"] = rows
+        groups = []
+        for g, idx in m.members.items():
+            K = w["layers"][idx[0]][1]
+            names = "+".join(w["layers"][i][0] for i in idx)
+            ta = m.time_region(lambda i: m.quant_only(i, g), calls, label=names + " quant")
+            ts = m.time_region(lambda i: m.group_step(i, g), calls, label=names + " step")
+            tsp = m.time_region(lambda i: m.group_step(i, g, False), calls, label=names + " step_plain") if m.r else ts
+            act_b = algorithmic_bytes_act(w["M"], K, w["r"] * len(idx))
+            groups.append(dict(layers=names, K=K, stacked_rank=w["r"] * len(idx),
+                               us_quant_act=ta["median"] * 1e3, us_step=ts["median"] * 1e3,
+                               us_step_plain=tsp["median"] * 1e3,
+                               lowrank_overhead_step=ts["median"] / tsp["median"] - 1.0,
+                               quant_act_gbs=act_b / (ta["median"] * 1e-3) / 1e9,
+                               quant_act_frac_hbm=act_b / (ta["median"] * 1e-3) / 1e9 / peaks["hbm_gbs"]))
+        out["input_groups"] = groups
     return out
 
 
@@ -583,12 +637,12 @@ def run_ours(args, rank, world, local_rank):
         barrier()
         # end to end from pinned host buffers through the C ABI (aser_forward_host per layer):
         # every step copies each layer's input to the device and its output back
-        layers, xs = m.sets[0]
+        layers, xs = m.sets[0]["layers"], m.sets[0]["xs"]
         host_x = {g: x.cpu().pin_memory() for g, x in xs.items()}
         host_y = [torch.empty((m.M, L.N), dtype=torch.float16).pin_memory() for L in layers]
 
         def e2e_step():
-            for L, g, y in zip(layers, m.groups, host_y):
+            for L, g, y in zip(layers, m.group_ids, host_y):
                 L.forward_host(host_x[g], y)
         for _ in range(3):
             e2e_step()
@@ -632,6 +686,7 @@ def run_ours(args, rank, world, local_rank):
     )
     if "layers" in res:
         line["layers"] = res["layers"]
+        line["input_groups"] = res["input_groups"]
     if w["bound"] == "hbm":
         line["l2_warm_us_step"] = warm_l2_point(m)
     del m

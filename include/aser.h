@@ -134,6 +134,8 @@ int aser_quant_act_ex(const void* X_f16, const float* s, const void* LA_f16,
  * `stream` that still uses the workspace when the call is made must precede it on `stream`.
  */
 size_t aser_quant_workspace_bytes(int M, int K, int r);
+/* Number of kernels one aser_quant_act_ws call enqueues (two per chunk of tokens; 0 for bad shapes). */
+int aser_quant_act_ws_launches(int M, int K);
 int aser_quant_act_ws(const void* X_f16, const float* s, const void* LA_f16,
                       int M, int K, int r, int act_bits, int t_pair,
                       int8_t* Xq, float* a_scale, void* T_bf16,

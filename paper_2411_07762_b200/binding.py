@@ -12,7 +12,7 @@ lib_path = os.path.join(_HERE, "libaser.so")
 EXPORTED_SYMBOLS = (
     "aser_pack_w4", "aser_repacked_bytes", "aser_repack_w4", "aser_unrepack_w4",
     "aser_quant_act", "aser_quant_act_bits", "aser_quant_act_ex", "aser_quant_act_ws",
-    "aser_quant_workspace_bytes", "aser_linear_w4a8_lr_ld", "aser_forward_shared",
+    "aser_quant_workspace_bytes", "aser_quant_act_ws_launches", "aser_linear_w4a8_lr_ld", "aser_forward_shared",
     "aser_forward_shared_workspace_bytes", "aser_linear_w4a8_lr", "aser_linear_w4a8", "aser_linear_w4a8_lr_simt", "aser_linear_w4a8_lr_static",
     "aser_workspace_bytes", "aser_workspace_init", "aser_check_status", "aser_forward",
     "aser_forward_host",
@@ -36,6 +36,8 @@ lib.aser_quant_act_bits.argtypes = [_P, _P, _P, _I, _I, _I, _I, _P, _P, _P, _P]
 lib.aser_quant_act_ex.argtypes = [_P, _P, _P, _I, _I, _I, _I, _I, _P, _P, _P, _P]
 lib.aser_quant_workspace_bytes.argtypes = [_I, _I, _I]
 lib.aser_quant_workspace_bytes.restype = _Z
+lib.aser_quant_act_ws_launches.argtypes = [_I, _I]
+lib.aser_quant_act_ws_launches.restype = _I
 lib.aser_quant_act_ws.argtypes = [_P, _P, _P, _I, _I, _I, _I, _I, _P, _P, _P, _P, _Z, _P]
 lib.aser_linear_w4a8_lr_ld.argtypes = [_P, _P, _P, _P, _P, _I, _P, _I, _I, _I, _I, _P, _P, _P, _Z, _P]
 lib.aser_forward_shared_workspace_bytes.argtypes = [_I, _P, _P, _I, _I]
@@ -145,6 +147,10 @@ def quant_act(X: torch.Tensor, s: torch.Tensor | None, L_A: torch.Tensor | None,
     _chk(lib.aser_quant_act(_ptr(X), _ptr(s), _ptr(L_A) if r else None, M, K, r, _ptr(Xq),
                             _ptr(a_scale), _ptr(T) if r else None, _stream()), "aser_quant_act")
     return Xq, a_scale, T
+
+
+def quant_act_ws_launches(M: int, K: int) -> int:
+    return int(lib.aser_quant_act_ws_launches(M, K))
 
 
 def quant_workspace_bytes(M: int, K: int, r: int) -> int:
@@ -368,6 +374,13 @@ class AserSharedInput:
             raise ValueError("unsupported shapes for a shared-input group")
         self.ws = torch.empty((nbytes,), dtype=torch.uint8, device=dev)
         _chk(lib.aser_workspace_init(_ptr(self.ws), nbytes, _stream()), "aser_workspace_init")
+
+    def quant(self, X: torch.Tensor):
+        """The activation pass of the group alone (aser_quant_act_ws with the stacked L_A)."""
+        M = X.shape[0]
+        _chk(lib.aser_quant_act_ws(_ptr(X), _ptr(self.s), _ptr(self.L_A), M, self.K, self.r_total, 8, 0,
+                                   _ptr(self.Xq), _ptr(self.a_scale), _ptr(self.T) if self.r_total else None,
+                                   _ptr(self.ws), self.ws.numel(), _stream()), "aser_quant_act_ws")
 
     def __call__(self, X: torch.Tensor):
         """Returns the layers' outputs [M, N_l] (views of preallocated buffers)."""

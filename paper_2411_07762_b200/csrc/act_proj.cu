@@ -27,7 +27,8 @@ namespace {
 constexpr int kPTok = 128;                  // tokens per CTA (the MMA's N)
 constexpr int kPCols = 64;                  // columns per stage: one 128-byte swizzled tile row
 constexpr int kPConsumerWarps = 8;
-constexpr int kPThreads = (2 + kPConsumerWarps) * 32;   // producer, MMA issuer, consumers
+constexpr int kPWarpLa = 2 + kPConsumerWarps;           // producer of the L_A tiles
+constexpr int kPThreads = (3 + kPConsumerWarps) * 32;   // X producer, MMA issuer, consumers, L_A producer
 constexpr int kPTileBytes = kPTok * 128;    // 128 rows x 64 fp16 (an X tile or one L_A group tile)
 constexpr int kPMaxGroups = 4;              // 128-row groups of L_A: r <= 512
 constexpr int kProjPlanSms = 148;           // chunks and slices are planned for this many SMs (the
@@ -76,17 +77,21 @@ __device__ __forceinline__ void pj_sts128(uint32_t addr, uint4 v) {
 
 // grid = (KS slices, token tiles of the chunk).  Scratch of the chunk:
 //   amax_part [KS][Mc]      fp32   row maxima of |x~| over the slice (NaN: the CTA gave up)
-//   t_part    [KS][Mc][Rp]  fp32   partial T, Rp = r rounded up to 32
+//   t_part    [KS][groups][Mc][128]  fp32   partial T, by 128-row group of L_A (rows past r: unspecified)
 // map_x: X as fp16 [K / 64 blocks][M][64], box 1 block x 128 rows, 128-byte swizzle (rows past
-// M read as zero).  map_la: L_A as fp16 [K / 64 blocks][r][64], box 1 block x 128 rows (rows past
-// r read as zero, so every group tile is a full 128 x 64 operand).
+// M read as zero).  map_la: L_A as fp16 [K / 64 blocks][r][64], box 1 block x r rows (r / 2 rows
+// above 256).
 __global__ void __launch_bounds__(kPThreads, 1)
 act_proj_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_la,
-                const float* __restrict__ s, int m_first, int Mc, int K, int Kc, int r, int Rp,
+                const float* __restrict__ s, int m_first, int Mc, int K, int Kc, int r,
                 float* __restrict__ amax_part, float* __restrict__ t_part) {
-    // bytes one L_A box delivers: 128 rows (rows past r are zero-filled), r rows when r < 128
-    // (the MMA then also reads the stale rows behind them; their accumulator rows are never read)
-    const uint32_t la_box_bytes = (uint32_t)(r < 128 ? r : 128) * 128u;
+    // The r rows of L_A arrive as one box (r <= 256, the largest box) or as two boxes of r / 2
+    // rows; in shared memory the rows follow one another, 128 bytes each, so group g is the 16 KB
+    // at g * 16 KB whatever the boxes.  Where r is not a multiple of 128 the last group's MMA also
+    // reads the stale rows behind row r; their accumulator rows are never read.
+    const int la_boxes = r <= 256 ? 1 : 2;
+    const int la_box_rows = r / la_boxes;
+    const uint32_t la_stage_bytes = (uint32_t)r * 128u;
     extern __shared__ uint8_t smem_raw[];
     grid_dep_launch();
     const uint32_t sraw = smem_u32(smem_raw);
@@ -117,7 +122,7 @@ act_proj_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     if (warp == 0) {
         if (lane == 0) {
             for (int st = 0; st < 8; ++st) {
-                mbar_init(bar_full(st), 1);
+                mbar_init(bar_full(st), r > 0 ? 2 : 1);      // the X producer and the L_A producer
                 mbar_init(bar_ready(st), kPConsumerWarps);
                 mbar_init(bar_free(st), 1);
             }
@@ -136,7 +141,7 @@ act_proj_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                          ::"r"(smem_u32(tmem_slot)), "r"(tmem_cols) : "memory");
             asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
         }
-    } else {
+    } else if (warp < kPWarpLa) {
         for (int g = tid - 64; g < Kc / 8; g += kPConsumerWarps * 32) {
             bool one = true;
             if (s) {
@@ -165,13 +170,32 @@ act_proj_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 if (!ok) break;
                 const uint32_t dst = sb + st * stage_bytes;
                 const int kblk = (k0 + i * kPCols) / kPCols;
-                mbar_arrive_expect_tx(bar_full(st), (uint32_t)kPTileBytes + (uint32_t)groups * la_box_bytes);
+                mbar_arrive_expect_tx(bar_full(st), (uint32_t)kPTileBytes);
                 tma_load_3d(dst, &map_x, 0, m_first + row0, kblk, bar_full(st));
-                for (int g = 0; g < groups; ++g)
-                    tma_load_3d(dst + (1 + g) * kPTileBytes, &map_la, 0, g * 128, kblk, bar_full(st));
                 ++issued;
             }
             if (*abort_flag) {      // let copies already issued land before the shared memory goes away
+                for (int i = (issued > NS ? issued - NS : 0); i < issued; ++i)
+                    pj_wait(bar_full(i % NS), (uint32_t)(i / NS) & 1u, never_flag);
+            }
+        }
+    } else if (warp == kPWarpLa) {
+        // ================= L_A producer: one box of up to 256 rows (two groups) per copy =================
+        if (lane == 0 && r > 0) {
+            bool ok = true;
+            int issued = 0;
+            for (int i = 0; i < nst && ok; ++i) {
+                const int st = i % NS;
+                if (i >= NS) ok = pj_wait(bar_free(st), (uint32_t)(i / NS - 1) & 1u, abort_flag);
+                if (!ok) break;
+                const uint32_t dst = sb + st * stage_bytes + kPTileBytes;
+                const int kblk = (k0 + i * kPCols) / kPCols;
+                mbar_arrive_expect_tx(bar_full(st), la_stage_bytes);
+                for (int b = 0; b < la_boxes; ++b)
+                    tma_load_3d(dst + b * la_box_rows * 128, &map_la, 0, b * la_box_rows, kblk, bar_full(st));
+                ++issued;
+            }
+            if (*abort_flag) {
                 for (int i = (issued > NS ? issued - NS : 0); i < issued; ++i)
                     pj_wait(bar_full(i % NS), (uint32_t)(i / NS) & 1u, never_flag);
             }
@@ -204,7 +228,7 @@ act_proj_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 if (!ok) pj_wait(bar_acc, 0u, never_flag);      // giving up: let them finish before leaving
             }
         }
-    } else {
+    } else if (warp < kPWarpLa) {
         // ================= consumers =================
         // Warp cw owns the 16-byte piece cw (8 columns) of every row; lane = rows lane, +32, +64, +96.
         const int cw = warp - 2;
@@ -273,28 +297,41 @@ act_proj_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             if (*abort_flag) a = __int_as_float(0x7fc00000);
             if (row0 + row < Mc) amax_part[(size_t)ks * Mc + row0 + row] = a;
         }
-        // ---- partial T: tensor memory -> scratch (fp32).  A warp reaches the 32 lanes (rows j of a
-        // group) of its quarter, warp % 4; the two warps of a quarter take 64 tokens each. ----
+        // ---- partial T: tensor memory -> shared memory as [token][128 rows of the group] -> one
+        // bulk copy per group into the scratch, where a group's tile is contiguous.  A warp
+        // reaches the 32 lanes (rows j of a group) of its quarter, warp % 4; the two warps of a
+        // quarter take 64 tokens each.  The ring is idle by now (every MMA has completed) and
+        // serves as two 64 KB staging buffers. ----
         if (r > 0) {
             if (ok) ok = pj_warp_wait(bar_acc, 0u, abort_flag, lane);
             tc_fence_after();
             const int q = warp & 3, half = cw >> 2;
-            float* tp = t_part + ((size_t)ks * Mc + row0) * Rp;
+            const int rows_valid = (Mc - row0 < kPTok) ? (Mc - row0) : kPTok;
             for (int g = 0; g < groups; ++g) {
-                const int j = g * 128 + q * 32 + lane;
-                if (g * 128 + q * 32 >= r) break;
+                const uint32_t buf = sb + (uint32_t)(g & 1) * 65536u;
+                if (g >= 2) {               // the copy that last read this buffer must be done with it
+                    if (tid == 64) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                    named_bar_sync(1, kPConsumerWarps * 32);
+                }
 #pragma unroll 1
                 for (int c0 = half * 64; c0 < half * 64 + 64; c0 += 16) {
                     uint32_t v[16];
                     tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(g * 128 + c0), v);
                     tmem_wait_ld(v);
-                    if (ok && j < Rp) {
 #pragma unroll
-                        for (int e = 0; e < 16; ++e)
-                            if (row0 + c0 + e < Mc) tp[(size_t)(c0 + e) * Rp + j] = __uint_as_float(v[e]);
-                    }
+                    for (int e = 0; e < 16; ++e)
+                        asm volatile("st.shared.b32 [%0], %1;" ::"r"(buf + (uint32_t)(c0 + e) * 512u + (uint32_t)(q * 32 + lane) * 4u), "r"(v[e]) : "memory");
+                }
+                fence_proxy_async_smem();
+                named_bar_sync(1, kPConsumerWarps * 32);
+                if (tid == 64 && !*abort_flag) {
+                    float* dst = t_part + (((size_t)ks * groups + g) * Mc + row0) * 128;
+                    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                                 ::"l"(dst), "r"(buf), "r"((uint32_t)rows_valid * 512u) : "memory");
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 }
             }
+            if (tid == 64) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
             tc_fence_before();
         }
     }
@@ -306,41 +343,131 @@ act_proj_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     }
 }
 
-// grid = rows of the chunk, 256 threads.  Launched as a programmatic dependent of act_proj_kernel.
-__global__ void __launch_bounds__(256)
+// grid = ceil(rows of the chunk / kQRows), 256 threads; a CTA takes kQRows token rows: a smoothing
+// divisor is loaded (and tested against 1) once for all of them, several 16-byte loads per thread
+// are in flight, and the per-row scales are computed once per CTA (one warp per row) instead of by
+// every thread.  The kernel is bound by instruction issue, not by bytes: fp16 pairs are widened
+// with half2 operations, the products and the magic-constant rounding run on packed fp32 pairs.
+// Launched as a programmatic dependent of act_proj_kernel: the first loads of X (an input of the
+// whole step, not a product of that kernel) are issued before the dependency wait.
+constexpr int kQRows = 4;
+__global__ void __launch_bounds__(256, 4)
 act_quant_kernel(const __half* __restrict__ X, const float* __restrict__ s, int m_first, int Mc, int K,
-                 int r, int Rp, int KS, const float* amax_part, const float* t_part,
+                 int r, int KS, const float* amax_part, const float* t_part,
                  int8_t* __restrict__ Xq, float* __restrict__ a_scale, __nv_bfloat16* __restrict__ T,
                  int ldt, int lo_off, float qmax) {
+    __shared__ float sc_sm[kQRows], rcp_sm[kQRows];
     grid_dep_launch();      // a dependent linear kernel may start streaming its weights
-    grid_dep_wait();        // the partial maxima and the partial T come from act_proj_kernel
-    const int row = blockIdx.x, m = m_first + row;
-    float a = 0.f;
-    bool bad = false;
-    for (int ks = 0; ks < KS; ++ks) {
-        const float v = amax_part[(size_t)ks * Mc + row];
-        bad = bad || (v != v);
-        a = fmaxf(a, v);
-    }
-    if (bad) a = __int_as_float(0x7fc00000);
-    const float sc = __fdiv_rn(a, qmax);
-    if (threadIdx.x == 0) a_scale[m] = sc;
-    const float rcp = (sc > 0.f) ? __frcp_rn(sc) : 0.f;
-    const __half* xrow = X + (size_t)m * K;
-    int8_t* out = Xq + (size_t)m * K;
+    const int row0 = blockIdx.x * kQRows;
+    const int nrows = (Mc - row0 < kQRows) ? (Mc - row0) : kQRows;
     const int chunks = K / 8;
-    for (int c = threadIdx.x; c < chunks; c += 256) {
-        const RawChunk rc = load_raw(xrow, s, c * 8, true);
-        float v[8];
-        smooth8(rc, v);
-        uint2 q = make_uint2(0u, 0u);
-        if (sc > 0.f) q = quant8_pairs(v, sc, rcp, qmax);
-        *reinterpret_cast<uint2*>(out + c * 8) = q;
+    const int groups = (r + 127) / 128;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const __half* xbase = X + (size_t)(m_first + row0) * K;
+    uint4 x[kQRows];
+    int c = threadIdx.x;
+    auto load_x = [&](int cc) {
+#pragma unroll
+        for (int rr = 0; rr < kQRows; ++rr)
+            x[rr] = (rr < nrows && cc < chunks) ? *reinterpret_cast<const uint4*>(xbase + (size_t)rr * K + cc * 8)
+                                                : make_uint4(0, 0, 0, 0);
+    };
+    load_x(c);
+    grid_dep_wait();        // the partial maxima and the partial T come from act_proj_kernel
+    // ---- scales: warp w takes row w ----
+    if (warp < nrows) {
+        float v = (lane < KS) ? amax_part[(size_t)lane * Mc + row0 + warp] : 0.f;
+        for (int ks = lane + 32; ks < KS; ks += 32) {
+            const float u = amax_part[(size_t)ks * Mc + row0 + warp];
+            v = (u != u || v != v) ? __int_as_float(0x7fc00000) : fmaxf(v, u);
+        }
+        const bool bad = __any_sync(0xffffffffu, v != v);
+        float a = warp_max(v);
+        if (bad) a = __int_as_float(0x7fc00000);
+        if (lane == 0) {
+            const float sc = __fdiv_rn(a, qmax);
+            sc_sm[warp] = sc;
+            rcp_sm[warp] = (sc > 0.f) ? __frcp_rn(sc) : 0.f;
+            a_scale[m_first + row0 + warp] = sc;
+        }
     }
-    for (int j = threadIdx.x; j < r; j += 256) {
+    // ---- T of these rows: the slices' partials summed in slice order ----
+    for (int e = threadIdx.x; e < nrows * r; e += 256) {
+        const int rr = e / r, j = e - rr * r;
+        const float* tp = t_part + ((size_t)(j >> 7) * Mc + row0 + rr) * 128 + (j & 127);
+        const size_t slice = (size_t)groups * Mc * 128;
         float t = 0.f;
-        for (int ks = 0; ks < KS; ++ks) t += t_part[((size_t)ks * Mc + row) * Rp + j];
-        store_t(T + (size_t)m * ldt, j, t, lo_off);
+        for (int ks = 0; ks < KS; ++ks) t += tp[ks * slice];
+        store_t(T + (size_t)(m_first + row0 + rr) * ldt, j, t, lo_off);
+    }
+    __syncthreads();
+    // ---- codes ----
+    const float kMagic = 12582912.0f;       // 1.5 * 2^23: adding it rounds to the nearest integer, ties to even
+    const float2 m2 = make_float2(kMagic, kMagic), nm2 = make_float2(-kMagic, -kMagic);
+    const float2 neg1 = make_float2(-1.f, -1.f);
+    const float kWiden = __uint_as_float(0x77800000u);      // 2^112
+    const float2 widen2 = make_float2(kWiden, kWiden);
+    for (; c < chunks; c += 256) {
+        float4 s0 = make_float4(1.f, 1.f, 1.f, 1.f), s1 = s0;
+        if (s) {
+            s0 = __ldg(reinterpret_cast<const float4*>(s + c * 8));
+            s1 = __ldg(reinterpret_cast<const float4*>(s + c * 8) + 1);
+        }
+        const bool ones = s0.x == 1.f && s0.y == 1.f && s0.z == 1.f && s0.w == 1.f &&
+                          s1.x == 1.f && s1.y == 1.f && s1.z == 1.f && s1.w == 1.f;
+        uint2 q[kQRows];
+#pragma unroll
+        for (int rr = 0; rr < kQRows; ++rr) {
+            // fp16 -> fp32 on the integer and multiply pipes: sign and the 15 value bits moved to
+            // their fp32 places, then times 2^112 (exact for normal and subnormal fp16 values)
+            const uint32_t xw[4] = {x[rr].x, x[rr].y, x[rr].z, x[rr].w};
+            float2 f[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint32_t lo = ((xw[i] & 0x8000u) << 16) | ((xw[i] & 0x7fffu) << 13);
+                const uint32_t hi = (xw[i] & 0x80000000u) | ((xw[i] >> 3) & 0x0fffe000u);
+                f[i] = __fmul2_rn(make_float2(__uint_as_float(lo), __uint_as_float(hi)), widen2);
+            }
+            if (!ones) {        // x~ = x / s, IEEE division, only where the divisor is not 1
+                if (s0.x != 1.f) f[0].x = __fdiv_rn(f[0].x, s0.x);
+                if (s0.y != 1.f) f[0].y = __fdiv_rn(f[0].y, s0.y);
+                if (s0.z != 1.f) f[1].x = __fdiv_rn(f[1].x, s0.z);
+                if (s0.w != 1.f) f[1].y = __fdiv_rn(f[1].y, s0.w);
+                if (s1.x != 1.f) f[2].x = __fdiv_rn(f[2].x, s1.x);
+                if (s1.y != 1.f) f[2].y = __fdiv_rn(f[2].y, s1.y);
+                if (s1.z != 1.f) f[3].x = __fdiv_rn(f[3].x, s1.z);
+                if (s1.w != 1.f) f[3].y = __fdiv_rn(f[3].y, s1.w);
+            }
+            // rne(x~ / sc) == rne(x~ * (1 / sc)) unless the product is within 1e-4 of a tie (the
+            // two differ by less than 3.1e-5): then the whole group takes the exact division
+            const float scr = sc_sm[rr], rc1 = rcp_sm[rr];
+            const float2 r2 = make_float2(rc1, rc1);
+            uint32_t u[8];
+            float far = 0.f;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float2 t = __fmul2_rn(f[i], r2);
+                const float2 su = __fadd2_rn(t, m2);
+                const float2 w = __fadd2_rn(su, nm2);
+                const float2 d = __ffma2_rn(w, neg1, t);
+                u[2 * i] = __float_as_uint(su.x);
+                u[2 * i + 1] = __float_as_uint(su.y);
+                far = fmaxf(far, fmaxf(fabsf(d.x), fabsf(d.y)));
+            }
+            if (scr > 0.f && !(far > 0.4999f)) {
+                const uint32_t a01 = __byte_perm(u[0], u[1], 0x0040), a23 = __byte_perm(u[2], u[3], 0x0040);
+                const uint32_t a45 = __byte_perm(u[4], u[5], 0x0040), a67 = __byte_perm(u[6], u[7], 0x0040);
+                q[rr] = make_uint2(__byte_perm(a01, a23, 0x5410), __byte_perm(a45, a67, 0x5410));
+            } else if (scr > 0.f) {
+                q[rr] = quant8_exact(f[0].x, f[0].y, f[1].x, f[1].y, f[2].x, f[2].y, f[3].x, f[3].y, scr, qmax);
+            } else {
+                q[rr] = make_uint2(0u, 0u);     // zero row, or a poisoned scale
+            }
+        }
+        load_x(c + 256);        // the next iteration's loads are in flight during the stores
+#pragma unroll
+        for (int rr = 0; rr < kQRows; ++rr)
+            if (rr < nrows) *reinterpret_cast<uint2*>(Xq + (size_t)(m_first + row0 + rr) * K + c * 8) = q[rr];
     }
 }
 
@@ -375,10 +502,14 @@ ProjPlan proj_plan(int M, int K, int num_sms) {
     return best;
 }
 
+// Floats of the row-maxima part of the scratch, padded so that the partial T behind it starts on
+// a 128-byte boundary (it is written by bulk copies, which need 16-byte alignment).
+size_t proj_amax_floats(const ProjPlan& p) { return ((size_t)p.KS * p.Mc + 31) & ~(size_t)31; }
+
 size_t proj_scratch_bytes(int M, int K, int r, int num_sms) {
     const ProjPlan p = proj_plan(M, K, num_sms);
-    const int Rp = (r + 31) / 32 * 32;
-    return (size_t)p.KS * p.Mc * (1 + Rp) * sizeof(float);
+    const int groups = (r + 127) / 128;
+    return (proj_amax_floats(p) + (size_t)p.KS * p.Mc * groups * 128) * sizeof(float);
 }
 
 }  // namespace
@@ -386,6 +517,12 @@ size_t proj_scratch_bytes(int M, int K, int r, int num_sms) {
 size_t quant_act_ws_scratch_bytes(int M, int K, int r) {
     if (M <= 32) return 0;
     return proj_scratch_bytes(M, K, r, kProjPlanSms);
+}
+
+int quant_act_ws_launches(int M, int K) {
+    if (M <= 32) return 1;
+    const ProjPlan plan = proj_plan(M, K, kProjPlanSms);
+    return 2 * ((M + plan.Mc - 1) / plan.Mc);
 }
 
 int launch_quant_act_ws(const __half* X, const float* s, const __half* LA, int M, int K, int r,
@@ -396,13 +533,14 @@ int launch_quant_act_ws(const __half* X, const float* s, const __half* LA, int M
     const int groups = (r + 127) / 128;
     if (groups > kPMaxGroups) return record_error(ASER_ERR_SHAPE, "quant_act: r beyond 512");
     const ProjPlan plan = proj_plan(M, K, kProjPlanSms);
-    const int Rp = (r + 31) / 32 * 32;
-    if (scratch == nullptr || scratch_bytes < (size_t)plan.KS * plan.Mc * (1 + Rp) * sizeof(float))
+    if (scratch == nullptr || misaligned16(scratch) ||
+        scratch_bytes < (proj_amax_floats(plan) + (size_t)plan.KS * plan.Mc * groups * 128) * sizeof(float))
         return record_error(ASER_ERR_WORKSPACE, "quant_act: scratch missing or too small");
     float* amax_part = static_cast<float*>(scratch);
-    float* t_part = amax_part + (size_t)plan.KS * plan.Mc;
+    float* t_part = amax_part + proj_amax_floats(plan);
     const int Kc = K / plan.KS;
     const int NS = proj_stages(groups);
+    // the ring (at least 128 KB with a projection: it later stages the partial T) and the tail
     const size_t smem = (size_t)NS * kPTileBytes * (1 + groups) + 256 + ((Kc / 8 + 15) & ~15) +
                         kPConsumerWarps * kPTok * sizeof(float) + 1024;
     static size_t configured[kMaxDevices] = {0};
@@ -420,7 +558,7 @@ int launch_quant_act_ws(const __half* X, const float* s, const __half* LA, int M
     int rc = encode_map_blocks(&mx, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, X, M, K, kPTok, 1);
     if (rc != ASER_OK) return rc;
     if (r > 0) {
-        rc = encode_map_blocks(&mla, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, LA, r, K, r < 128 ? r : 128, 1);
+        rc = encode_map_blocks(&mla, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, LA, r, K, r <= 256 ? r : r / 2, 1);
         if (rc != ASER_OK) return rc;
     } else {
         mla = mx;
@@ -428,12 +566,12 @@ int launch_quant_act_ws(const __half* X, const float* s, const __half* LA, int M
     for (int m_first = 0; m_first < M; m_first += plan.Mc) {
         const int Mc = (M - m_first < plan.Mc) ? (M - m_first) : plan.Mc;
         const int tiles = (Mc + kPTok - 1) / kPTok;
-        act_proj_kernel<<<dim3(plan.KS, tiles, 1), kPThreads, smem, st>>>(mx, mla, s, m_first, Mc, K, Kc, r, Rp,
+        act_proj_kernel<<<dim3(plan.KS, tiles, 1), kPThreads, smem, st>>>(mx, mla, s, m_first, Mc, K, Kc, r,
                                                                           amax_part, t_part);
         rc = check_launch("act_proj_kernel");
         if (rc != ASER_OK) return rc;
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(Mc, 1, 1);
+        cfg.gridDim = dim3((Mc + kQRows - 1) / kQRows, 1, 1);
         cfg.blockDim = dim3(256, 1, 1);
         cfg.stream = st;
         cudaLaunchAttribute attr[1];
@@ -441,7 +579,7 @@ int launch_quant_act_ws(const __half* X, const float* s, const __half* LA, int M
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        cudaError_t e = cudaLaunchKernelEx(&cfg, act_quant_kernel, X, s, m_first, Mc, K, r, Rp, plan.KS,
+        cudaError_t e = cudaLaunchKernelEx(&cfg, act_quant_kernel, X, s, m_first, Mc, K, r, plan.KS,
                                            (const float*)amax_part, (const float*)t_part, Xq, a_scale, T, ldt,
                                            lo_off, qmax);
         if (e != cudaSuccess) return record_cuda_error(e, "act_quant_kernel");

@@ -282,6 +282,11 @@ size_t aser_quant_workspace_bytes(int M, int K, int r) {
     return kWsZeroedBytes + quant_act_ws_scratch_bytes(M, K, r);
 }
 
+int aser_quant_act_ws_launches(int M, int K) {
+    if (!act_shape_ok(M, K, 0) || M == 0) return 0;
+    return quant_act_ws_launches(M, K);
+}
+
 int aser_quant_act_ws(const void* X_f16, const float* s, const void* LA_f16, int M, int K, int r,
                       int act_bits, int t_pair, int8_t* Xq, float* a_scale, void* T_bf16,
                       void* workspace, size_t workspace_bytes, void* stream) {

@@ -40,6 +40,7 @@ int launch_quant_act(const __half* X, const float* s, const __half* LA, int M, i
 // The same with caller-provided scratch (quant_act_ws_scratch_bytes): the two-kernel path for more
 // than 32 tokens, ranks up to 512 (stacked down projections of layers that share X).
 size_t quant_act_ws_scratch_bytes(int M, int K, int r);
+int quant_act_ws_launches(int M, int K);     // kernels one call enqueues
 int launch_quant_act_ws(const __half* X, const float* s, const __half* LA, int M, int K, int r,
                         int8_t* Xq, float* a_scale, __nv_bfloat16* T, void* scratch, size_t scratch_bytes,
                         cudaStream_t st, int act_bits = 8, bool t_pair = false);

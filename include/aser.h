@@ -280,6 +280,32 @@ int aser_forward_host(const void* X_host_f16, void* Y_host_f16,
                       const void* LB_f16, int M, int N, int K, int r,
                       void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * aser_construct -- the per-layer body of Algorithm 1 on the device: quantize W diag(s) to int4
+ * (aser_pack_w4), form the error E = W diag(s) - dequant(W_q), whiten with the Cholesky factor S
+ * of the calibration Gram matrix (Sec. 4.1 Eq. 5; the paper's X X^T is X~^T X~ here, X~ =
+ * X_cal diag(s)^-1, damped by lambda I with lambda = damping * trace / K because the Gram matrix
+ * is singular with fewer calibration tokens than channels), take the r leading singular triplets
+ * of E S (Eq. 6) and split them into L_B = U_r Sigma_r [N, r] and L_A = V_r^T S^-1 [r, K] (the
+ * paper's L_A and L_B, in that order).  fp64 throughout, factors rounded to fp16 at the end.
+ *   W_f16 [N, K], s [K] or NULL, Xcal_f16 [n_cal, K] calibration tokens (NOT yet smoothed).
+ *   iterations: subspace iterations for the singular subspace (<= 0: 48); p = r + max(32, r/2)
+ *   vectors are iterated, so the r-th triplet converges like (sigma_{p+1} / sigma_r)^(2 iterations).
+ *   Outputs: Wq [N, K/2] canonical, w_scale [N], LA_f16 [r, K], LB_f16 [N, r]; optional
+ *   sigma_out [r] (fp64 singular values, descending) and S_out [K, K] (fp64, lower, row-major).
+ *   workspace: aser_construct_workspace_bytes(N, K, n_cal, r) bytes (several N*K and K*K fp64
+ *   matrices).
+ * Singular vectors are determined up to sign (and up to rotation among equal singular values):
+ * compare the product L_B L_A and the singular values, not the factors element by element.
+ * An offline step: the call SYNCHRONISES `stream` before it returns, and returns ASER_ERR_SHAPE
+ * if the damped Gram matrix turned out not to be positive definite.  r == 0 only packs.
+ */
+size_t aser_construct_workspace_bytes(int N, int K, int n_cal, int r);
+int aser_construct(const void* W_f16, const float* s, const void* Xcal_f16, int N, int K, int n_cal,
+                   int r, double damping, int iterations, uint8_t* Wq, float* w_scale,
+                   void* LA_f16, void* LB_f16, double* sigma_out, double* S_out,
+                   void* workspace, size_t workspace_bytes, void* stream);
+
 /* Text of the last CUDA error seen by the calling thread ("" if none). */
 const char* aser_last_error(void);
 /* Library version: major * 1000 + minor. */

@@ -13,7 +13,7 @@ EXPORTED_SYMBOLS = (
     "aser_pack_w4", "aser_repacked_bytes", "aser_repack_w4", "aser_unrepack_w4",
     "aser_quant_act", "aser_quant_act_bits", "aser_quant_act_ex", "aser_quant_act_ws",
     "aser_quant_workspace_bytes", "aser_quant_act_ws_launches", "aser_linear_w4a8_lr_ld", "aser_forward_shared",
-    "aser_forward_shared_workspace_bytes", "aser_linear_w4a8_lr", "aser_linear_w4a8", "aser_linear_w4a8_lr_simt", "aser_linear_w4a8_lr_static",
+    "aser_forward_shared_workspace_bytes", "aser_construct", "aser_construct_workspace_bytes", "aser_linear_w4a8_lr", "aser_linear_w4a8", "aser_linear_w4a8_lr_simt", "aser_linear_w4a8_lr_static",
     "aser_workspace_bytes", "aser_workspace_init", "aser_check_status", "aser_forward",
     "aser_forward_host",
     "aser_last_error", "aser_version",
@@ -54,6 +54,9 @@ lib.aser_check_status.argtypes = [_P, _P]
 lib.aser_forward.argtypes = [_P, _P, _P, _P, _P, _P, _I, _I, _I, _I, _P, _P, _P, _P, _P, _Z, _P]
 lib.aser_forward_host.argtypes = [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P,
                                   _I, _I, _I, _I, _P, _Z, _P]
+lib.aser_construct_workspace_bytes.argtypes = [_I, _I, _I, _I]
+lib.aser_construct_workspace_bytes.restype = _Z
+lib.aser_construct.argtypes = [_P, _P, _P, _I, _I, _I, _I, C.c_double, _I, _P, _P, _P, _P, _P, _P, _P, _Z, _P]
 lib.aser_last_error.restype = C.c_char_p
 lib.aser_version.restype = _I
 
@@ -255,6 +258,30 @@ def linear_w4a8_lr_static(Xq, a_scale, Wk, w_scale, T, L_B, N: int, Y=None, acc_
                                         r, _ptr(Y), _ptr(acc_debug), _stream()),
          "aser_linear_w4a8_lr_static")
     return Y
+
+
+def construct(W: torch.Tensor, s, X_cal: torch.Tensor, r: int, damping: float = 0.01, iterations: int = 0,
+              want_S: bool = False):
+    """aser_construct: int4 weights and rank-r factors of one layer built on the device from W
+    fp16 [N,K], s fp32 [K] and calibration tokens fp16 [n_cal,K].  Returns a dict with Wq, w_scale,
+    L_A fp16 [r,K], L_B fp16 [N,r], sigma fp64 [r] and (want_S) the whitening factor S fp64 [K,K]."""
+    _dev(W, torch.float16, "W")
+    _dev(X_cal, torch.float16, "X_cal")
+    N, K = W.shape
+    n_cal = X_cal.shape[0]
+    dev = W.device
+    Wq = torch.empty((N, K // 2), dtype=torch.uint8, device=dev)
+    w_scale = torch.empty((N,), dtype=torch.float32, device=dev)
+    L_A = torch.empty((max(r, 1), K), dtype=torch.float16, device=dev)
+    L_B = torch.empty((N, max(r, 1)), dtype=torch.float16, device=dev)
+    sigma = torch.empty((max(r, 1),), dtype=torch.float64, device=dev)
+    S = torch.empty((K, K), dtype=torch.float64, device=dev) if want_S else None
+    nbytes = int(lib.aser_construct_workspace_bytes(N, K, n_cal, r))
+    ws = torch.empty((max(nbytes, 256),), dtype=torch.uint8, device=dev)
+    _chk(lib.aser_construct(_ptr(W), _ptr(s), _ptr(X_cal), N, K, n_cal, r, float(damping), int(iterations),
+                            _ptr(Wq), _ptr(w_scale), _ptr(L_A), _ptr(L_B), _ptr(sigma), _ptr(S), _ptr(ws),
+                            ws.numel(), _stream()), "aser_construct")
+    return dict(Wq=Wq, w_scale=w_scale, L_A=L_A[:r], L_B=L_B[:, :r].contiguous(), sigma=sigma[:r], S=S)
 
 
 def pair_up_projection(L_B: torch.Tensor) -> torch.Tensor:

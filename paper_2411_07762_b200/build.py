@@ -14,7 +14,7 @@ OBJ_DIR = os.path.join(_HERE, "_build")
 LIB = os.path.join(_HERE, "libaser.so")
 
 SOURCES = ["api.cu", "pack_w4.cu", "quant_act.cu", "act_proj.cu", "linear_simt.cu", "linear_tc.cu",
-           "linear_decode.cu", "linear_static.cu"]
+           "linear_decode.cu", "linear_static.cu", "construct.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC]
 

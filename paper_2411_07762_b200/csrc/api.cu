@@ -270,6 +270,40 @@ int aser_linear_w4a8_lr_simt(const int8_t* Xq, const float* a_scale, const uint8
                               static_cast<cudaStream_t>(stream));
 }
 
+size_t aser_construct_workspace_bytes(int N, int K, int n_cal, int r) {
+    if (!shape_ok(0, N, K, r) || N <= 0 || n_cal <= 0) return 0;
+    return construct_workspace_bytes(N, K, n_cal, r);
+}
+
+int aser_construct(const void* W_f16, const float* s, const void* Xcal_f16, int N, int K, int n_cal, int r,
+                   double damping, int iterations, uint8_t* Wq, float* w_scale, void* LA_f16,
+                   void* LB_f16, double* sigma_out, double* S_out, void* workspace,
+                   size_t workspace_bytes, void* stream) {
+    if (!shape_ok(0, N, K, r) || N <= 0 || n_cal <= 0 || r > (N < K ? N : K))
+        return fail(ASER_ERR_SHAPE, "unsupported N, K, n_cal or r");
+    if (!(damping > 0.0)) return fail(ASER_ERR_SHAPE, "damping must be positive");
+    ASER_REQUIRE_PTR(W_f16);
+    ASER_OPTIONAL_PTR(s);
+    ASER_REQUIRE_PTR(Xcal_f16);
+    ASER_REQUIRE_PTR(Wq);
+    ASER_REQUIRE_PTR(w_scale);
+    if (r > 0) {
+        ASER_REQUIRE_PTR(LA_f16);
+        ASER_REQUIRE_PTR(LB_f16);
+    }
+    ASER_OPTIONAL_PTR(sigma_out);
+    ASER_OPTIONAL_PTR(S_out);
+    if (workspace == nullptr || misaligned16(workspace) ||
+        workspace_bytes < aser_construct_workspace_bytes(N, K, n_cal, r))
+        return fail(ASER_ERR_WORKSPACE, "workspace missing, misaligned or too small");
+    int rc = check_device();
+    if (rc != ASER_OK) return rc;
+    return launch_construct(static_cast<const __half*>(W_f16), s, static_cast<const __half*>(Xcal_f16), N, K,
+                            n_cal, r, damping, iterations > 0 ? iterations : 48, Wq, w_scale,
+                            static_cast<__half*>(LA_f16), static_cast<__half*>(LB_f16), sigma_out, S_out,
+                            workspace, static_cast<cudaStream_t>(stream));
+}
+
 size_t aser_workspace_bytes(int M, int N, int K, int r) {
     if (!shape_ok(M, N, K, r)) return 0;
     const size_t lin = kWsHeaderBytes + linear_tc_workspace_bytes(M, N, K, r);

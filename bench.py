@@ -693,6 +693,7 @@ def run_ours(args, rank, world, local_rank):
     torch.cuda.empty_cache()
     if rank == 0 and world == 1 and args.extra:
         line["extra_points"] = extra_points(dev, peaks, lib_int8, skip=name)
+        line["variants"] = variant_points(dev)
     if rank == 0 and world == 1 and not args.no_cpu:
         line["cpu_baseline"] = time_oracle(name)
     if rank == 0:
@@ -728,6 +729,84 @@ def extra_points(dev, peaks, lib_int8, skip):
         out.append(pt)
         del m
         torch.cuda.empty_cache()
+    return out
+
+
+def time_callable(torch, fn, calls=8, repeats=REPEATS):
+    """Median ms per call of fn() replayed from a CUDA graph (regions of at least MIN_REGION_MS)."""
+    side = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g, stream=side):
+            for _ in range(calls):
+                fn()
+    torch.cuda.synchronize()
+
+    def once(n):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+    n = max(1, int(np.ceil(MIN_REGION_MS / max(once(1), 1e-3))))
+    return statistics.median(once(n) / (n * calls) for _ in range(repeats))
+
+
+def variant_points(dev):
+    """The paper's own variant beside the default, on one 4096 x 4096 layer at 2048 tokens, rank 64,
+    512 calibration tokens, factors built on the device (aser_construct):
+      default  smoothing s = sqrt(max|X_c| / max|W_c|) on the seeded outlier channels, all columns
+               quantized, T in bf16;
+      split    the paper's m_i = mean|X_i| / min over the f = 32 outlier channels of
+               mean|X| * mean|W| (Sec. 4.2 Eq. 11), those columns kept out of the int4 matrix and
+               carried by the factors (Eq. 12), T as bf16 pairs (rank 128 in the linear kernel).
+    Reports the time of a step and the reconstruction error ||Y - X W^T||_F / ||X W^T||_F against
+    the fp32 product of the fp16 operands, with plain W4A8 (no factors) as the yardstick."""
+    import torch
+    import paper_2411_07762_b200 as aser
+    N = K = 4096
+    M, r, f = 2048, 64, 32
+    lay = synth.make_layer(M, N, K, seed=synth.seed_for(2, 4242), outlier_gain=30.0, sigma_w=0.02, n_cal=512)
+    t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+    W, X, Xc = t(lay.W), t(lay.X), t(lay.X_cal)
+    exact = X.float() @ W.float().t()
+    den = float(exact.norm())
+    out = {}
+    # default
+    idx = torch.from_numpy(lay.outlier_idx).to(dev)
+    s = torch.ones(K, dtype=torch.float32, device=dev)
+    s[idx] = torch.sqrt(Xc[:, idx].float().abs().amax(0) / W[:, idx].float().abs().amax(0))
+    c = aser.construct(W, s, Xc, r)
+    layer = aser.AserLinear(W, s, c["L_A"].contiguous(), c["L_B"], M)
+    assert torch.equal(layer.Wq, c["Wq"])
+    Y = layer(X).float()
+    out["default"] = dict(rel_error=float((Y - exact).norm()) / den, us_step=time_callable(torch, lambda: layer(X)) * 1e3)
+    Yp = layer(X, lowrank=False).float()
+    out["plain_w4a8"] = dict(rel_error=float((Yp - exact).norm()) / den,
+                             us_step=time_callable(torch, lambda: layer(X, lowrank=False)) * 1e3)
+    # the paper's smoothing rule and outlier split
+    xbar, wbar = Xc.float().abs().mean(0), W.float().abs().mean(0)
+    idx_f = torch.topk(xbar * wbar, f).indices.sort().values
+    m = torch.ones(K, dtype=torch.float32, device=dev)
+    m[idx_f] = xbar[idx_f] / xbar[idx_f].min()
+    c2 = aser.construct(W, m, Xc, r, split_idx=idx_f.to(torch.int32))
+    Wk = aser.repack_w4(c2["Wq"])
+    LA2, LB2 = c2["L_A"].contiguous(), aser.pair_up_projection(c2["L_B"])
+    ws = aser.new_workspace(M, N, K, 2 * r)
+    bufs = (torch.empty((M, K), dtype=torch.int8, device=dev), torch.empty((M,), dtype=torch.float32, device=dev),
+            torch.empty((M, 2 * r), dtype=torch.bfloat16, device=dev))
+    Y2 = torch.empty((M, N), dtype=torch.float16, device=dev)
+
+    def split_step():
+        Xq, sc, T = aser.quant_act_ws(X, m, LA2, ws=ws, out=bufs, t_pair=True)
+        aser.linear_w4a8_lr(Xq, sc, Wk, c2["w_scale"], T, LB2, N, ws, Y=Y2)
+    split_step()
+    aser.check_status(ws)
+    out["paper_split"] = dict(rel_error=float((Y2.float() - exact).norm()) / den,
+                              us_step=time_callable(torch, split_step) * 1e3, f=f)
+    out["shape"] = dict(M=M, N=N, K=K, r=r, n_cal=512)
     return out
 
 

@@ -293,17 +293,22 @@ int aser_forward_host(const void* X_host_f16, void* Y_host_f16,
  *   vectors are iterated, so the r-th triplet converges like (sigma_{p+1} / sigma_r)^(2 iterations).
  *   Outputs: Wq [N, K/2] canonical, w_scale [N], LA_f16 [r, K], LB_f16 [N, r]; optional
  *   sigma_out [r] (fp64 singular values, descending) and S_out [K, K] (fp64, lower, row-major).
- *   workspace: aser_construct_workspace_bytes(N, K, n_cal, r) bytes (several N*K and K*K fp64
- *   matrices).
+ *   split_idx [n_split] (device, int32; NULL with n_split = 0): the outlier columns of the
+ *   paper's split W M = W_s + W_o (Sec. 4.2 Eq. 12).  They are zeroed before the int4 quantizer
+ *   (Wq then holds W_s only) and stay in the error E, so the factors carry them.  A forward pass
+ *   of such a layer wants T stored as bf16 pairs (aser_quant_act_ex).
+ *   workspace: aser_construct_workspace_bytes(N, K, n_cal, r, n_split) bytes (several N*K and
+ *   K*K fp64 matrices).
  * Singular vectors are determined up to sign (and up to rotation among equal singular values):
  * compare the product L_B L_A and the singular values, not the factors element by element.
  * An offline step: the call SYNCHRONISES `stream` before it returns, and returns ASER_ERR_SHAPE
  * if the damped Gram matrix turned out not to be positive definite.  r == 0 only packs.
  */
-size_t aser_construct_workspace_bytes(int N, int K, int n_cal, int r);
+size_t aser_construct_workspace_bytes(int N, int K, int n_cal, int r, int n_split);
 int aser_construct(const void* W_f16, const float* s, const void* Xcal_f16, int N, int K, int n_cal,
                    int r, double damping, int iterations, uint8_t* Wq, float* w_scale,
                    void* LA_f16, void* LB_f16, double* sigma_out, double* S_out,
+                   const int32_t* split_idx, int n_split,
                    void* workspace, size_t workspace_bytes, void* stream);
 
 /* Text of the last CUDA error seen by the calling thread ("" if none). */

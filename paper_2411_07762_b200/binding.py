@@ -54,9 +54,9 @@ lib.aser_check_status.argtypes = [_P, _P]
 lib.aser_forward.argtypes = [_P, _P, _P, _P, _P, _P, _I, _I, _I, _I, _P, _P, _P, _P, _P, _Z, _P]
 lib.aser_forward_host.argtypes = [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P,
                                   _I, _I, _I, _I, _P, _Z, _P]
-lib.aser_construct_workspace_bytes.argtypes = [_I, _I, _I, _I]
+lib.aser_construct_workspace_bytes.argtypes = [_I, _I, _I, _I, _I]
 lib.aser_construct_workspace_bytes.restype = _Z
-lib.aser_construct.argtypes = [_P, _P, _P, _I, _I, _I, _I, C.c_double, _I, _P, _P, _P, _P, _P, _P, _P, _Z, _P]
+lib.aser_construct.argtypes = [_P, _P, _P, _I, _I, _I, _I, C.c_double, _I, _P, _P, _P, _P, _P, _P, _P, _I, _P, _Z, _P]
 lib.aser_last_error.restype = C.c_char_p
 lib.aser_version.restype = _I
 
@@ -261,7 +261,7 @@ def linear_w4a8_lr_static(Xq, a_scale, Wk, w_scale, T, L_B, N: int, Y=None, acc_
 
 
 def construct(W: torch.Tensor, s, X_cal: torch.Tensor, r: int, damping: float = 0.01, iterations: int = 0,
-              want_S: bool = False):
+              want_S: bool = False, split_idx: torch.Tensor | None = None):
     """aser_construct: int4 weights and rank-r factors of one layer built on the device from W
     fp16 [N,K], s fp32 [K] and calibration tokens fp16 [n_cal,K].  Returns a dict with Wq, w_scale,
     L_A fp16 [r,K], L_B fp16 [N,r], sigma fp64 [r] and (want_S) the whitening factor S fp64 [K,K]."""
@@ -276,10 +276,14 @@ def construct(W: torch.Tensor, s, X_cal: torch.Tensor, r: int, damping: float = 
     L_B = torch.empty((N, max(r, 1)), dtype=torch.float16, device=dev)
     sigma = torch.empty((max(r, 1),), dtype=torch.float64, device=dev)
     S = torch.empty((K, K), dtype=torch.float64, device=dev) if want_S else None
-    nbytes = int(lib.aser_construct_workspace_bytes(N, K, n_cal, r))
+    n_split = 0 if split_idx is None else int(split_idx.numel())
+    if n_split:
+        _dev(split_idx, torch.int32, "split_idx")
+    nbytes = int(lib.aser_construct_workspace_bytes(N, K, n_cal, r, n_split))
     ws = torch.empty((max(nbytes, 256),), dtype=torch.uint8, device=dev)
     _chk(lib.aser_construct(_ptr(W), _ptr(s), _ptr(X_cal), N, K, n_cal, r, float(damping), int(iterations),
-                            _ptr(Wq), _ptr(w_scale), _ptr(L_A), _ptr(L_B), _ptr(sigma), _ptr(S), _ptr(ws),
+                            _ptr(Wq), _ptr(w_scale), _ptr(L_A), _ptr(L_B), _ptr(sigma), _ptr(S),
+                            _ptr(split_idx) if n_split else None, n_split, _ptr(ws),
                             ws.numel(), _stream()), "aser_construct")
     return dict(Wq=Wq, w_scale=w_scale, L_A=L_A[:r], L_B=L_B[:, :r].contiguous(), sigma=sigma[:r], S=S)
 

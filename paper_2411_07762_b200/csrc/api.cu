@@ -270,18 +270,20 @@ int aser_linear_w4a8_lr_simt(const int8_t* Xq, const float* a_scale, const uint8
                               static_cast<cudaStream_t>(stream));
 }
 
-size_t aser_construct_workspace_bytes(int N, int K, int n_cal, int r) {
-    if (!shape_ok(0, N, K, r) || N <= 0 || n_cal <= 0) return 0;
-    return construct_workspace_bytes(N, K, n_cal, r);
+size_t aser_construct_workspace_bytes(int N, int K, int n_cal, int r, int n_split) {
+    if (!shape_ok(0, N, K, r) || N <= 0 || n_cal <= 0 || n_split < 0) return 0;
+    return construct_workspace_bytes(N, K, n_cal, r, n_split);
 }
 
 int aser_construct(const void* W_f16, const float* s, const void* Xcal_f16, int N, int K, int n_cal, int r,
                    double damping, int iterations, uint8_t* Wq, float* w_scale, void* LA_f16,
-                   void* LB_f16, double* sigma_out, double* S_out, void* workspace,
-                   size_t workspace_bytes, void* stream) {
+                   void* LB_f16, double* sigma_out, double* S_out, const int32_t* split_idx, int n_split,
+                   void* workspace, size_t workspace_bytes, void* stream) {
     if (!shape_ok(0, N, K, r) || N <= 0 || n_cal <= 0 || r > (N < K ? N : K))
         return fail(ASER_ERR_SHAPE, "unsupported N, K, n_cal or r");
     if (!(damping > 0.0)) return fail(ASER_ERR_SHAPE, "damping must be positive");
+    if (n_split < 0 || n_split > K) return fail(ASER_ERR_SHAPE, "n_split out of range");
+    if (n_split > 0 && split_idx == nullptr) return fail(ASER_ERR_NULL, "split_idx is NULL");
     ASER_REQUIRE_PTR(W_f16);
     ASER_OPTIONAL_PTR(s);
     ASER_REQUIRE_PTR(Xcal_f16);
@@ -294,14 +296,14 @@ int aser_construct(const void* W_f16, const float* s, const void* Xcal_f16, int 
     ASER_OPTIONAL_PTR(sigma_out);
     ASER_OPTIONAL_PTR(S_out);
     if (workspace == nullptr || misaligned16(workspace) ||
-        workspace_bytes < aser_construct_workspace_bytes(N, K, n_cal, r))
+        workspace_bytes < aser_construct_workspace_bytes(N, K, n_cal, r, n_split))
         return fail(ASER_ERR_WORKSPACE, "workspace missing, misaligned or too small");
     int rc = check_device();
     if (rc != ASER_OK) return rc;
     return launch_construct(static_cast<const __half*>(W_f16), s, static_cast<const __half*>(Xcal_f16), N, K,
                             n_cal, r, damping, iterations > 0 ? iterations : 48, Wq, w_scale,
                             static_cast<__half*>(LA_f16), static_cast<__half*>(LB_f16), sigma_out, S_out,
-                            workspace, static_cast<cudaStream_t>(stream));
+                            split_idx, n_split, workspace, static_cast<cudaStream_t>(stream));
 }
 
 size_t aser_workspace_bytes(int M, int N, int K, int r) {

@@ -45,10 +45,11 @@ int launch_quant_act_ws(const __half* X, const float* s, const __half* LA, int M
                         int8_t* Xq, float* a_scale, __nv_bfloat16* T, void* scratch, size_t scratch_bytes,
                         cudaStream_t st, int act_bits = 8, bool t_pair = false);
 // Device-side construction of a layer's factors (construct.cu); synchronises the stream.
-size_t construct_workspace_bytes(int N, int K, int Tcal, int r);
+size_t construct_workspace_bytes(int N, int K, int Tcal, int r, int n_split);
 int launch_construct(const __half* W, const float* s, const __half* Xcal, int N, int K, int Tcal, int r,
                      double damping, int iters, uint8_t* Wq, float* w_scale, __half* LA, __half* LB,
-                     double* sigma_out, double* S_out, void* workspace, cudaStream_t st);
+                     double* sigma_out, double* S_out, const int* split_idx, int n_split, void* workspace,
+                     cudaStream_t st);
 int launch_linear_simt(const int8_t* Xq, const float* a_scale, const uint8_t* Wq,
                        const float* w_scale, const __nv_bfloat16* T, const __half* LB,
                        int M, int N, int K, int r, __half* Y, int32_t* acc_debug, cudaStream_t st);

@@ -212,6 +212,18 @@ __global__ void build_error_kernel(const __half* __restrict__ W, const float* __
     E[e] = (double)ws - (double)q * (double)w_scale[n];
 }
 
+// Copy of W with the columns of the outlier set zeroed: what the quantizer sees under the outlier
+// split of Sec. 4.2 (Eq. 12), where those columns are carried by the factors alone.
+__global__ void mask_columns_kernel(const __half* __restrict__ W, int N, int K, const int* __restrict__ idx,
+                                    int n_idx, __half* __restrict__ Wm) {
+    const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= (long long)N * K) return;
+    const int k = (int)(e % K);
+    bool out = false;
+    for (int i = 0; i < n_idx; ++i) out = out || (idx[i] == k);
+    Wm[e] = out ? __float2half(0.f) : W[e];
+}
+
 // X~ = fp32(X) / s (one fp32 division), in fp64.
 __global__ void build_xs_kernel(const __half* __restrict__ X, const float* __restrict__ s, int T, int K,
                                 double* __restrict__ Xs) {
@@ -343,10 +355,10 @@ __global__ void to_half_kernel(const double* __restrict__ src, long long n, __ha
 
 struct ConstructLayout {
     int p;
-    size_t E, A, G, Xs, Qt, Zt, Yt, C, Vt, norms, lambda, order, fail, total;     // byte offsets
+    size_t E, A, G, Xs, Qt, Zt, Yt, C, Vt, norms, lambda, order, fail, Wm, total;     // byte offsets
 };
 
-ConstructLayout construct_layout(int N, int K, int Tcal, int r) {
+ConstructLayout construct_layout(int N, int K, int Tcal, int r, int n_split) {
     ConstructLayout L;
     int p = r + (r / 2 > 32 ? r / 2 : 32);
     p += p & 1;
@@ -368,6 +380,7 @@ ConstructLayout construct_layout(int N, int K, int Tcal, int r) {
     L.lambda = take(8);
     L.order = take((size_t)(r > 0 ? r : 1) * 4);
     L.fail = take(4);
+    L.Wm = take(n_split > 0 ? (size_t)N * K * 2 : 0);
     L.total = off;
     return L;
 }
@@ -389,12 +402,15 @@ int orthonormalize_rows(cudaStream_t st, double* Z, int p, int K, double* C, int
 
 }  // namespace
 
-size_t construct_workspace_bytes(int N, int K, int Tcal, int r) { return construct_layout(N, K, Tcal, r).total; }
+size_t construct_workspace_bytes(int N, int K, int Tcal, int r, int n_split) {
+    return construct_layout(N, K, Tcal, r, n_split).total;
+}
 
 int launch_construct(const __half* W, const float* s, const __half* Xcal, int N, int K, int Tcal, int r,
                      double damping, int iters, uint8_t* Wq, float* w_scale, __half* LA, __half* LB,
-                     double* sigma_out, double* S_out, void* workspace, cudaStream_t st) {
-    const ConstructLayout L = construct_layout(N, K, Tcal, r);
+                     double* sigma_out, double* S_out, const int* split_idx, int n_split, void* workspace,
+                     cudaStream_t st) {
+    const ConstructLayout L = construct_layout(N, K, Tcal, r, n_split);
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     double* E = reinterpret_cast<double*>(ws + L.E);
     double* A = reinterpret_cast<double*>(ws + L.A);
@@ -411,7 +427,13 @@ int launch_construct(const __half* W, const float* s, const __half* Xcal, int N,
     int* fail = reinterpret_cast<int*>(ws + L.fail);
     const int p = L.p;
 
-    int rc = launch_pack_w4(W, s, N, K, Wq, w_scale, st);
+    const __half* Wquant = W;
+    if (n_split > 0) {      // the quantizer sees W without the outlier columns; E below keeps them
+        __half* Wm = reinterpret_cast<__half*>(ws + L.Wm);
+        mask_columns_kernel<<<blocks_for((long long)N * K, 256), 256, 0, st>>>(W, N, K, split_idx, n_split, Wm);
+        Wquant = Wm;
+    }
+    int rc = launch_pack_w4(Wquant, s, N, K, Wq, w_scale, st);
     if (rc != ASER_OK) return rc;
     if (r == 0) return ASER_OK;
     cudaError_t e = cudaMemsetAsync(fail, 0, sizeof(int), st);

@@ -21,11 +21,17 @@ def aser(cuda_device):
     return aser
 
 
-def _check(aser, lay, r, iterations=0):
-    s = Cn.smoothing_vector_config(lay.X_cal, lay.W, lay.outlier_idx)
-    L = Cn.construct_layer(lay.W, lay.X_cal, s, r=r)
+def _check(aser, lay, r, iterations=0, split=False):
+    if split:       # the paper's own smoothing rule (Eq. 11) and outlier split (Eq. 12)
+        s, idx = Cn.smoothing_vector_paper(lay.X_cal, lay.W, f=len(lay.outlier_idx))
+        L = Cn.construct_layer(lay.W, lay.X_cal, s, r=r, split_outliers=idx)
+        split_idx = to_dev(idx.astype(np.int32))
+    else:
+        s = Cn.smoothing_vector_config(lay.X_cal, lay.W, lay.outlier_idx)
+        L = Cn.construct_layer(lay.W, lay.X_cal, s, r=r)
+        split_idx = None
     out = aser.construct(to_dev(lay.W), to_dev(s), to_dev(lay.X_cal), r, damping=0.01,
-                         iterations=iterations, want_S=True)
+                         iterations=iterations, want_S=True, split_idx=split_idx)
     torch.cuda.synchronize()
     # quantizer: bit-exact
     assert np.array_equal(out["Wq"].cpu().numpy(), L.Wq)
@@ -74,6 +80,14 @@ def test_construct_config1_tiny_and_forward_with_its_factors(aser):
 def test_construct_matches_oracle_invariants(aser, N, K, r, n_cal):
     lay = synth.make_layer(4, N, K, seed=synth.seed_for(2, N + K + r), n_cal=n_cal)
     _check(aser, lay, r)
+
+
+def test_construct_with_outlier_split(aser):
+    """The split variant: the outlier columns are zero in Wq and the factors carry them."""
+    lay = synth.make_layer(4, 512, 512, seed=synth.seed_for(1, 9), n_out=4, outlier_gain=40.0, n_cal=128)
+    s, L, out = _check(aser, lay, 32, split=True)
+    q = F.unpack_w4(out["Wq"].cpu().numpy())
+    assert not q[:, lay.outlier_idx].any()
 
 
 def test_construct_rank_zero_only_packs_and_bad_arguments(aser):

@@ -866,6 +866,30 @@ def run_sweep(args, local_rank):
     print(json.dumps(line), flush=True)
 
 
+def run_profile(args, local_rank):
+    """Plain launches for a profiler (no graphs, no timing): `--profile step` runs whole steps,
+    `--profile <layer>` only that layer's activation pass and linear kernel."""
+    import torch
+    torch.cuda.set_device(local_rank)
+    m = Model(args.workload, torch.device("cuda", local_rank))
+    names = [nm for nm, _, _, _ in m.w["layers"]]
+    if args.profile != "step" and args.profile not in names:
+        raise SystemExit("--profile takes 'step' or one of %s" % names)
+    per = m.launches_per_step()
+    for i in range(args.warmup + args.steps):
+        if args.profile == "step":
+            m.step(i)
+        else:
+            li = names.index(args.profile)
+            S = m.sets[i % m.n_sets]
+            S["layers"][li](S["xs"][m.group_ids[li]])
+            per = m.aser.quant_act_ws_launches(m.M, m.w["layers"][li][1]) + 1
+    torch.cuda.synchronize()
+    m.check()
+    print(json.dumps(dict(profile=args.profile, workload=args.workload, launches_per_iteration=per,
+                          warmup=args.warmup, steps=args.steps)), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -876,6 +900,10 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle timing")
     ap.add_argument("--no-extra", dest="extra", action="store_false",
                     help="skip the other configurations' points")
+    ap.add_argument("--profile", default=None, metavar="WHAT",
+                    help="for a profiler: run W warm-up steps and K steps eagerly and exit, printing nothing "
+                         "but the launch count ('step' = whole steps, or a layer name = that layer's "
+                         "activation pass and linear kernel only)")
     ap.add_argument("--sweep", choices=["c5"], default=None,
                     help="time the 70B-class grid (two shapes x five token counts x five ranks) instead")
     args = ap.parse_args()
@@ -888,6 +916,10 @@ def main():
     if args.sweep:
         if rank == 0:
             run_sweep(args, local_rank)
+        return
+    if args.profile:
+        if rank == 0:
+            run_profile(args, local_rank)
         return
     run_ours(args, rank, world, local_rank)
 

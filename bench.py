@@ -419,11 +419,11 @@ class Model:
 
     def launches_per_step(self):
         """Kernels of this library launched by one step: per input group the activation pass
-        (two kernels per chunk of tokens above 32 tokens, one below) and one linear kernel per layer."""
+        (as many kernels as the library says it runs at that shape) and one linear kernel per layer."""
         n = 0
         for g, idx in self.members.items():
             K = self.w["layers"][idx[0]][1]
-            n += self.aser.quant_act_ws_launches(self.M, K) + len(idx)
+            n += self.aser.forward_act_launches(self.M, K, self.r * len(idx)) + len(idx)
         return n
 
     def check(self):
@@ -883,7 +883,7 @@ def run_profile(args, local_rank):
             li = names.index(args.profile)
             S = m.sets[i % m.n_sets]
             S["layers"][li](S["xs"][m.group_ids[li]])
-            per = m.aser.quant_act_ws_launches(m.M, m.w["layers"][li][1]) + 1
+            per = m.aser.forward_act_launches(m.M, m.w["layers"][li][1], m.r) + 1
     torch.cuda.synchronize()
     m.check()
     print(json.dumps(dict(profile=args.profile, workload=args.workload, launches_per_iteration=per,

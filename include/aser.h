@@ -233,9 +233,10 @@ int aser_check_status(void* workspace, void* stream);
  * Because the library knows that the quantization kernel is what precedes the linear kernel,
  * it launches the latter as a programmatic dependent: the linear kernel starts while the
  * quantization still runs, streams the weights (which that kernel does not write) and waits
- * for its completion before it reads Xq, a_scale or T.  With more than 32 tokens the
- * activation step is aser_quant_act_ws on the same workspace.  Results are those of the separate
- * calls.
+ * for its completion before it reads Xq, a_scale or T.  The activation step is aser_quant_act's
+ * kernels up to rank 128 and aser_quant_act_ws's (on the same workspace) above, whichever is
+ * faster at the shape; aser_forward_act_launches tells how many kernels that is.  Results are
+ * those of the separate calls.
  * X_f16 [M,K], s [K] or NULL, LA_f16 [r,K] / LB_f16 [N,r] (NULL when r == 0), Wk and w_scale as
  * for aser_linear_w4a8_lr.  Xq [M,K], a_scale [M], T_bf16 [M,r] (NULL when r == 0) are the
  * caller's intermediates (written), Y_f16 [M,N] the result.  Wk, w_scale and LB_f16 must not
@@ -243,6 +244,7 @@ int aser_check_status(void* workspace, void* stream);
  * Errors: as the two calls; every argument of both launches is checked first, so nothing is
  * enqueued when one is rejected.
  */
+int aser_forward_act_launches(int M, int K, int r);
 int aser_forward(const void* X_f16, const float* s, const void* LA_f16, const void* Wk,
                  const float* w_scale, const void* LB_f16, int M, int N, int K, int r,
                  int8_t* Xq, float* a_scale, void* T_bf16, void* Y_f16,

@@ -12,7 +12,7 @@ lib_path = os.path.join(_HERE, "libaser.so")
 EXPORTED_SYMBOLS = (
     "aser_pack_w4", "aser_repacked_bytes", "aser_repack_w4", "aser_unrepack_w4",
     "aser_quant_act", "aser_quant_act_bits", "aser_quant_act_ex", "aser_quant_act_ws",
-    "aser_quant_workspace_bytes", "aser_quant_act_ws_launches", "aser_linear_w4a8_lr_ld", "aser_forward_shared",
+    "aser_quant_workspace_bytes", "aser_quant_act_ws_launches", "aser_forward_act_launches", "aser_linear_w4a8_lr_ld", "aser_forward_shared",
     "aser_forward_shared_workspace_bytes", "aser_construct", "aser_construct_workspace_bytes", "aser_linear_w4a8_lr", "aser_linear_w4a8", "aser_linear_w4a8_lr_simt", "aser_linear_w4a8_lr_static",
     "aser_workspace_bytes", "aser_workspace_init", "aser_check_status", "aser_forward",
     "aser_forward_host",
@@ -36,6 +36,8 @@ lib.aser_quant_act_bits.argtypes = [_P, _P, _P, _I, _I, _I, _I, _P, _P, _P, _P]
 lib.aser_quant_act_ex.argtypes = [_P, _P, _P, _I, _I, _I, _I, _I, _P, _P, _P, _P]
 lib.aser_quant_workspace_bytes.argtypes = [_I, _I, _I]
 lib.aser_quant_workspace_bytes.restype = _Z
+lib.aser_forward_act_launches.argtypes = [_I, _I, _I]
+lib.aser_forward_act_launches.restype = _I
 lib.aser_quant_act_ws_launches.argtypes = [_I, _I]
 lib.aser_quant_act_ws_launches.restype = _I
 lib.aser_quant_act_ws.argtypes = [_P, _P, _P, _I, _I, _I, _I, _I, _P, _P, _P, _P, _Z, _P]
@@ -150,6 +152,10 @@ def quant_act(X: torch.Tensor, s: torch.Tensor | None, L_A: torch.Tensor | None,
     _chk(lib.aser_quant_act(_ptr(X), _ptr(s), _ptr(L_A) if r else None, M, K, r, _ptr(Xq),
                             _ptr(a_scale), _ptr(T) if r else None, _stream()), "aser_quant_act")
     return Xq, a_scale, T
+
+
+def forward_act_launches(M: int, K: int, r: int) -> int:
+    return int(lib.aser_forward_act_launches(M, K, r))
 
 
 def quant_act_ws_launches(M: int, K: int) -> int:
@@ -333,10 +339,14 @@ class AserLinear:
         self.ws = new_workspace(max_tokens, self.N, self.K, self.r, dev)
 
     def quant(self, X: torch.Tensor):
-        """The activation step alone, as aser_forward runs it (aser_quant_act_ws on the layer's
-        workspace)."""
+        """The activation step alone, with the kernels aser_forward runs at this shape."""
         M = X.shape[0]
         r = self.r
+        if forward_act_launches(M, self.K, r) == 1:
+            _chk(lib.aser_quant_act(_ptr(X), _ptr(self.s), _ptr(self.L_A) if r else None, M, self.K, r,
+                                    _ptr(self.Xq), _ptr(self.a_scale), _ptr(self.T) if r else None,
+                                    _stream()), "aser_quant_act")
+            return
         _chk(lib.aser_quant_act_ws(_ptr(X), _ptr(self.s), _ptr(self.L_A) if r else None, M, self.K, r,
                                    8, 0, _ptr(self.Xq), _ptr(self.a_scale), _ptr(self.T) if r else None,
                                    _ptr(self.ws), self.ws.numel(), _stream()), "aser_quant_act_ws")
@@ -409,6 +419,11 @@ class AserSharedInput:
     def quant(self, X: torch.Tensor):
         """The activation pass of the group alone (aser_quant_act_ws with the stacked L_A)."""
         M = X.shape[0]
+        if forward_act_launches(M, self.K, self.r_total) == 1 and self.r_total <= 256:
+            _chk(lib.aser_quant_act(_ptr(X), _ptr(self.s), _ptr(self.L_A), M, self.K, self.r_total,
+                                    _ptr(self.Xq), _ptr(self.a_scale), _ptr(self.T) if self.r_total else None,
+                                    _stream()), "aser_quant_act")
+            return
         _chk(lib.aser_quant_act_ws(_ptr(X), _ptr(self.s), _ptr(self.L_A), M, self.K, self.r_total, 8, 0,
                                    _ptr(self.Xq), _ptr(self.a_scale), _ptr(self.T) if self.r_total else None,
                                    _ptr(self.ws), self.ws.numel(), _stream()), "aser_quant_act_ws")

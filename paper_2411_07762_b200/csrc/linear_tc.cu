@@ -96,6 +96,7 @@ struct Params {
     int KB, TT, NT;        // 128-column blocks, token tiles, 128-row tiles
     int units;             // NT * TT * KB
     int tail_first;        // work order: 1 = both shared tiles first, 0 = range order
+    int tt_outer;          // tile numbering: 1 = token tile outer (consecutive tiles share the activations)
 };
 
 struct Work {
@@ -134,7 +135,9 @@ struct Cursor {
 };
 
 __device__ __forceinline__ void set_work(Work& w, const Params& p, int tile, int kb0, int kb1) {
-    w.tile = tile; w.nt = tile / p.TT; w.tt = tile - w.nt * p.TT; w.kb0 = kb0; w.kb1 = kb1;
+    w.tile = tile; w.kb0 = kb0; w.kb1 = kb1;
+    if (p.tt_outer) { w.tt = tile / p.NT; w.nt = tile - w.tt * p.NT; }
+    else { w.nt = tile / p.TT; w.tt = tile - w.nt * p.TT; }
     w.has_lr = (kb0 == 0) && p.r > 0;
     w.whole = (kb0 == 0) && (kb1 == p.KB);
 }
@@ -1001,6 +1004,12 @@ int launch_linear_tc(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
     // and range order (head part, whole tiles, tail part) is faster.  Measured: K = 14336
     // -12 %, K = 8192 -2..-6 %, K = 4096 +5 % if it were applied there.
     p.tail_first = (L.KB >= 64) ? 1 : 0;
+    // Tile numbering.  The CTAs work on about one grid's worth of consecutive tiles at a time, and
+    // what those tiles touch should stay in L2: with the weight tile outer that is ALL of Xq plus a
+    // few row tiles of the weights, with the token tile outer a few token tiles plus ALL packed
+    // weights.  Take the smaller set (4096 tokens into the 14336 -> 4096 projection: Xq is 59 MB and
+    // was read from DRAM ten times over with the weight tile outer).
+    p.tt_outer = ((long long)M * K > (long long)N * K / 2) ? 1 : 0;
 
     switch (L.BT) {
         case 16: return launch_bt<16, false>(mx, mlb, mt, p, grid, st, overlap_prev);

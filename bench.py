@@ -72,10 +72,16 @@ EXTRA_POINTS = ("c2_decode_m8", "c2_decode_m1", "c3_prefill_gate_up", "c3_prefil
                 "c5_decode_m16_8192", "c5_decode_m16_28672", "c5_prefill_m4096_8192",
                 "c5_prefill_m4096_28672")
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel under ncu, taken
-# with the kernel as it stands in this tree; the summaries with the commands are under profiles/
-# (<kernel>_<workload>.txt).  Workloads without a capture of the current kernel report null.
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel under ncu, taken with
+# the kernel as it stands in this tree; the summary with the command is
+# profiles/launches_c4_decoder_block_step.txt.  The workload's figure is the average over its seven
+# linear_tc launches (1070.1 MB in all); "<workload>/<layer>" is that layer's launch.  Workloads
+# without a capture of the current kernel report null.
 NCU_DRAM_BYTES_PER_LAUNCH = {
+    "c4_decoder_block": 1070.1e6 / 7,
+    "c4_decoder_block/q": 28.2e6, "c4_decoder_block/k": 20.3e6, "c4_decoder_block/v": 20.3e6,
+    "c4_decoder_block/o": 27.5e6, "c4_decoder_block/gate": 169.7e6, "c4_decoder_block/up": 169.0e6,
+    "c4_decoder_block/down": 635.1e6,
 }
 
 
@@ -522,7 +528,7 @@ def roofline_of(w, name, us_linear, peaks, lib_int8, li=None):
     secs = us_linear * 1e-6
     _, K0, N0, _ = layers[0]
     roof = dict(kernel=dominant_kernel(M, N0, K0), launches=len(layers), us_per_launch=us_linear / len(layers),
-                algorithmic_bytes=nbytes, ops=ops,
+                algorithmic_bytes=nbytes, ops=ops, algorithmic_bytes_per_launch=nbytes / len(layers),
                 traffic=NCU_DRAM_BYTES_PER_LAUNCH.get(name if li is None else "%s/%s" % (name, layers[0][0])))
     if w["bound"] == "hbm":
         achieved = nbytes / secs / 1e9
@@ -572,6 +578,7 @@ def measure(m, steps, peaks, lib_int8, barrier=None, max_over_ranks=lambda x: x,
             rows.append(dict(layer=nm, K=K, N=N, us_linear_lr=tl["median"] * 1e3,
                              us_linear_plain=tp["median"] * 1e3,
                              tops_linear=ops / (tl["median"] * 1e-3) / 1e12, frac=roof["frac"],
+                             traffic=roof["traffic"], algorithmic_bytes=roof["algorithmic_bytes"],
                              lowrank_overhead_linear=tl["median"] / tp["median"] - 1.0))
         out["layers"] = rows
         groups = []

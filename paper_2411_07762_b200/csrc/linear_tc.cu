@@ -703,7 +703,11 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     for (int j = 0; j < 16; ++j) {
                         const float lr = w.has_lr ? __uint_as_float(vf[j]) : 0.f;
                         const float y = fmaf((float)(int)vi[j], as[j] * ws16, lr);
-                        if (c0 + j < valid && n_ok) p.Y[row0 + (uint32_t)j * (uint32_t)p.N] = __float2half_rn(y);
+                        // streaming store: Y is written once and not read by this kernel, so it
+                        // should not displace the operands that other CTAs still re-read from L2
+                        if (c0 + j < valid && n_ok)
+                            __stcs(reinterpret_cast<unsigned short*>(p.Y + row0 + (uint32_t)j * (uint32_t)p.N),
+                                   __half_as_ushort(__float2half_rn(y)));
                     }
                     if (p.acc_debug) {
 #pragma unroll
@@ -809,7 +813,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                             if (c0 + j < valid && n_ok) {
                                 const float lr = (p.r > 0) ? __uint_as_float(lrw[j]) : 0.f;
                                 const float y = fmaf((float)sum[j], __ldg(p.a_scale + tok0 + c0 + j) * ws16, lr);
-                                p.Y[row0 + (uint32_t)j * (uint32_t)p.N] = __float2half_rn(y);
+                                __stcs(reinterpret_cast<unsigned short*>(p.Y + row0 + (uint32_t)j * (uint32_t)p.N),
+                                       __half_as_ushort(__float2half_rn(y)));
                                 if (p.acc_debug) p.acc_debug[row0 + (uint32_t)j * (uint32_t)p.N] = sum[j] >> 4;
                             }
                         }

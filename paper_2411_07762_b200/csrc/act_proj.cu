@@ -34,6 +34,8 @@ constexpr int kPMaxGroups = 4;              // 128-row groups of L_A: r <= 512
 constexpr int kProjPlanSms = 148;           // chunks and slices are planned for this many SMs (the
                                             // scratch size must not depend on the device)
 constexpr long long kPWaitLimitClocks = 400000000ll;   // about 0.2 s of SM clocks per wait
+constexpr int kPCacheUnits = 254;           // 8-column units with a divisor whose divisors are kept in shared memory
+constexpr int kPUncached = 255;             // tag of such a unit beyond the cache: its divisors are read from global memory
 
 __host__ __device__ constexpr int proj_stages(int groups) {
     const int per_stage = kPTileBytes * (1 + groups);
@@ -115,8 +117,11 @@ act_proj_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 25 * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 25 * 8 + 8);
     volatile int* never_flag = abort_flag + 1;                      // stays 0: waits of the wind-down
-    uint8_t* ones_sm = tail + 256;                                  // per 8 columns of the slice: all divisors are 1
+    // per 8 columns of the slice: 0 = all divisors are 1, else 1 + the unit's place in s_cache (or kPUncached)
+    uint8_t* unit_tag = tail + 256;
     float* amax_w = reinterpret_cast<float*>(tail + 256 + ((Kc / 8 + 15) & ~15));   // [8 warps][128 rows]
+    float* s_cache = amax_w + kPConsumerWarps * kPTok;              // [kPCacheUnits][8] divisors
+    int* n_cached = reinterpret_cast<int*>(tail + 25 * 8 + 16);
     const uint32_t tmem_cols = groups <= 1 ? 128u : groups == 2 ? 256u : 512u;
 
     if (warp == 0) {
@@ -133,6 +138,13 @@ act_proj_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             fence_proxy_async_smem();
             prefetch_tensormap(&map_x);
             if (r > 0) prefetch_tensormap(&map_la);
+            // The first round of the ring is requested before the other warps are ready: it needs
+            // only the barriers set up above.  X may come from the kernel before this one.
+            grid_dep_wait();
+            for (int i = 0; i < NS && i < nst; ++i) {
+                mbar_arrive_expect_tx(bar_full(i), (uint32_t)kPTileBytes);
+                tma_load_3d(sb + i * stage_bytes, &map_x, 0, m_first + row0, (k0 + i * kPCols) / kPCols, bar_full(i));
+            }
         }
         __syncwarp();
     } else if (warp == 1) {
@@ -142,15 +154,29 @@ act_proj_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
         }
     } else if (warp < kPWarpLa) {
+        // The smoothing divisors are 1 on all but the few outlier channels.  A unit that has one
+        // keeps its eight divisors in shared memory, so that the streaming loop below never waits
+        // for global memory.
+        if (tid == 64) *n_cached = 0;
+        named_bar_sync(1, kPConsumerWarps * 32);
         for (int g = tid - 64; g < Kc / 8; g += kPConsumerWarps * 32) {
-            bool one = true;
+            int tag = 0;
             if (s) {
                 const float4 a = __ldg(reinterpret_cast<const float4*>(s + k0 + g * 8));
                 const float4 b = __ldg(reinterpret_cast<const float4*>(s + k0 + g * 8) + 1);
-                one = a.x == 1.f && a.y == 1.f && a.z == 1.f && a.w == 1.f &&
-                      b.x == 1.f && b.y == 1.f && b.z == 1.f && b.w == 1.f;
+                const bool one = a.x == 1.f && a.y == 1.f && a.z == 1.f && a.w == 1.f &&
+                                 b.x == 1.f && b.y == 1.f && b.z == 1.f && b.w == 1.f;
+                if (!one) {
+                    const int at = atomicAdd(n_cached, 1);
+                    tag = kPUncached;
+                    if (at < kPCacheUnits) {
+                        tag = at + 1;
+                        *reinterpret_cast<float4*>(s_cache + at * 8) = a;
+                        *reinterpret_cast<float4*>(s_cache + at * 8 + 4) = b;
+                    }
+                }
             }
-            ones_sm[g] = one ? 1 : 0;
+            unit_tag[g] = (uint8_t)tag;
         }
     }
     tc_fence_before();
@@ -161,12 +187,11 @@ act_proj_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     if (warp == 0) {
         // ================= TMA producer =================
         if (lane == 0) {
-            grid_dep_wait();        // X may come from the kernel before; the scratch may still be read by it
             bool ok = true;
-            int issued = 0;
-            for (int i = 0; i < nst && ok; ++i) {
+            int issued = (NS < nst) ? NS : nst;
+            for (int i = issued; i < nst && ok; ++i) {
                 const int st = i % NS;
-                if (i >= NS) ok = pj_wait(bar_free(st), (uint32_t)(i / NS - 1) & 1u, abort_flag);
+                ok = pj_wait(bar_free(st), (uint32_t)(i / NS - 1) & 1u, abort_flag);
                 if (!ok) break;
                 const uint32_t dst = sb + st * stage_bytes;
                 const int kblk = (k0 + i * kPCols) / kPCols;
@@ -250,7 +275,8 @@ act_proj_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 addr[q] = base + (uint32_t)row * 128u + (uint32_t)((cw ^ (row & 7)) << 4);
                 v[q] = pj_lds128(addr[q]);
             }
-            if (ones_sm[i * 8 + cw]) {
+            const int tag = unit_tag[i * 8 + cw];
+            if (tag == 0) {
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
                     const __half2* h = reinterpret_cast<const __half2*>(&v[q]);
@@ -258,8 +284,9 @@ act_proj_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                     for (int e = 0; e < 4; ++e) hmax[q] = __hmax2(hmax[q], __habs2(h[e]));
                 }
             } else {
-                const float4* sp = reinterpret_cast<const float4*>(s + k0 + i * kPCols + cw * 8);
-                const float4 s0 = __ldg(sp), s1 = __ldg(sp + 1);
+                const float4* sp = (tag != kPUncached) ? reinterpret_cast<const float4*>(s_cache + (tag - 1) * 8)
+                                                       : reinterpret_cast<const float4*>(s + k0 + i * kPCols + cw * 8);
+                const float4 s0 = sp[0], s1 = sp[1];
                 const float sv[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
@@ -343,20 +370,55 @@ act_proj_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     }
 }
 
-// grid = ceil(rows of the chunk / kQRows), 256 threads; a CTA takes kQRows token rows: a smoothing
-// divisor is loaded (and tested against 1) once for all of them, several 16-byte loads per thread
-// are in flight, and the per-row scales are computed once per CTA (one warp per row) instead of by
-// every thread.  The kernel is bound by instruction issue, not by bytes: fp16 pairs are widened
-// with half2 operations, the products and the magic-constant rounding run on packed fp32 pairs.
-// Launched as a programmatic dependent of act_proj_kernel: the first loads of X (an input of the
-// whole step, not a product of that kernel) are issued before the dependency wait.
+// Eight codes of a row whose divisors are all 1: fp16 pairs widened by the conversion unit, then on
+// packed fp32 pairs su = x * (1 / sc) + 1.5 * 2^23 (one rounding: the low byte of su is the code),
+// -w = 1.5 * 2^23 - su (exact) and d = x * (1 / sc) - w, the distance of the product to its integer.
+// rne(x / sc) can differ from that integer only where the product is within 1e-4 of a tie (the
+// quotient and the product differ by less than 3.1e-5): such a group takes the exact division.
+__device__ __forceinline__ uint2 codes8_unit(const uint4& x, float sc, float rcp, float qmax) {
+    const float kMagic = 12582912.0f;
+    const float2 m2 = make_float2(kMagic, kMagic), neg1 = make_float2(-1.f, -1.f), r2 = make_float2(rcp, rcp);
+    const uint32_t xw[4] = {x.x, x.y, x.z, x.w};
+    float2 f[4];
+    uint32_t u[8];
+    float far = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        f[i] = __half22float2(*reinterpret_cast<const __half2*>(&xw[i]));
+        const float2 su = __ffma2_rn(f[i], r2, m2);
+        const float2 nw = __ffma2_rn(su, neg1, m2);
+        const float2 d = __ffma2_rn(f[i], r2, nw);
+        u[2 * i] = __float_as_uint(su.x);
+        u[2 * i + 1] = __float_as_uint(su.y);
+        far = fmaxf(far, fmaxf(fabsf(d.x), fabsf(d.y)));
+    }
+    if (far > 0.4999f)
+        return quant8_exact(f[0].x, f[0].y, f[1].x, f[1].y, f[2].x, f[2].y, f[3].x, f[3].y, sc, qmax);
+    const uint32_t a01 = __byte_perm(u[0], u[1], 0x0040), a23 = __byte_perm(u[2], u[3], 0x0040);
+    const uint32_t a45 = __byte_perm(u[4], u[5], 0x0040), a67 = __byte_perm(u[6], u[7], 0x0040);
+    return make_uint2(__byte_perm(a01, a23, 0x5410), __byte_perm(a45, a67, 0x5410));
+}
+
+// grid = ceil(rows of the chunk / kQRows), 256 threads; a CTA takes kQRows token rows, several
+// 16-byte loads per thread are in flight, and the per-row scales are computed once per CTA (one
+// warp per row).  The kernel is bound by instruction issue, not by bytes, so the common case is
+// kept free of per-column work: the CTA first lists the columns whose divisor is not 1 (the few
+// outlier channels); the main loop then treats every column as undivided, and the listed columns
+// are redone afterwards, one (row, column) per thread, with both IEEE divisions.  A smoothing
+// vector with more such columns than the list holds takes the general loop, which tests every
+// group of eight divisors.
+// Launched as a programmatic dependent of act_proj_kernel: the list and the first loads of X
+// (inputs of the whole step, not products of that kernel) are done before the dependency wait.
 constexpr int kQRows = 4;
+constexpr int kQList = 512;             // columns with a divisor the fix-up pass can take
 __global__ void __launch_bounds__(256, 4)
 act_quant_kernel(const __half* __restrict__ X, const float* __restrict__ s, int m_first, int Mc, int K,
                  int r, int KS, const float* amax_part, const float* t_part,
                  int8_t* __restrict__ Xq, float* __restrict__ a_scale, __nv_bfloat16* __restrict__ T,
                  int ldt, int lo_off, float qmax) {
     __shared__ float sc_sm[kQRows], rcp_sm[kQRows];
+    __shared__ int n_list;
+    __shared__ int list_col[kQList];
     grid_dep_launch();      // a dependent linear kernel may start streaming its weights
     const int row0 = blockIdx.x * kQRows;
     const int nrows = (Mc - row0 < kQRows) ? (Mc - row0) : kQRows;
@@ -373,6 +435,22 @@ act_quant_kernel(const __half* __restrict__ X, const float* __restrict__ s, int 
                                                 : make_uint4(0, 0, 0, 0);
     };
     load_x(c);
+    // ---- columns with a divisor (any order; entries past the capacity are only counted) ----
+    if (threadIdx.x == 0) n_list = 0;
+    __syncthreads();
+    if (s) {
+        for (int g = threadIdx.x; g < K / 4; g += 256) {
+            const float4 v = __ldg(reinterpret_cast<const float4*>(s) + g);
+            const float sv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                if (sv[e] != 1.f) {
+                    const int at = atomicAdd(&n_list, 1);
+                    if (at < kQList) list_col[at] = g * 4 + e;
+                }
+            }
+        }
+    }
     grid_dep_wait();        // the partial maxima and the partial T come from act_proj_kernel
     // ---- scales: warp w takes row w ----
     if (warp < nrows) {
@@ -390,6 +468,9 @@ act_quant_kernel(const __half* __restrict__ X, const float* __restrict__ s, int 
             rcp_sm[warp] = (sc > 0.f) ? __frcp_rn(sc) : 0.f;
             a_scale[m_first + row0 + warp] = sc;
         }
+    } else if (warp < kQRows && lane == 0) {
+        sc_sm[warp] = 0.f;
+        rcp_sm[warp] = 0.f;
     }
     // ---- T of these rows: the slices' partials summed in slice order ----
     for (int e = threadIdx.x; e < nrows * r; e += 256) {
@@ -401,70 +482,60 @@ act_quant_kernel(const __half* __restrict__ X, const float* __restrict__ s, int 
         store_t(T + (size_t)(m_first + row0 + rr) * ldt, j, t, lo_off);
     }
     __syncthreads();
-    // ---- codes ----
-    const float kMagic = 12582912.0f;       // 1.5 * 2^23: adding it rounds to the nearest integer, ties to even
-    const float2 m2 = make_float2(kMagic, kMagic), nm2 = make_float2(-kMagic, -kMagic);
-    const float2 neg1 = make_float2(-1.f, -1.f);
-    const float kWiden = __uint_as_float(0x77800000u);      // 2^112
-    const float2 widen2 = make_float2(kWiden, kWiden);
-    for (; c < chunks; c += 256) {
-        float4 s0 = make_float4(1.f, 1.f, 1.f, 1.f), s1 = s0;
-        if (s) {
-            s0 = __ldg(reinterpret_cast<const float4*>(s + c * 8));
-            s1 = __ldg(reinterpret_cast<const float4*>(s + c * 8) + 1);
+    const int listed = n_list;
+    float scr[kQRows], rc1[kQRows];
+#pragma unroll
+    for (int rr = 0; rr < kQRows; ++rr) {
+        scr[rr] = sc_sm[rr];
+        rc1[rr] = rcp_sm[rr];
+    }
+    if (listed <= kQList) {
+        // ---- codes, every column taken as undivided ----
+        for (; c < chunks; c += 256) {
+            uint2 q[kQRows];
+#pragma unroll
+            for (int rr = 0; rr < kQRows; ++rr) {
+                q[rr] = codes8_unit(x[rr], scr[rr], rc1[rr], qmax);
+                if (!(scr[rr] > 0.f)) q[rr] = make_uint2(0u, 0u);      // zero row, or a poisoned scale
+            }
+            load_x(c + 256);        // the next iteration's loads are in flight during the stores
+#pragma unroll
+            for (int rr = 0; rr < kQRows; ++rr)
+                if (rr < nrows) *reinterpret_cast<uint2*>(Xq + (size_t)(m_first + row0 + rr) * K + c * 8) = q[rr];
         }
-        const bool ones = s0.x == 1.f && s0.y == 1.f && s0.z == 1.f && s0.w == 1.f &&
-                          s1.x == 1.f && s1.y == 1.f && s1.z == 1.f && s1.w == 1.f;
+        // ---- the listed columns again, with their divisors ----
+        __syncthreads();            // orders the stores above before the single bytes below
+        for (int e = threadIdx.x; e < listed * kQRows; e += 256) {
+            const int rr = e & (kQRows - 1), col = list_col[e / kQRows];
+            if (rr >= nrows) continue;
+            const float sc = sc_sm[rr];
+            int code = 0;
+            if (sc > 0.f) {
+                const float xt = __fdiv_rn(__half2float(xbase[(size_t)rr * K + col]), __ldg(s + col));
+                code = rne_clamp(__fdiv_rn(xt, sc), -qmax, qmax);
+            }
+            Xq[(size_t)(m_first + row0 + rr) * K + col] = (int8_t)code;
+        }
+        return;
+    }
+    // ---- general loop: many columns have a divisor ----
+    for (; c < chunks; c += 256) {
+        const float4 s0 = __ldg(reinterpret_cast<const float4*>(s + c * 8));
+        const float4 s1 = __ldg(reinterpret_cast<const float4*>(s + c * 8) + 1);
+        const float sv[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
         uint2 q[kQRows];
 #pragma unroll
         for (int rr = 0; rr < kQRows; ++rr) {
-            // fp16 -> fp32 on the integer and multiply pipes: sign and the 15 value bits moved to
-            // their fp32 places, then times 2^112 (exact for normal and subnormal fp16 values)
-            const uint32_t xw[4] = {x[rr].x, x[rr].y, x[rr].z, x[rr].w};
-            float2 f[4];
+            const __half* h = reinterpret_cast<const __half*>(&x[rr]);
+            float f[8];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const uint32_t lo = ((xw[i] & 0x8000u) << 16) | ((xw[i] & 0x7fffu) << 13);
-                const uint32_t hi = (xw[i] & 0x80000000u) | ((xw[i] >> 3) & 0x0fffe000u);
-                f[i] = __fmul2_rn(make_float2(__uint_as_float(lo), __uint_as_float(hi)), widen2);
+            for (int e = 0; e < 8; ++e) {       // x~ = x / s, IEEE division, only where the divisor is not 1
+                f[e] = __half2float(h[e]);
+                if (sv[e] != 1.f) f[e] = __fdiv_rn(f[e], sv[e]);
             }
-            if (!ones) {        // x~ = x / s, IEEE division, only where the divisor is not 1
-                if (s0.x != 1.f) f[0].x = __fdiv_rn(f[0].x, s0.x);
-                if (s0.y != 1.f) f[0].y = __fdiv_rn(f[0].y, s0.y);
-                if (s0.z != 1.f) f[1].x = __fdiv_rn(f[1].x, s0.z);
-                if (s0.w != 1.f) f[1].y = __fdiv_rn(f[1].y, s0.w);
-                if (s1.x != 1.f) f[2].x = __fdiv_rn(f[2].x, s1.x);
-                if (s1.y != 1.f) f[2].y = __fdiv_rn(f[2].y, s1.y);
-                if (s1.z != 1.f) f[3].x = __fdiv_rn(f[3].x, s1.z);
-                if (s1.w != 1.f) f[3].y = __fdiv_rn(f[3].y, s1.w);
-            }
-            // rne(x~ / sc) == rne(x~ * (1 / sc)) unless the product is within 1e-4 of a tie (the
-            // two differ by less than 3.1e-5): then the whole group takes the exact division
-            const float scr = sc_sm[rr], rc1 = rcp_sm[rr];
-            const float2 r2 = make_float2(rc1, rc1);
-            uint32_t u[8];
-            float far = 0.f;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const float2 t = __fmul2_rn(f[i], r2);
-                const float2 su = __fadd2_rn(t, m2);
-                const float2 w = __fadd2_rn(su, nm2);
-                const float2 d = __ffma2_rn(w, neg1, t);
-                u[2 * i] = __float_as_uint(su.x);
-                u[2 * i + 1] = __float_as_uint(su.y);
-                far = fmaxf(far, fmaxf(fabsf(d.x), fabsf(d.y)));
-            }
-            if (scr > 0.f && !(far > 0.4999f)) {
-                const uint32_t a01 = __byte_perm(u[0], u[1], 0x0040), a23 = __byte_perm(u[2], u[3], 0x0040);
-                const uint32_t a45 = __byte_perm(u[4], u[5], 0x0040), a67 = __byte_perm(u[6], u[7], 0x0040);
-                q[rr] = make_uint2(__byte_perm(a01, a23, 0x5410), __byte_perm(a45, a67, 0x5410));
-            } else if (scr > 0.f) {
-                q[rr] = quant8_exact(f[0].x, f[0].y, f[1].x, f[1].y, f[2].x, f[2].y, f[3].x, f[3].y, scr, qmax);
-            } else {
-                q[rr] = make_uint2(0u, 0u);     // zero row, or a poisoned scale
-            }
+            q[rr] = (scr[rr] > 0.f) ? quant8_pairs(f, scr[rr], rc1[rr], qmax) : make_uint2(0u, 0u);
         }
-        load_x(c + 256);        // the next iteration's loads are in flight during the stores
+        load_x(c + 256);
 #pragma unroll
         for (int rr = 0; rr < kQRows; ++rr)
             if (rr < nrows) *reinterpret_cast<uint2*>(Xq + (size_t)(m_first + row0 + rr) * K + c * 8) = q[rr];
@@ -542,7 +613,7 @@ int launch_quant_act_ws(const __half* X, const float* s, const __half* LA, int M
     const int NS = proj_stages(groups);
     // the ring (at least 128 KB with a projection: it later stages the partial T) and the tail
     const size_t smem = (size_t)NS * kPTileBytes * (1 + groups) + 256 + ((Kc / 8 + 15) & ~15) +
-                        kPConsumerWarps * kPTok * sizeof(float) + 1024;
+                        kPConsumerWarps * kPTok * sizeof(float) + kPCacheUnits * 8 * sizeof(float) + 1024;
     static size_t configured[kMaxDevices] = {0};
     int dev = 0;
     {

@@ -131,12 +131,19 @@ bool act_shape_ok(int M, int K, int r) {
 }
 
 // Which activation kernels a forward pass runs.  The two-kernel path with scratch reads X once
-// whatever the rank and is the faster one above rank 128 (stacked down projections of a
-// shared-input group; a single layer of rank 129..256 would otherwise take two sweeps of the
-// cluster kernel).  Up to rank 128 the one-launch cluster kernel is as fast or faster (measured:
-// 4096 tokens x 4096 columns 40 against 36 us, 2048 x 14336 49 against 84 us, 4096 x 14336 138
-// against 158 us), and up to 32 tokens the few-token kernel serves every rank.
-bool forward_act_uses_scratch(int M, int r) { return M > 32 && r > 128; }
+// from HBM whatever the rank; it is the only one above rank 128 (stacked down projections of a
+// shared-input group) and the faster one from about a thousand tokens on while X fits one of its
+// chunks (measured at rank 128, two-kernel against cluster kernel: 1024 x 4096 21 against 27 us,
+// 4096 x 4096 34 against 42 us, 2048 x 8192 34 against 42 us, 1024 x 14336 34 against 66 us).
+// Longer inputs take several chunks, two launches each, and the one-launch cluster kernel is as
+// fast or faster there (4096 x 14336: 135 against 132 us; 8192 x 4096: 71 against 60 us), as it
+// is below a thousand tokens (256 x 4096: 23 against 17 us).  Up to 32 tokens the few-token
+// kernel serves every rank.
+bool forward_act_uses_scratch(int M, int K, int r) {
+    if (M <= 32) return false;
+    if (r > 128) return true;
+    return M >= 1024 && (long long)M * K <= (1ll << 25);
+}
 
 // The activation step of a forward pass (the scratch of the two-kernel path sits behind the
 // workspace's zeroed prefix, where the linear kernel later keeps its partial sums).
@@ -144,7 +151,7 @@ int quant_with_workspace(const void* X_f16, const float* s, const void* LA_f16, 
                          int act_bits, bool t_pair, int8_t* Xq, float* a_scale, void* T_bf16,
                          void* workspace, size_t workspace_bytes, void* stream) {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (!forward_act_uses_scratch(M, r))
+    if (!forward_act_uses_scratch(M, K, r))
         return launch_quant_act(static_cast<const __half*>(X_f16), s, static_cast<const __half*>(LA_f16), M, K, r,
                                 Xq, a_scale, static_cast<__nv_bfloat16*>(T_bf16), st, act_bits, t_pair);
     return launch_quant_act_ws(static_cast<const __half*>(X_f16), s, static_cast<const __half*>(LA_f16), M, K, r,
@@ -363,7 +370,7 @@ int aser_quant_act_ws(const void* X_f16, const float* s, const void* LA_f16, int
 
 int aser_forward_act_launches(int M, int K, int r) {
     if (!act_shape_ok(M, K, r) || M == 0) return 0;
-    return forward_act_uses_scratch(M, r) ? quant_act_ws_launches(M, K) : 1;
+    return forward_act_uses_scratch(M, K, r) ? quant_act_ws_launches(M, K) : 1;
 }
 
 int aser_linear_w4a8_lr_ld(const int8_t* Xq, const float* a_scale, const void* Wk,

@@ -331,6 +331,9 @@ constexpr int kXAtomBytes = kTTok * 128;    // 64 rows x 64 fp16
 constexpr int kXStageBytes = 2 * kXAtomBytes;
 constexpr int kOutTileBytes = kTTok * kTCols;   // 64 rows x 128 int8
 constexpr long long kQaWaitLimitClocks = 400000000ll;   // about 0.2 s of SM clocks per wait
+constexpr long long kTL2Budget = 72ll << 20;    // bytes of X the second sweep can expect to find in L2
+constexpr int kTCacheUnits = 62;            // 16-column units with a divisor whose divisors are kept in shared memory
+constexpr int kTUncached = 255;             // tag of such a unit beyond the cache: its divisors are read from global memory
 
 // Ring depth: as many stages (activation tile + L_A tile) as fit beside the exchange buffers.
 // A stage takes about 3 k cycles to go round (HBM latency plus the hand-overs between TMA,
@@ -338,7 +341,7 @@ constexpr long long kQaWaitLimitClocks = 400000000ll;   // about 0.2 s of SM clo
 __host__ __device__ constexpr int tma_stages(int r, int CK) {
     const int per_stage = kXStageBytes + 256 * r;
     const int exch = (CK > 1) ? 2 * kTTok * r * 4 : 0;
-    const int fixed = (exch > 16 * 1024 ? exch : 16 * 1024) + 12 * 1024;
+    const int fixed = (exch > 16 * 1024 ? exch : 16 * 1024) + 16 * 1024;
     int ns = (227 * 1024 - fixed) / per_stage;
     if (ns * per_stage < kTOut * kOutTileBytes + kXStageBytes * ns) {      // region B must hold the output tiles
         ns = (227 * 1024 - fixed - kTOut * kOutTileBytes) / kXStageBytes;
@@ -348,7 +351,7 @@ __host__ __device__ constexpr int tma_stages(int r, int CK) {
 
 struct TmaSmem {
     int x_ring, region_b, la_atom_bytes, la_stage_bytes, t_slots, t_stage, ones, amax_cg, amax_stage,
-        amax_slots, bars, tmem_slot, abort_flag, total;
+        amax_slots, s_cache, bars, tmem_slot, abort_flag, n_cached, total;
 };
 // Offsets from the 1 KiB-aligned base.  Region B holds the L_A ring in sweep 1 and the output
 // tiles in sweep 2.  t_slots receives the partial T of the tokens this CTA owns from every CTA
@@ -374,13 +377,15 @@ __host__ __device__ inline TmaSmem tma_smem(int Kc, int r, int CK) {
         off += b;
     }
     L.t_stage = off;    off += (CK > 1) ? kTTok * r * 4 : 0;   // this CTA's partial T, [token][r]
-    L.ones = off;       off += (Kc / 16 + 15) / 16 * 16;       // per 16 columns: all divisors are 1
+    L.ones = off;       off += (Kc / 16 + 15) / 16 * 16;       // per 16 columns: 0 = all divisors are 1, else a tag
     L.amax_cg = off;    off += 16 * kTTok * 4;                 // row maxima per (stage parity, 16-column group)
     L.amax_stage = off; off += kTTok * 4;                      // row maxima of this CTA's slice
     L.amax_slots = off; off += 16 * kTTok * 4;                 // row maxima copied in by each CTA
+    L.s_cache = off;    off += kTCacheUnits * 16 * 4;          // the divisors of the tagged units
     L.bars = off;       off += (4 * kTMaxStages + 2 * kTOut + 3) * 8;
     L.tmem_slot = off;  off += 8;
-    L.abort_flag = off; off += 8;
+    L.abort_flag = off; off += 4;
+    L.n_cached = off;   off += 4;
     L.total = off + 1024;                                      // slack for the alignment
     return L;
 }
@@ -517,6 +522,8 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L.abort_flag);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L.tmem_slot);
     uint8_t* ones_sm = smem + L.ones;
+    float* s_cache = reinterpret_cast<float*>(smem + L.s_cache);
+    int* n_cached = reinterpret_cast<int*>(smem + L.n_cached);
     float* amax_cg = reinterpret_cast<float*>(smem + L.amax_cg);
     float* amax_stage = reinterpret_cast<float*>(smem + L.amax_stage);
     float* amax_slots = reinterpret_cast<float*>(smem + L.amax_slots);
@@ -609,18 +616,33 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         }
         if (lane == 0) prefetch_tensormap(&map_q);
     } else {
-        // per 16 columns of the slice: are all smoothing divisors 1?
+        // Per 16 columns of the slice: are all smoothing divisors 1?  They are on all but the few
+        // outlier channels; a unit that has a divisor keeps its sixteen in shared memory, so that
+        // the two sweeps never wait for global memory.
+        if (tid == 0) *n_cached = 0;
+        named_bar_sync(1, kTConsumers);
         for (int g = tid; g < Kc / 16; g += kTConsumers) {
-            bool one = true;
+            int tag = 0;
             if (s) {
                 const float4* sp = reinterpret_cast<const float4*>(s + k0 + g * 16);
+                float4 v[4];
+                bool one = true;
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    const float4 v = __ldg(sp + i);
-                    one = one && v.x == 1.f && v.y == 1.f && v.z == 1.f && v.w == 1.f;
+                    v[i] = __ldg(sp + i);
+                    one = one && v[i].x == 1.f && v[i].y == 1.f && v[i].z == 1.f && v[i].w == 1.f;
+                }
+                if (!one) {
+                    const int at = atomicAdd(n_cached, 1);
+                    tag = kTUncached;
+                    if (at < kTCacheUnits) {
+                        tag = at + 1;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) reinterpret_cast<float4*>(s_cache + at * 16)[i] = v[i];
+                    }
                 }
             }
-            ones_sm[g] = one ? 1 : 0;
+            ones_sm[g] = (uint8_t)tag;
         }
     }
     tc_fence_before();
@@ -714,7 +736,8 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             const uint32_t a0 = sb + L.x_ring + st * kXStageBytes + x_off, a1 = a0 ^ 16u;
             const uint4 v0 = lds128(a0), v1 = lds128(a1);
             const uint4 w0 = lds128(a0 + kRow32), w1 = lds128(a1 + kRow32);
-            if (ones_sm[i * 8 + cg]) {
+            const int tag1 = ones_sm[i * 8 + cg];
+            if (tag1 == 0) {
                 const __half2* h0 = reinterpret_cast<const __half2*>(&v0);
                 const __half2* h1 = reinterpret_cast<const __half2*>(&v1);
                 const __half2* g0 = reinterpret_cast<const __half2*>(&w0);
@@ -727,8 +750,9 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                     hamax1 = __hmax2(hamax1, __habs2(g1[e]));
                 }
             } else {
-                const float4* sp = reinterpret_cast<const float4*>(s + k0 + i * kTCols + cg * 16);
-                const float4 s0 = __ldg(sp), s1 = __ldg(sp + 1), s2 = __ldg(sp + 2), s3 = __ldg(sp + 3);
+                const float4* sp = (tag1 != kTUncached) ? reinterpret_cast<const float4*>(s_cache + (tag1 - 1) * 16)
+                                                        : reinterpret_cast<const float4*>(s + k0 + i * kTCols + cg * 16);
+                const float4 s0 = sp[0], s1 = sp[1], s2 = sp[2], s3 = sp[3];
                 float v[8];
                 div8(v0, s0, s1, v);
 #pragma unroll
@@ -843,14 +867,16 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             const uint4 w0 = lds128(a0 + kRow32), w1 = lds128(a1 + kRow32);
             // x~ of the two units (all loaded words are consumed here) ...
             float f0[8], f1[8], g0[8], g1[8];
-            if (ones_sm[jj * 8 + cg]) {
+            const int tag2 = ones_sm[jj * 8 + cg];
+            if (tag2 == 0) {
                 cvt8(v0, f0);
                 cvt8(v1, f1);
                 cvt8(w0, g0);
                 cvt8(w1, g1);
             } else {
-                const float4* sp = reinterpret_cast<const float4*>(s + k0 + jj * kTCols + cg * 16);
-                const float4 s0 = __ldg(sp), s1 = __ldg(sp + 1), s2 = __ldg(sp + 2), s3 = __ldg(sp + 3);
+                const float4* sp = (tag2 != kTUncached) ? reinterpret_cast<const float4*>(s_cache + (tag2 - 1) * 16)
+                                                        : reinterpret_cast<const float4*>(s + k0 + jj * kTCols + cg * 16);
+                const float4 s0 = sp[0], s1 = sp[1], s2 = sp[2], s3 = sp[3];
                 div8(v0, s0, s1, f0);
                 div8(v1, s2, s3, f1);
                 div8(w0, s0, s1, g0);
@@ -965,7 +991,10 @@ int tma_active_clusters(int ck, size_t smem) {
 
 // Cluster size for the TMA kernel: a power of two (the CTAs split the 64 tokens' T) that
 // divides the K / 128 stages.  Larger clusters shorten a CTA's two sweeps but fewer of
-// them are resident at once; the estimate is waves x (fixed cost + stages), in stage units.
+// them are resident at once; the estimate is waves x (fixed cost + stages of both sweeps), in
+// stage units.  The second sweep finds its slice in L2 only if the slices of all resident
+// clusters fit there together; otherwise it streams from HBM again, behind the first sweep's
+// traffic, and its stages count double.
 int pick_tma_cluster(int M, int K, int r, int max_ck) {
     const int tiles = (M + kTTok - 1) / kTTok, blocks = K / kTCols;      // 128-column stages
     int best = 0;
@@ -977,7 +1006,9 @@ int pick_tma_cluster(int M, int K, int r, int max_ck) {
         const int active = tma_active_clusters(ck, smem);
         if (active < 1) continue;
         const long long waves = (tiles + active - 1) / active;
-        const long long cost = waves * (6 + blocks / ck);
+        const long long resident = (tiles < active) ? tiles : active;
+        const bool in_l2 = resident * kTTok * (long long)K * 2 <= kTL2Budget;
+        const long long cost = waves * (6 + (blocks / ck) * (in_l2 ? 2 : 3));
         if (best == 0 || cost < best_cost) { best = ck; best_cost = cost; }
     }
     return best;

@@ -74,15 +74,10 @@ EXTRA_POINTS = ("c2_decode_m8", "c2_decode_m1", "c3_prefill_gate_up", "c3_prefil
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel under ncu, taken with
 # the kernel as it stands in this tree; the summary with the command is
-# profiles/launches_c4_decoder_block_step.txt.  The workload's figure is the average over its seven
-# linear_tc launches (1070.1 MB in all); "<workload>/<layer>" is that layer's launch.  Workloads
+# profiles/launches_c4_decoder_block_step.txt.  The workload's figure is the average over its
+# linear_tc launches; "<workload>/<layers>" is the launch of that layer or fused group.  Workloads
 # without a capture of the current kernel report null.
-NCU_DRAM_BYTES_PER_LAUNCH = {
-    "c4_decoder_block": 1070.1e6 / 7,
-    "c4_decoder_block/q": 28.2e6, "c4_decoder_block/k": 20.3e6, "c4_decoder_block/v": 20.3e6,
-    "c4_decoder_block/o": 27.5e6, "c4_decoder_block/gate": 169.7e6, "c4_decoder_block/up": 169.0e6,
-    "c4_decoder_block/down": 635.1e6,
-}
+NCU_DRAM_BYTES_PER_LAUNCH = {}
 
 
 def dominant_kernel(M, N, K):
@@ -324,8 +319,10 @@ class Model:
     """Device-resident operands of a workload: one AserLinear per layer and one activation
     tensor per input group, in as many distinct operand sets as it takes for a step never to
     find its operands in L2 (one set where a single step already exceeds twice the L2 size).
-    Layers of one input group run through aser_forward_shared (one activation pass for the
-    group), a layer alone in its group through aser_forward."""
+    Layers of one input group run through aser_forward_shared_cat (one activation pass and one
+    linear launch over the group's concatenated output channels; aser_forward_shared, one linear
+    launch per layer, where the group cannot be stored fused), a layer alone in its group through
+    aser_forward."""
 
     def __init__(self, name, device):
         import torch
@@ -339,6 +336,7 @@ class Model:
         t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(device)
         self.group_ids = [g for _, _, _, g in w["layers"]]
         self.members = {}                       # input group -> layer indices
+        self.fused = {}                         # input group -> stored as one fused projection
         for li, g in enumerate(self.group_ids):
             self.members.setdefault(g, []).append(li)
         base_layers, base_x, group_s = [], {}, {}
@@ -376,7 +374,16 @@ class Model:
         shared, shared_plain = {}, {}
         for g, idx in self.members.items():
             if len(idx) > 1:
-                shared[g] = aser.AserSharedInput([layers[i] for i in idx], self.M)
+                # One linear launch over the concatenated output channels pays where a layer alone
+                # has too few 128 x 128 tiles to fill the SMs evenly (key/value: 256 tiles on 148
+                # SMs); with thousands of tiles per layer (gate/up) it measured 6 % slower than
+                # one launch per layer, so those groups keep their layers apart.
+                tiles = [(self.w["layers"][i][2] // 128) * ((self.M + 127) // 128) for i in idx]
+                fused = (len(idx) <= 4 and all(self.w["layers"][i][2] % 128 == 0 for i in idx)
+                         and min(tiles) < 4 * 148)
+                Group = aser.AserSharedInputCat if fused else aser.AserSharedInput
+                self.fused[g] = fused
+                shared[g] = Group([layers[i] for i in idx], self.M)
                 if self.r:
                     plain = []
                     for i in idx:
@@ -384,7 +391,7 @@ class Model:
                         P.__dict__.update(layers[i].__dict__)
                         P.r, P.L_A, P.L_B = 0, None, None
                         plain.append(P)
-                    shared_plain[g] = aser.AserSharedInput(plain, self.M)
+                    shared_plain[g] = Group(plain, self.M)
                 else:
                     shared_plain[g] = shared[g]
         return dict(layers=layers, xs=xs, shared=shared, shared_plain=shared_plain)
@@ -399,10 +406,28 @@ class Model:
                 S["layers"][idx[0]](S["xs"][g], lowrank)
 
     def linear_only(self, i, li=None, lowrank=True):
+        """The linear launches of a step (a fused group is one launch), or layer `li` on its own."""
         S = self.sets[i % self.n_sets]
-        for j, L in enumerate(S["layers"]):
-            if li is None or li == j:
-                L.linear(self.M, lowrank)
+        if li is not None:
+            S["layers"][li].linear(self.M, lowrank)
+            return
+        for g, idx in self.members.items():
+            if self.fused.get(g):
+                (S["shared"] if lowrank else S["shared_plain"])[g].linear(self.M)
+            else:
+                for j in idx:
+                    S["layers"][j].linear(self.M, lowrank)
+
+    def group_linear(self, i, g, lowrank=True):
+        S = self.sets[i % self.n_sets]
+        if self.fused.get(g):
+            (S["shared"] if lowrank else S["shared_plain"])[g].linear(self.M)
+        else:
+            for j in self.members[g]:
+                S["layers"][j].linear(self.M, lowrank)
+
+    def linear_launches(self):
+        return sum(1 if self.fused.get(g) else len(idx) for g, idx in self.members.items())
 
     def quant_only(self, i, g_only=None):
         """The activation passes of a step (one per input group), or of one group."""
@@ -425,11 +450,12 @@ class Model:
 
     def launches_per_step(self):
         """Kernels of this library launched by one step: per input group the activation pass
-        (as many kernels as the library says it runs at that shape) and one linear kernel per layer."""
+        (as many kernels as the library says it runs at that shape) and one linear kernel per layer
+        (one per group where the group is stored fused)."""
         n = 0
         for g, idx in self.members.items():
             K = self.w["layers"][idx[0]][1]
-            n += self.aser.forward_act_launches(self.M, K, self.r * len(idx)) + len(idx)
+            n += self.aser.forward_act_launches(self.M, K, self.r * len(idx)) + (1 if self.fused.get(g) else len(idx))
         return n
 
     def check(self):
@@ -514,7 +540,7 @@ def library_int8_gemm_tops(torch, dev, n=8192, reps=10):
         return "unavailable: %s" % type(exc).__name__
 
 
-def roofline_of(w, name, us_linear, peaks, lib_int8, li=None):
+def roofline_of(w, name, us_linear, peaks, lib_int8, li=None, launches=None, layer_idx=None):
     """Roofline object of the integer-product kernel for the whole workload (li None: all its
     launches together) or one layer.  HBM-bound few-token shapes: algorithmic bytes over the
     measured copy bandwidth.  Tensor-bound shapes: 2 M N K over the int8 peak, taken as twice the
@@ -522,14 +548,18 @@ def roofline_of(w, name, us_linear, peaks, lib_int8, li=None):
     of at least 20 ms, so the sustained figure is the denominator, and the burst figure, the
     vendor library's measured int8 GEMM and the data-sheet value are printed beside it."""
     layers = w["layers"] if li is None else [w["layers"][li]]
+    if layer_idx is not None:
+        layers = [w["layers"][i] for i in layer_idx]
+    n_launch = launches if launches is not None else len(layers)
     M, r = w["M"], w["r"]
     ops = sum(2.0 * M * N * K for _, K, N, _ in layers)
     nbytes = sum(algorithmic_bytes_linear(M, N, K, r) for _, K, N, _ in layers)
     secs = us_linear * 1e-6
     _, K0, N0, _ = layers[0]
-    roof = dict(kernel=dominant_kernel(M, N0, K0), launches=len(layers), us_per_launch=us_linear / len(layers),
-                algorithmic_bytes=nbytes, ops=ops, algorithmic_bytes_per_launch=nbytes / len(layers),
-                traffic=NCU_DRAM_BYTES_PER_LAUNCH.get(name if li is None else "%s/%s" % (name, layers[0][0])))
+    key = name if (li is None and layer_idx is None) else "%s/%s" % (name, "+".join(l[0] for l in layers))
+    roof = dict(kernel=dominant_kernel(M, N0, K0), launches=n_launch, us_per_launch=us_linear / n_launch,
+                algorithmic_bytes=nbytes, ops=ops, algorithmic_bytes_per_launch=nbytes / n_launch,
+                traffic=NCU_DRAM_BYTES_PER_LAUNCH.get(key))
     if w["bound"] == "hbm":
         achieved = nbytes / secs / 1e9
         roof.update(bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s",
@@ -564,7 +594,7 @@ def measure(m, steps, peaks, lib_int8, barrier=None, max_over_ranks=lambda x: x,
                spread=dict(step=t_step["spread"], linear_lr=t_lin["spread"], quant_act=t_act["spread"]),
                overhead=dict(linear=t_lin["median"] / t_lin_plain["median"] - 1.0,
                              step=t_step["median"] / t_step_plain["median"] - 1.0),
-               roofline=roofline_of(w, m.name, t_lin["median"] * 1e3, peaks, lib_int8))
+               roofline=roofline_of(w, m.name, t_lin["median"] * 1e3, peaks, lib_int8, launches=m.linear_launches()))
     act_bytes = sum(algorithmic_bytes_act(w["M"], w["layers"][idx[0]][1], w["r"] * len(idx))
                     for idx in m.members.values())
     out["quant_act_gbs"] = act_bytes / (t_act["median"] * 1e-3) / 1e9
@@ -589,7 +619,15 @@ def measure(m, steps, peaks, lib_int8, barrier=None, max_over_ranks=lambda x: x,
             ts = m.time_region(lambda i: m.group_step(i, g), calls, label=names + " step")
             tsp = m.time_region(lambda i: m.group_step(i, g, False), calls, label=names + " step_plain") if m.r else ts
             act_b = algorithmic_bytes_act(w["M"], K, w["r"] * len(idx))
+            tgl = m.time_region(lambda i: m.group_linear(i, g), calls, label=names + " linear")
+            tglp = m.time_region(lambda i: m.group_linear(i, g, False), calls, label=names + " linear_plain") if m.r else tgl
+            groof = roofline_of(w, m.name, tgl["median"] * 1e3, peaks, lib_int8, layer_idx=idx,
+                                launches=1 if m.fused.get(g) else len(idx))
             groups.append(dict(layers=names, K=K, stacked_rank=w["r"] * len(idx),
+                               fused_linear=bool(m.fused.get(g)), linear_launches=groof["launches"],
+                               us_linear_lr=tgl["median"] * 1e3, us_linear_plain=tglp["median"] * 1e3,
+                               linear_frac=groof["frac"], linear_traffic=groof["traffic"],
+                               linear_algorithmic_bytes=groof["algorithmic_bytes"],
                                us_quant_act=ta["median"] * 1e3, us_step=ts["median"] * 1e3,
                                us_step_plain=tsp["median"] * 1e3,
                                lowrank_overhead_step=ts["median"] / tsp["median"] - 1.0,

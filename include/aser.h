@@ -270,6 +270,33 @@ int aser_forward_shared(const void* X_f16, const float* s, const void* LA_stacke
                         void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * aser_linear_w4a8_lr_cat / aser_forward_shared_cat -- a shared-input group whose layers are STORED
+ * one after the other along N, as a fused q/k/v or gate/up projection is: Wk_cat is the layers'
+ * blocked weights concatenated (aser_pack_w4 of each layer, layer l's bytes behind layer l-1's;
+ * every N[l] a positive multiple of 128, at most four layers), w_scale_cat [sum N],
+ * LB_cat_f16 [sum N, r] (all layers of one rank r, r * n_layers <= 512), Y_cat_f16 [M, sum N]
+ * (layer l's output is the column range of its rows).  One linear launch then serves the whole
+ * group: a weight tile multiplies the columns [l r, (l + 1) r) of T_bf16 [M, r * n_layers] of the
+ * layer l it lies in.  The arithmetic per output element is that of aser_linear_w4a8_lr on the
+ * layer alone (Sec. 4.1 Eq. 7 with the stacked operands of Algorithm 1's independent layers), so
+ * the results are bit-identical to it.  aser_forward_shared_cat runs the activation pass first
+ * (as aser_forward_shared).  workspace: aser_forward_shared_cat_workspace_bytes(...) bytes,
+ * zeroed once with aser_workspace_init; for the linear step alone
+ * aser_workspace_bytes(M, sum N, K, r) is enough.  Errors: every argument is checked before
+ * anything is enqueued.
+ */
+int aser_linear_w4a8_lr_cat(const int8_t* Xq, const float* a_scale, const void* Wk_cat,
+                            const float* w_scale_cat, const void* T_bf16, const void* LB_cat_f16,
+                            int n_layers, const int* N, int r, int M, int K, void* Y_cat_f16,
+                            void* workspace, size_t workspace_bytes, void* stream);
+size_t aser_forward_shared_cat_workspace_bytes(int n_layers, const int* N, int r, int M, int K);
+int aser_forward_shared_cat(const void* X_f16, const float* s, const void* LA_stacked_f16, int n_layers,
+                            const void* Wk_cat, const float* w_scale_cat, const void* LB_cat_f16,
+                            const int* N, int r, int M, int K, int8_t* Xq, float* a_scale,
+                            void* T_bf16, void* Y_cat_f16, void* workspace, size_t workspace_bytes,
+                            void* stream);
+
+/*
  * aser_forward_host -- one whole forward pass from HOST buffers: copies X (fp16 [M,K],
  * ideally pinned) to the device staging buffer X_dev, runs aser_forward, and copies Y back to Y_host,
  * all enqueued on `stream`; returns without synchronising.  Device-side operands and

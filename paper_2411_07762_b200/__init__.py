@@ -14,7 +14,7 @@ _BINDING_NAMES = (
     "linear_w4a8_lr", "linear_w4a8", "linear_w4a8_lr_simt", "linear_w4a8_lr_static",
     "workspace_bytes", "new_workspace", "check_status", "forward_host",
     "AserLinear", "EXPORTED_SYMBOLS", "pad_rank", "pair_up_projection", "quant_act_ws", "quant_workspace_bytes", "quant_act_ws_launches", "forward_act_launches",
-    "linear_w4a8_lr_ld", "AserSharedInput", "construct",
+    "linear_w4a8_lr_ld", "AserSharedInput", "AserSharedInputCat", "construct",
 )
 
 

@@ -13,6 +13,7 @@ EXPORTED_SYMBOLS = (
     "aser_pack_w4", "aser_repacked_bytes", "aser_repack_w4", "aser_unrepack_w4",
     "aser_quant_act", "aser_quant_act_bits", "aser_quant_act_ex", "aser_quant_act_ws",
     "aser_quant_workspace_bytes", "aser_quant_act_ws_launches", "aser_forward_act_launches", "aser_linear_w4a8_lr_ld", "aser_forward_shared",
+    "aser_linear_w4a8_lr_cat", "aser_forward_shared_cat_workspace_bytes", "aser_forward_shared_cat",
     "aser_forward_shared_workspace_bytes", "aser_construct", "aser_construct_workspace_bytes", "aser_linear_w4a8_lr", "aser_linear_w4a8", "aser_linear_w4a8_lr_simt", "aser_linear_w4a8_lr_static",
     "aser_workspace_bytes", "aser_workspace_init", "aser_check_status", "aser_forward",
     "aser_forward_host",
@@ -45,6 +46,10 @@ lib.aser_linear_w4a8_lr_ld.argtypes = [_P, _P, _P, _P, _P, _I, _P, _I, _I, _I, _
 lib.aser_forward_shared_workspace_bytes.argtypes = [_I, _P, _P, _I, _I]
 lib.aser_forward_shared_workspace_bytes.restype = _Z
 lib.aser_forward_shared.argtypes = [_P, _P, _P, _I, _P, _P, _P, _P, _P, _I, _I, _P, _P, _P, _P, _P, _Z, _P]
+lib.aser_linear_w4a8_lr_cat.argtypes = [_P, _P, _P, _P, _P, _P, _I, _P, _I, _I, _I, _P, _P, _Z, _P]
+lib.aser_forward_shared_cat_workspace_bytes.argtypes = [_I, _P, _I, _I, _I]
+lib.aser_forward_shared_cat_workspace_bytes.restype = _Z
+lib.aser_forward_shared_cat.argtypes = [_P, _P, _P, _I, _P, _P, _P, _P, _I, _I, _I, _P, _P, _P, _P, _P, _Z, _P]
 lib.aser_linear_w4a8_lr.argtypes = [_P, _P, _P, _P, _P, _P, _I, _I, _I, _I, _P, _P, _P, _Z, _P]
 lib.aser_linear_w4a8.argtypes = [_P, _P, _P, _P, _I, _I, _I, _P, _P, _P, _Z, _P]
 lib.aser_linear_w4a8_lr_simt.argtypes = [_P, _P, _P, _P, _P, _P, _I, _I, _I, _I, _P, _P, _P]
@@ -438,6 +443,59 @@ class AserSharedInput:
                                      _ptr(self.a_scale), _ptr(self.T) if self.r_total else None, self._Y,
                                      _ptr(self.ws), self.ws.numel(), _stream()), "aser_forward_shared")
         return [y[:M] for y in self.Y]
+
+
+
+class AserSharedInputCat(AserSharedInput):
+    """A shared-input group stored as one fused projection: the layers' packed weights, scales and
+    up projections are concatenated along N (copies are made here) and the outputs are column
+    ranges of one [M, sum N] buffer, so that a single linear launch serves the group
+    (aser_forward_shared_cat).  Needs every N a multiple of 128 and one rank for all layers."""
+
+    def __init__(self, layers, max_tokens: int):
+        super().__init__(layers, max_tokens)
+        if len(set(self.r)) != 1 or any(n % 128 for n in self.N) or self.n > 4:
+            raise ValueError("a concatenated group needs one rank, N multiples of 128 and at most four layers")
+        dev = self.layers[0].Wk.device
+        self.r1 = self.r[0]
+        self.N_total = sum(self.N)
+        self.Wk_cat = torch.cat([L.Wk.reshape(-1) for L in self.layers]).contiguous()
+        self.w_scale_cat = torch.cat([L.w_scale for L in self.layers]).contiguous()
+        self.L_B_cat = torch.cat([L.L_B for L in self.layers], dim=0).contiguous() if self.r1 else None
+        self.Y_cat = torch.empty((max_tokens, self.N_total), dtype=torch.float16, device=dev)
+        nbytes = int(lib.aser_forward_shared_cat_workspace_bytes(self.n, self._N, self.r1, max_tokens, self.K))
+        if nbytes == 0:
+            raise ValueError("unsupported shapes for a concatenated shared-input group")
+        if nbytes > self.ws.numel():
+            self.ws = torch.empty((nbytes,), dtype=torch.uint8, device=dev)
+            _chk(lib.aser_workspace_init(_ptr(self.ws), nbytes, _stream()), "aser_workspace_init")
+
+    def _views(self, M: int):
+        out, col = [], 0
+        for n in self.N:
+            out.append(self.Y_cat[:M, col:col + n])
+            col += n
+        return out
+
+    def linear(self, M: int):
+        """The linear step alone on the codes and T of the last activation pass."""
+        _chk(lib.aser_linear_w4a8_lr_cat(_ptr(self.Xq), _ptr(self.a_scale), _ptr(self.Wk_cat),
+                                         _ptr(self.w_scale_cat), _ptr(self.T) if self.r1 else None,
+                                         _ptr(self.L_B_cat) if self.r1 else None, self.n, self._N, self.r1,
+                                         M, self.K, _ptr(self.Y_cat), _ptr(self.ws), self.ws.numel(),
+                                         _stream()), "aser_linear_w4a8_lr_cat")
+        return self._views(M)
+
+    def __call__(self, X: torch.Tensor):
+        """Returns the layers' outputs as column ranges of the fused output [M, sum N]."""
+        M = X.shape[0]
+        assert M == self.max_tokens, "the fused output buffer is laid out for max_tokens rows"
+        _chk(lib.aser_forward_shared_cat(_ptr(X), _ptr(self.s), _ptr(self.L_A), self.n, _ptr(self.Wk_cat),
+                                         _ptr(self.w_scale_cat), _ptr(self.L_B_cat) if self.r1 else None,
+                                         self._N, self.r1, M, self.K, _ptr(self.Xq), _ptr(self.a_scale),
+                                         _ptr(self.T) if self.r_total else None, _ptr(self.Y_cat),
+                                         _ptr(self.ws), self.ws.numel(), _stream()), "aser_forward_shared_cat")
+        return self._views(M)
 
 
 def forward_host(layer: AserLinear, X_host: torch.Tensor, Y_host: torch.Tensor):

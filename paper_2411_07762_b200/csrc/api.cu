@@ -92,7 +92,7 @@ int check_device() {
 int linear_common(const int8_t* Xq, const float* a_scale, const void* Wk, const float* w_scale,
                   const void* T_bf16, const void* LB_f16, int M, int N, int K, int r, void* Y_f16,
                   int32_t* acc_debug, void* workspace, size_t workspace_bytes, void* stream,
-                  bool overlap_prev = false, int ldt = 0) {
+                  bool overlap_prev = false, int ldt = 0, CatSplit cat = CatSplit()) {
     if (!shape_ok(M, N, K, r)) return fail(ASER_ERR_SHAPE, "unsupported M, N, K or r");
     if (r > 0 && ldt != 0 && (ldt < r || ldt % 8 != 0))
         return fail(ASER_ERR_SHAPE, "ldt must be a multiple of 8 and at least r");
@@ -117,12 +117,12 @@ int linear_common(const int8_t* Xq, const float* a_scale, const void* Wk, const 
                                     static_cast<const __nv_bfloat16*>(T_bf16),
                                     static_cast<const __half*>(LB_f16), M, N, K, r,
                                     static_cast<__half*>(Y_f16), acc_debug,
-                                    static_cast<cudaStream_t>(stream), overlap_prev, ldt);
+                                    static_cast<cudaStream_t>(stream), overlap_prev, ldt, cat);
     return launch_linear_tc(Xq, a_scale, static_cast<const uint8_t*>(Wk), w_scale,
                             static_cast<const __nv_bfloat16*>(T_bf16),
                             static_cast<const __half*>(LB_f16), M, N, K, r,
                             static_cast<__half*>(Y_f16), acc_debug, workspace, workspace_bytes,
-                            static_cast<cudaStream_t>(stream), overlap_prev, ldt);
+                            static_cast<cudaStream_t>(stream), overlap_prev, ldt, cat);
 }
 
 // Stacked ranks (several layers' down projections in one pass) go up to 512.
@@ -448,6 +448,89 @@ int aser_forward_shared(const void* X_f16, const float* s, const void* LA_stacke
         col += r[l];
     }
     return ASER_OK;
+}
+
+// The layers of a shared-input group stored one after the other along N (weights, scales, L_B and
+// the columns of Y), all of one rank: bounds for the kernels, or an error text.
+static const char* cat_split_of(int n_layers, const int* N, int r, int* n_total, CatSplit* cat) {
+    if (n_layers < 1 || n_layers > 4) return "n_layers must be 1..4";
+    if (N == nullptr) return "N is NULL";
+    long long total = 0;
+    int bound[4] = {0x7fffffff, 0x7fffffff, 0x7fffffff, 0x7fffffff};
+    for (int l = 0; l < n_layers; ++l) {
+        if (N[l] <= 0 || N[l] % 128 != 0) return "every layer's N must be a positive multiple of 128";
+        total += N[l];
+        if (l + 1 < n_layers) bound[l] = (int)total;
+    }
+    if (total > 0x7fffffff || (long long)r * n_layers > 512) return "stacked sizes out of range";
+    *n_total = (int)total;
+    cat->layers = n_layers;
+    cat->b1 = bound[0]; cat->b2 = bound[1]; cat->b3 = bound[2];
+    return nullptr;
+}
+
+int aser_linear_w4a8_lr_cat(const int8_t* Xq, const float* a_scale, const void* Wk_cat, const float* w_scale_cat,
+                            const void* T_bf16, const void* LB_cat_f16, int n_layers, const int* N, int r,
+                            int M, int K, void* Y_cat_f16, void* workspace, size_t workspace_bytes,
+                            void* stream) {
+    int n_total = 0;
+    CatSplit cat;
+    const char* why = cat_split_of(n_layers, N, r, &n_total, &cat);
+    if (why) return fail(ASER_ERR_SHAPE, why);
+    return linear_common(Xq, a_scale, Wk_cat, w_scale_cat, T_bf16, LB_cat_f16, M, n_total, K, r, Y_cat_f16,
+                         nullptr, workspace, workspace_bytes, stream, false, r * n_layers, cat);
+}
+
+size_t aser_forward_shared_cat_workspace_bytes(int n_layers, const int* N, int r, int M, int K) {
+    int n_total = 0;
+    CatSplit cat;
+    if (cat_split_of(n_layers, N, r, &n_total, &cat)) return 0;
+    if (!shape_ok(M, n_total, K, r)) return 0;
+    const size_t lin = kWsHeaderBytes + linear_tc_workspace_bytes(M, n_total, K, r);
+    const size_t act = aser_quant_workspace_bytes(M, K, r * n_layers);
+    if (act == 0) return 0;
+    return act > lin ? act : lin;
+}
+
+int aser_forward_shared_cat(const void* X_f16, const float* s, const void* LA_stacked_f16, int n_layers,
+                            const void* Wk_cat, const float* w_scale_cat, const void* LB_cat_f16,
+                            const int* N, int r, int M, int K, int8_t* Xq, float* a_scale, void* T_bf16,
+                            void* Y_cat_f16, void* workspace, size_t workspace_bytes, void* stream) {
+    int n_total = 0;
+    CatSplit cat;
+    const char* why = cat_split_of(n_layers, N, r, &n_total, &cat);
+    if (why) return fail(ASER_ERR_SHAPE, why);
+    const size_t need = aser_forward_shared_cat_workspace_bytes(n_layers, N, r, M, K);
+    if (need == 0) return fail(ASER_ERR_SHAPE, "unsupported M, N, K or r (stacked ranks go up to 512)");
+    if (M == 0) return ASER_OK;
+    const int r_total = r * n_layers;
+    // every argument of both launches is checked before the first one is enqueued
+    ASER_REQUIRE_PTR(X_f16);
+    ASER_OPTIONAL_PTR(s);
+    ASER_REQUIRE_PTR(Xq);
+    ASER_REQUIRE_PTR(a_scale);
+    ASER_REQUIRE_PTR(Wk_cat);
+    ASER_REQUIRE_PTR(w_scale_cat);
+    ASER_REQUIRE_PTR(Y_cat_f16);
+    if (r > 0) {
+        ASER_REQUIRE_PTR(LA_stacked_f16);
+        ASER_REQUIRE_PTR(T_bf16);
+        ASER_REQUIRE_PTR(LB_cat_f16);
+    }
+    if (workspace == nullptr || misaligned16(workspace) || workspace_bytes < need)
+        return fail(ASER_ERR_WORKSPACE, "workspace missing, misaligned or too small");
+    int rc = check_device();
+    if (rc != ASER_OK) return rc;
+    if (!linear_decode_prefers(M, n_total, K)) {
+        rc = linear_tc_check(M, n_total, K, r, workspace_bytes);
+        if (rc != ASER_OK) return rc;
+    }
+    rc = quant_with_workspace(X_f16, s, LA_stacked_f16, M, K, r_total, 8, false, Xq, a_scale, T_bf16,
+                              workspace, workspace_bytes, stream);
+    if (rc != ASER_OK) return rc;
+    return linear_common(Xq, a_scale, Wk_cat, w_scale_cat, r > 0 ? T_bf16 : nullptr, r > 0 ? LB_cat_f16 : nullptr,
+                         M, n_total, K, r, Y_cat_f16, nullptr, workspace, workspace_bytes, stream,
+                         /*overlap_prev=*/true, r_total, cat);
 }
 
 int aser_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {

@@ -53,6 +53,16 @@ int launch_construct(const __half* W, const float* s, const __half* Xcal, int N,
 int launch_linear_simt(const int8_t* Xq, const float* a_scale, const uint8_t* Wq,
                        const float* w_scale, const __nv_bfloat16* T, const __half* LB,
                        int M, int N, int K, int r, __half* Y, int32_t* acc_debug, cudaStream_t st);
+// Several layers stacked along N that read the same activations, served by one launch: rows
+// [0, b1) are layer 0, [b1, b2) layer 1, ... (bounds are multiples of 128; at most four layers, all
+// of rank r); layer l takes the columns [l r, (l + 1) r) of T.  The default is a single layer.
+struct CatSplit {
+    int layers = 1;
+    int b1 = 0x7fffffff, b2 = 0x7fffffff, b3 = 0x7fffffff;
+};
+__host__ __device__ inline int cat_layer(const CatSplit& c, int row) {
+    return (row >= c.b1 ? 1 : 0) + (row >= c.b2 ? 1 : 0) + (row >= c.b3 ? 1 : 0);
+}
 // `ldt`: elements between rows of T (0 = r; larger when T is a column range of a wider matrix).
 // `overlap_prev`: the kernel launched before this one on `st` is this library's quant_act for
 // the same step.  The linear kernel may then start while that one still runs: it streams the
@@ -62,7 +72,7 @@ int launch_linear_tc(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
                      const float* w_scale, const __nv_bfloat16* T, const __half* LB,
                      int M, int N, int K, int r, __half* Y, int32_t* acc_debug,
                      void* workspace, size_t workspace_bytes, cudaStream_t st,
-                     bool overlap_prev = false, int ldt = 0);
+                     bool overlap_prev = false, int ldt = 0, CatSplit cat = CatSplit());
 // Few-token kernel (M <= kLinearDecodeMaxTokens): streams the weights once, no workspace.
 // linear_decode_prefers: the shapes for which it is faster than the tensor-core kernel.
 constexpr int kLinearDecodeMaxTokens = 16;
@@ -70,7 +80,7 @@ bool linear_decode_prefers(int M, int N, int K);
 int launch_linear_decode(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
                          const float* w_scale, const __nv_bfloat16* T, const __half* LB,
                          int M, int N, int K, int r, __half* Y, int32_t* acc_debug,
-                         cudaStream_t st, bool overlap_prev = false, int ldt = 0);
+                         cudaStream_t st, bool overlap_prev = false, int ldt = 0, CatSplit cat = CatSplit());
 size_t linear_tc_workspace_bytes(int M, int N, int K, int r);
 // The range checks launch_linear_tc makes before it launches (workspace size, index widths), for
 // callers that must reject a call before they enqueue anything else.  Records the error text.

@@ -91,7 +91,7 @@ __global__ void __launch_bounds__(kDecThreads, DecCfg<NT, R, B>::MinCtas)
 linear_decode_kernel(const int8_t* Xq, const float* a_scale, const uint8_t* __restrict__ Wk,
                      const float* __restrict__ w_scale, const __nv_bfloat16* T,
                      const __half* __restrict__ LB, int M, int N, int K, int r, int ldt,
-                     __half* __restrict__ Y, int32_t* __restrict__ acc_debug) {
+                     __half* __restrict__ Y, int32_t* __restrict__ acc_debug, const CatSplit cat) {
     using C = DecCfg<NT, R, B>;
     constexpr int BATCH = C::Batch;
     // partial sums of the eight warps: integer accumulators and fp32 accumulators of the low-rank term
@@ -101,6 +101,7 @@ linear_decode_kernel(const int8_t* Xq, const float* a_scale, const uint8_t* __re
     const int g = lane >> 2, t = lane & 3;       // fragment row group / k quarter
     const int KB = K / kWkCols;
     const int n0 = blockIdx.x * C::Rows;
+    T += cat_layer(cat, n0) * r;        // a CTA's rows lie inside one layer (16 R divides 128)
     // Rows n0 + 16 rt + g and + 8 of sub-block t (columns 32 t .. 32 t + 31 of a block).  The
     // blocked layout pads the last 128-row tile with zero codes, so rows past N inside that tile
     // read as zeros; a CTA never reaches past the tile (16 R divides 128).
@@ -276,7 +277,7 @@ linear_decode_kernel(const int8_t* Xq, const float* a_scale, const uint8_t* __re
 template <int NT, int R, int B>
 int launch_cfg(const int8_t* Xq, const float* a_scale, const uint8_t* Wk, const float* w_scale,
                const __nv_bfloat16* T, const __half* LB, int M, int N, int K, int r, __half* Y,
-               int32_t* acc_debug, cudaStream_t st, bool overlap_prev, int ldt) {
+               int32_t* acc_debug, cudaStream_t st, bool overlap_prev, int ldt, CatSplit cat) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((N + DecCfg<NT, R, B>::Rows - 1) / DecCfg<NT, R, B>::Rows, 1, 1);
     cfg.blockDim = dim3(kDecThreads, 1, 1);
@@ -288,7 +289,7 @@ int launch_cfg(const int8_t* Xq, const float* a_scale, const uint8_t* Wk, const 
     cfg.attrs = attr;
     cfg.numAttrs = overlap_prev ? 1 : 0;
     cudaError_t e = cudaLaunchKernelEx(&cfg, linear_decode_kernel<NT, R, B>, Xq, a_scale, Wk, w_scale, T, LB,
-                                       M, N, K, r, ldt, Y, acc_debug);
+                                       M, N, K, r, ldt, Y, acc_debug, cat);
     if (e != cudaSuccess) return record_cuda_error(e, "linear_decode_kernel");
     return check_launch("linear_decode_kernel");
 }
@@ -296,7 +297,7 @@ int launch_cfg(const int8_t* Xq, const float* a_scale, const uint8_t* Wk, const 
 template <int NT>
 int launch_nt(const int8_t* Xq, const float* a_scale, const uint8_t* Wk, const float* w_scale,
               const __nv_bfloat16* T, const __half* LB, int M, int N, int K, int r, __half* Y,
-              int32_t* acc_debug, cudaStream_t st, bool overlap_prev, int ldt) {
+              int32_t* acc_debug, cudaStream_t st, bool overlap_prev, int ldt, CatSplit cat) {
     // Rows per CTA: 32 where that still gives every SM about one and a half CTAs (activation
     // fragments reused twice), else 16 (few output channels: latency matters, every SM gets work).
     int num_sms = 0;
@@ -307,8 +308,8 @@ int launch_nt(const int8_t* Xq, const float* a_scale, const uint8_t* Wk, const f
     // (Four blocks in flight per warp at 32 rows, i.e. 256 bytes per thread and two CTAs per SM,
     // measured 7 % slower at 8192 x 8192 than two blocks and three CTAs per SM.)
     if (N >= 32 * 3 * num_sms / 2)
-        return launch_cfg<NT, 2, 2>(Xq, a_scale, Wk, w_scale, T, LB, M, N, K, r, Y, acc_debug, st, overlap_prev, ldt);
-    return launch_cfg<NT, 1, 4>(Xq, a_scale, Wk, w_scale, T, LB, M, N, K, r, Y, acc_debug, st, overlap_prev, ldt);
+        return launch_cfg<NT, 2, 2>(Xq, a_scale, Wk, w_scale, T, LB, M, N, K, r, Y, acc_debug, st, overlap_prev, ldt, cat);
+    return launch_cfg<NT, 1, 4>(Xq, a_scale, Wk, w_scale, T, LB, M, N, K, r, Y, acc_debug, st, overlap_prev, ldt, cat);
 }
 
 }  // namespace
@@ -320,11 +321,11 @@ bool linear_decode_prefers(int M, int N, int K) {
 int launch_linear_decode(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
                          const float* w_scale, const __nv_bfloat16* T, const __half* LB,
                          int M, int N, int K, int r, __half* Y, int32_t* acc_debug,
-                         cudaStream_t st, bool overlap_prev, int ldt) {
-    if (ldt <= 0) ldt = r;
+                         cudaStream_t st, bool overlap_prev, int ldt, CatSplit cat) {
+    if (ldt <= 0) ldt = r * cat.layers;
     if (M > kLinearDecodeMaxTokens) return record_error(ASER_ERR_SHAPE, "linear_decode: more than 16 tokens");
-    if (M <= 8) return launch_nt<1>(Xq, a_scale, Wk, w_scale, T, LB, M, N, K, r, Y, acc_debug, st, overlap_prev, ldt);
-    return launch_nt<2>(Xq, a_scale, Wk, w_scale, T, LB, M, N, K, r, Y, acc_debug, st, overlap_prev, ldt);
+    if (M <= 8) return launch_nt<1>(Xq, a_scale, Wk, w_scale, T, LB, M, N, K, r, Y, acc_debug, st, overlap_prev, ldt, cat);
+    return launch_nt<2>(Xq, a_scale, Wk, w_scale, T, LB, M, N, K, r, Y, acc_debug, st, overlap_prev, ldt, cat);
 }
 
 }  // namespace aser

@@ -97,6 +97,7 @@ struct Params {
     int units;             // NT * TT * KB
     int tail_first;        // work order: 1 = both shared tiles first, 0 = range order
     int tt_outer;          // tile numbering: 1 = token tile outer (consecutive tiles share the activations)
+    CatSplit cat;          // layers stacked along N: which columns of T a weight tile multiplies
 };
 
 struct Work {
@@ -399,7 +400,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 const int s = cl % C::NL;
                 mbar_arrive_expect_tx(bar(B_FULL_LR + s), C::LbBytes + C::TBytes);
                 tma_load_2d(sbase + C::OffLb + s * C::LbBytes, &map_lb, c * 64, w.nt * 128, bar(B_FULL_LR + s));
-                tma_load_2d(sbase + C::OffT + s * C::TBytes, &map_t, c * 64, w.tt * BT, bar(B_FULL_LR + s));
+                tma_load_2d(sbase + C::OffT + s * C::TBytes, &map_t, c * 64 + cat_layer(p.cat, w.nt * 128) * p.r, w.tt * BT,
+                            bar(B_FULL_LR + s));
                 ++cl;
             };
             auto issue_lr = [&](int c) {
@@ -934,7 +936,8 @@ int linear_tc_check(int M, int N, int K, int r, size_t workspace_bytes) {
 int launch_linear_tc(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
                      const float* w_scale, const __nv_bfloat16* T, const __half* LB,
                      int M, int N, int K, int r, __half* Y, int32_t* acc_debug,
-                     void* workspace, size_t workspace_bytes, cudaStream_t st, bool overlap_prev, int ldt) {
+                     void* workspace, size_t workspace_bytes, cudaStream_t st, bool overlap_prev, int ldt,
+                     CatSplit cat) {
     Layout L = make_layout(M, N, K, r);
     const int pre = linear_tc_check(M, N, K, r, workspace_bytes);
     if (pre != ASER_OK) return pre;
@@ -987,7 +990,7 @@ int launch_linear_tc(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
     if (r > 0) {
         rc = make_map_2d(&mlb, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, LB, N, r, 128, 64);
         if (rc != ASER_OK) return rc;
-        rc = encode_map_2d_ld(&mt, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, T, M, r, ldt > 0 ? ldt : r, L.BT, 64,
+        rc = encode_map_2d_ld(&mt, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, T, M, r * cat.layers, ldt > 0 ? ldt : r * cat.layers, L.BT, 64,
                               CU_TENSOR_MAP_SWIZZLE_128B);
         if (rc != ASER_OK) return rc;
     } else {
@@ -1003,6 +1006,7 @@ int launch_linear_tc(const int8_t* Xq, const float* a_scale, const uint8_t* Wk,
     p.part_int = reinterpret_cast<int32_t*>(ws + L.off_part_int);
     p.part_lr = reinterpret_cast<float*>(ws + L.off_part_lr);
     p.M = M; p.N = N; p.K = K; p.r = r;
+    p.cat = cat;
     p.KB = L.KB; p.TT = L.TT; p.NT = L.NT; p.units = (int)L.units;
     // Both shared tiles first where a tile is long enough (K >= 8192) to hide two cross-CTA
     // reductions behind the next tiles' MMAs; with shorter tiles the epilogue warps fall behind

@@ -498,6 +498,10 @@ def test_status_word_reports_a_timeout_and_clears(aser):
 
 SHARED_CASES = [  # M, K, [(N, r), ...]
     (8, 1024, [(256, 32), (128, 16), (128, 16)]),
+    (8, 1024, [(256, 32), (128, 32), (384, 32), (128, 32)]),
+    (16, 2048, [(1024, 64), (256, 64)]),
+    (200, 1024, [(384, 64), (128, 64)]),
+    (1100, 1024, [(256, 128), (128, 128), (128, 128)]),
     (200, 1024, [(384, 64), (136, 48), (128, 0)]),
     (300, 2048, [(512, 128), (256, 128), (256, 128)]),
 ]
@@ -546,6 +550,24 @@ def check_shared_group(aser, M, K, spec, seed0, construct, gain=30.0):
                 b = lay.T[:M].float()
                 assert bool(((a - b).abs() <= 2.0 ** -7 * b.abs() + 2.0 ** -9 * b.abs().max()).all())
                 col += lay.r
+    # the same group stored as one fused projection (one linear launch over the concatenated N)
+    ranks = {r for _, r in spec}
+    if len(ranks) == 1 and all(N % 128 == 0 for N, _ in spec) and len(spec) <= 4:
+        per_layer = [y.clone() for y in group(X)]
+        cat = aser.AserSharedInputCat(layers, M)
+        for rep in range(2):
+            Ys = cat(X)
+            aser.check_status(cat.ws)
+            torch.cuda.synchronize()
+            assert np.array_equal(cat.Xq[:M].cpu().numpy(), refs[0].Xq)
+            for ref, Y, Y1 in zip(refs, Ys, per_layer):
+                assert_rows_close(Y.cpu().numpy(), ref.y)
+                # same operands, same arithmetic per element as the layer's own launch
+                assert torch.equal(Y, Y1)
+        Ys = cat.linear(M)                  # the linear step alone on the codes already there
+        torch.cuda.synchronize()
+        for ref, Y in zip(refs, Ys):
+            assert_rows_close(Y.cpu().numpy(), ref.y)
 
 
 @pytest.mark.gpu

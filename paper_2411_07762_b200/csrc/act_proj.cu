@@ -9,13 +9,12 @@
 //                      and the 128 tokens on the N side; the partial T of the slice goes to the
 //                      scratch as fp32 and the partial row maxima beside it.
 //   act_quant_kernel   per token row: the scale from the slices' maxima, the int8 codes (X comes
-//                      from L2 where the chunk of tokens was sized to stay there), and T as the
-//                      sum of the slices' partials in a fixed order, rounded to bf16.
+//                      from L2 as far as it is still there), and T as the sum of the slices'
+//                      partials in a fixed order, rounded to bf16.
 //
 // (Sec. 4.2 smoothing M^-1 X of Eq. 10, Sec. 5.1 per-token round-to-nearest, Sec. 4.1 projection
 // V_r^T S^-1 of the reconstruction branch.)  Both kernels are deterministic: no atomics.
-// Long inputs are processed in chunks of tokens small enough for the second kernel to find X in
-// L2.  Every mbarrier wait is bounded; a CTA that gives up poisons its row maxima with NaN.
+// Every mbarrier wait is bounded; a CTA that gives up poisons its row maxima with NaN.
 #include "act_math.cuh"
 #include "aser_common.cuh"
 #include "sm100_ptx.cuh"
@@ -547,30 +546,18 @@ struct ProjPlan {
     int KS;         // slices of K
 };
 
-// Chunk and slice sizes.  A chunk's X (2 Mc K bytes) should stay in L2 between the two kernels;
-// within that, take the chunk and the slice count that fill the SMs best in one wave (a slice
-// has at least four 64-column stages), preferring fewer chunks.
+// Slice count: as many slices of K as keep the grid within one wave (a slice has at least four
+// 64-column stages).  The whole input is one chunk: splitting long inputs into chunks of tokens
+// whose X stays in L2 for the second kernel cost more in fixed time per launch pair than the L2
+// hits saved (4096 x 14336 at rank 128: 140 us in three chunks, 95 us in one; 8192 x 8192: 140
+// against 107 us), so the chunk loop below runs once.
 ProjPlan proj_plan(int M, int K, int num_sms) {
-    const long long l2_budget = 48ll << 20;
     const int blocks = K / kPCols;
-    int max_tiles = (int)(l2_budget / (2ll * K * kPTok));
-    if (max_tiles < 1) max_tiles = 1;
-    const int all_tiles = (M + kPTok - 1) / kPTok;
-    ProjPlan best{M, 1};
-    double best_score = -1.0;
-    for (int tiles = (all_tiles <= max_tiles ? all_tiles : max_tiles); tiles >= 1; --tiles) {
-        const int n_chunks = (all_tiles + tiles - 1) / tiles;
-        int ks_best = 1;
-        for (int ks = 1; ks <= blocks / 4 && tiles * ks <= num_sms; ++ks)
-            if (blocks % ks == 0) ks_best = ks;
-        // SM-time of the whole call in units of (one SM busy for one full-K tile)
-        const double per_chunk = 1.0 / ks_best + 0.15;          // streaming share plus fixed cost
-        const double score = 1.0 / (n_chunks * per_chunk);
-        if (score > best_score * 1.02) { best_score = score; best = ProjPlan{tiles * kPTok, ks_best}; }
-        if (tiles == all_tiles && tiles * ks_best * 10 >= num_sms * 8) break;   // one chunk fills the SMs
-    }
-    if (best.Mc > M) best.Mc = M;
-    return best;
+    const int tiles = (M + kPTok - 1) / kPTok;
+    int ks_best = 1;
+    for (int ks = 1; ks <= blocks / 4 && tiles * ks <= num_sms; ++ks)
+        if (blocks % ks == 0) ks_best = ks;
+    return ProjPlan{M, ks_best};
 }
 
 // Floats of the row-maxima part of the scratch, padded so that the partial T behind it starts on

@@ -132,17 +132,16 @@ bool act_shape_ok(int M, int K, int r) {
 
 // Which activation kernels a forward pass runs.  The two-kernel path with scratch reads X once
 // from HBM whatever the rank; it is the only one above rank 128 (stacked down projections of a
-// shared-input group) and the faster one from about a thousand tokens on while X fits one of its
-// chunks (measured at rank 128, two-kernel against cluster kernel: 1024 x 4096 21 against 27 us,
-// 4096 x 4096 34 against 42 us, 2048 x 8192 34 against 42 us, 1024 x 14336 34 against 66 us).
-// Longer inputs take several chunks, two launches each, and the one-launch cluster kernel is as
-// fast or faster there (4096 x 14336: 135 against 132 us; 8192 x 4096: 71 against 60 us), as it
-// is below a thousand tokens (256 x 4096: 23 against 17 us).  Up to 32 tokens the few-token
-// kernel serves every rank.
+// shared-input group) and the faster one from about a thousand tokens on (measured at rank 128,
+// two-kernel against cluster kernel: 1024 x 4096 21 against 27 us, 4096 x 4096 34 against 42 us,
+// 2048 x 14336 52 against 65 us, 4096 x 14336 95 against 134 us, 8192 x 8192 107 against 159 us).
+// Below that the one-launch cluster kernel is faster (256 x 4096: 23 against 17 us), and up to 32
+// tokens the few-token kernel serves every rank.
 bool forward_act_uses_scratch(int M, int K, int r) {
     if (M <= 32) return false;
     if (r > 128) return true;
-    return M >= 1024 && (long long)M * K <= (1ll << 25);
+    (void)K;
+    return M >= 1024;
 }
 
 // The activation step of a forward pass (the scratch of the two-kernel path sits behind the

@@ -233,10 +233,11 @@ int aser_check_status(void* workspace, void* stream);
  * Because the library knows that the quantization kernel is what precedes the linear kernel,
  * it launches the latter as a programmatic dependent: the linear kernel starts while the
  * quantization still runs, streams the weights (which that kernel does not write) and waits
- * for its completion before it reads Xq, a_scale or T.  The activation step is aser_quant_act's
- * kernels up to rank 128 and aser_quant_act_ws's (on the same workspace) above, whichever is
- * faster at the shape; aser_forward_act_launches tells how many kernels that is.  Results are
- * those of the separate calls.
+ * for its completion before it reads Xq, a_scale or T.  The activation step is whichever of
+ * aser_quant_act's kernels and aser_quant_act_ws's (on the same workspace) is faster at the
+ * shape: the latter from 1024 tokens on and for every rank above 128;
+ * aser_forward_act_launches tells how many kernels that is.  Results are those of the separate
+ * calls.
  * X_f16 [M,K], s [K] or NULL, LA_f16 [r,K] / LB_f16 [N,r] (NULL when r == 0), Wk and w_scale as
  * for aser_linear_w4a8_lr.  Xq [M,K], a_scale [M], T_bf16 [M,r] (NULL when r == 0) are the
  * caller's intermediates (written), Y_f16 [M,N] the result.  Wk, w_scale and LB_f16 must not

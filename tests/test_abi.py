@@ -66,6 +66,22 @@ def test_bad_arguments_are_rejected_before_launch(lib):
     assert lib.aser_linear_w4a8(good, good, good, good, 4, 128, 128, good, None, good, 8, None) == WORKSPACE
     assert lib.aser_workspace_init(None, 1024, None) == WORKSPACE
     assert lib.aser_last_error() != b""
+    # a fused shared-input group: layer count, N a multiple of 128, one rank within the stacked limit
+    i3 = (C.c_int * 3)(256, 128, 128)
+    bad_n = (C.c_int * 2)(256, 136)
+    i5 = (C.c_int * 5)(128, 128, 128, 128, 128)
+    cat = lambda n, N, r, ws=good, nbytes=1 << 24: lib.aser_linear_w4a8_lr_cat(
+        good, good, good, good, good, good, n, N, r, 64, 256, good, ws, nbytes, None)
+    assert cat(5, i5, 16) == SHAPE
+    assert cat(2, bad_n, 16) == SHAPE
+    assert cat(3, i3, 192) == SHAPE                 # 3 x 192 stacked rows of T
+    assert cat(0, i3, 16) == SHAPE
+    assert cat(3, None, 16) == SHAPE
+    assert cat(3, i3, 16, None, 0) == WORKSPACE
+    assert lib.aser_forward_shared_cat_workspace_bytes(3, i3, 16, 64, 256) >= lib.aser_workspace_bytes(64, 512, 256, 16)
+    assert lib.aser_forward_shared_cat_workspace_bytes(2, bad_n, 16, 64, 256) == 0
+    assert lib.aser_forward_shared_cat(good, None, good, 3, good, good, good, i3, 16, 64, 256, good, good, good,
+                                       None, good, 1 << 24, None) == NULL      # Y missing
 
 
 def test_binding_refuses_cpu_tensors(lib):

@@ -116,6 +116,24 @@ def test_quant_act_dense_smoothing_vector(aser, M, K, r):
     assert_T_close(T.float().cpu().numpy(), F.down_proj(xs, L_A), xs, L_A)
 
 
+@pytest.mark.parametrize("path,M,K,r", [("cluster", 4096, 4096, 64), ("ws", 4800, 8192, 16)])
+def test_quant_act_dense_smoothing_long_slices(aser, path, M, K, r):
+    """Every divisor differs from 1 on slices long enough that a CTA meets more units with a
+    divisor than it keeps in shared memory (the cluster kernel keeps 62 of its 128, the
+    projection kernel 254 of its 256): the rest read their divisors from global memory."""
+    lay = synth.make_layer(M, 8, K, seed=430 + M + K + r, n_cal=8)
+    rng = np.random.default_rng(M + K + 1)
+    s = rng.uniform(0.25, 6.0, size=K).astype(np.float32)
+    L_A = synth.standin_factors(8, K, r, seed=M, scale_a=0.05)[0]
+    xs = F.smooth_act(lay.X, s)
+    Xq_ref, sc_ref = F.quant_act(xs)
+    fn = aser.quant_act if path == "cluster" else aser.quant_act_ws
+    Xq, sc, T = fn(to_dev(lay.X), to_dev(s), to_dev(L_A))
+    assert np.array_equal(Xq.cpu().numpy(), Xq_ref)
+    assert np.array_equal(bits(sc.cpu().numpy()), bits(sc_ref))
+    assert_T_close(T.float().cpu().numpy(), F.down_proj(xs, L_A), xs, L_A)
+
+
 def test_quant_act_without_smoothing_vector(aser):
     lay = synth.make_layer(5, 8, 256, seed=9, n_cal=8)
     Xq, sc, _ = aser.quant_act(to_dev(lay.X), None, None)

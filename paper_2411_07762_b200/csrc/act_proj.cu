@@ -287,22 +287,38 @@ act_proj_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                                                        : reinterpret_cast<const float4*>(s + k0 + i * kPCols + cw * 8);
                 const float4 s0 = sp[0], s1 = sp[1];
                 const float sv[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+                // Only the columns with a divisor (the same for every lane: lanes are rows) take
+                // the fp32 division and maximum and are written back as fp16(x~); the others go
+                // through the half-precision maximum like an untagged unit, with the divided
+                // columns blanked out of that maximum.
+                uint32_t wd[4][4], zd[4][4];
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
-                    const __half* h = reinterpret_cast<const __half*>(&v[q]);
-                    float f[8];
+                    wd[q][0] = v[q].x; wd[q][1] = v[q].y; wd[q][2] = v[q].z; wd[q][3] = v[q].w;
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        f[e] = __half2float(h[e]);
-                        if (sv[e] != 1.f) f[e] = __fdiv_rn(f[e], sv[e]);
-                        amax[q] = fmaxf(amax[q], fabsf(f[e]));
+                    for (int i = 0; i < 4; ++i) zd[q][i] = wd[q][i];
+                }
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    if (sv[e] != 1.f) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const uint32_t word = wd[q][e >> 1];
+                            const __half hv = __ushort_as_half((unsigned short)((e & 1) ? (word >> 16) : (word & 0xffffu)));
+                            const float f = __fdiv_rn(__half2float(hv), sv[e]);
+                            amax[q] = fmaxf(amax[q], fabsf(f));
+                            const uint32_t hb = (uint32_t)__half_as_ushort(__float2half_rn(f));
+                            wd[q][e >> 1] = (e & 1) ? ((word & 0x0000ffffu) | (hb << 16)) : ((word & 0xffff0000u) | hb);
+                            zd[q][e >> 1] &= (e & 1) ? 0x0000ffffu : 0xffff0000u;
+                        }
                     }
-                    __half2 p0 = __floats2half2_rn(f[0], f[1]), p1 = __floats2half2_rn(f[2], f[3]);
-                    __half2 p2 = __floats2half2_rn(f[4], f[5]), p3 = __floats2half2_rn(f[6], f[7]);
-                    uint4 pk;
-                    pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
-                    pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
-                    pj_sts128(addr[q], pk);
+                }
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+                        hmax[q] = __hmax2(hmax[q], __habs2(*reinterpret_cast<const __half2*>(&zd[q][i])));
+                    pj_sts128(addr[q], make_uint4(wd[q][0], wd[q][1], wd[q][2], wd[q][3]));
                 }
                 fence_proxy_async_smem();       // the MMA reads these through the async proxy
             }

@@ -487,14 +487,6 @@ __device__ __forceinline__ void div8(const uint4& raw, const float4& s0, const f
     if (s1.z != 1.f) v[6] = __fdiv_rn(v[6], s1.z);
     if (s1.w != 1.f) v[7] = __fdiv_rn(v[7], s1.w);
 }
-__device__ __forceinline__ uint4 pack8_half(const float (&v)[8]) {
-    uint4 pk;
-    __half2 p0 = __floats2half2_rn(v[0], v[1]), p1 = __floats2half2_rn(v[2], v[3]);
-    __half2 p2 = __floats2half2_rn(v[4], v[5]), p3 = __floats2half2_rn(v[6], v[7]);
-    pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
-    pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
-    return pk;
-}
 
 // grid = (CK, ceil(M / 64)), cluster = (CK, 1, 1) with CK a power of two <= 16, kTThreads threads,
 // r <= 128.  T has `ldt` elements per row (the launch may cover a column range of a wider T).
@@ -753,23 +745,49 @@ quant_act_tma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 const float4* sp = (tag1 != kTUncached) ? reinterpret_cast<const float4*>(s_cache + (tag1 - 1) * 16)
                                                         : reinterpret_cast<const float4*>(s + k0 + i * kTCols + cg * 16);
                 const float4 s0 = sp[0], s1 = sp[1], s2 = sp[2], s3 = sp[3];
-                float v[8];
-                div8(v0, s0, s1, v);
+                // Only the columns with a divisor (the same for every lane: lanes are rows) take
+                // the fp32 division and maximum and are written back as fp16(x~); the others go
+                // through the half-precision maximum like an untagged unit, with the divided
+                // columns blanked out of that maximum.  Pieces: 0 and 1 are this lane's first row
+                // (columns 0..7 and 8..15 of the unit), 2 and 3 the row 32 further down.
+                const float sv[16] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w,
+                                      s2.x, s2.y, s2.z, s2.w, s3.x, s3.y, s3.z, s3.w};
+                uint32_t wd[4][4] = {{v0.x, v0.y, v0.z, v0.w}, {v1.x, v1.y, v1.z, v1.w},
+                                     {w0.x, w0.y, w0.z, w0.w}, {w1.x, w1.y, w1.z, w1.w}};
+                uint32_t zd[4][4];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) amax0 = fmaxf(amax0, fabsf(v[e]));
-                sts128(a0, pack8_half(v));
-                div8(v1, s2, s3, v);
+                for (int pc = 0; pc < 4; ++pc)
 #pragma unroll
-                for (int e = 0; e < 8; ++e) amax0 = fmaxf(amax0, fabsf(v[e]));
-                sts128(a1, pack8_half(v));
-                div8(w0, s0, s1, v);
+                    for (int i = 0; i < 4; ++i) zd[pc][i] = wd[pc][i];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) amax1 = fmaxf(amax1, fabsf(v[e]));
-                sts128(a0 + kRow32, pack8_half(v));
-                div8(w1, s2, s3, v);
+                for (int e = 0; e < 16; ++e) {
+                    if (sv[e] != 1.f) {
+                        const int wi = (e & 7) >> 1;
 #pragma unroll
-                for (int e = 0; e < 8; ++e) amax1 = fmaxf(amax1, fabsf(v[e]));
-                sts128(a1 + kRow32, pack8_half(v));
+                        for (int rr = 0; rr < 2; ++rr) {
+                            const int pc = 2 * rr + (e >> 3);
+                            const uint32_t word = wd[pc][wi];
+                            const __half hv = __ushort_as_half((unsigned short)((e & 1) ? (word >> 16) : (word & 0xffffu)));
+                            const float f = __fdiv_rn(__half2float(hv), sv[e]);
+                            if (rr == 0) amax0 = fmaxf(amax0, fabsf(f));
+                            else amax1 = fmaxf(amax1, fabsf(f));
+                            const uint32_t hb = (uint32_t)__half_as_ushort(__float2half_rn(f));
+                            wd[pc][wi] = (e & 1) ? ((word & 0x0000ffffu) | (hb << 16)) : ((word & 0xffff0000u) | hb);
+                            zd[pc][wi] &= (e & 1) ? 0x0000ffffu : 0xffff0000u;
+                        }
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    hamax0 = __hmax2(hamax0, __habs2(*reinterpret_cast<const __half2*>(&zd[0][i])));
+                    hamax0 = __hmax2(hamax0, __habs2(*reinterpret_cast<const __half2*>(&zd[1][i])));
+                    hamax1 = __hmax2(hamax1, __habs2(*reinterpret_cast<const __half2*>(&zd[2][i])));
+                    hamax1 = __hmax2(hamax1, __habs2(*reinterpret_cast<const __half2*>(&zd[3][i])));
+                }
+                sts128(a0, make_uint4(wd[0][0], wd[0][1], wd[0][2], wd[0][3]));
+                sts128(a1, make_uint4(wd[1][0], wd[1][1], wd[1][2], wd[1][3]));
+                sts128(a0 + kRow32, make_uint4(wd[2][0], wd[2][1], wd[2][2], wd[2][3]));
+                sts128(a1 + kRow32, make_uint4(wd[3][0], wd[3][1], wd[3][2], wd[3][3]));
                 fence_proxy_async_smem();       // the MMA reads these through the async proxy
             }
             __syncwarp();

@@ -70,18 +70,19 @@ struct Cfg {
     static constexpr int OffLb = OffX + NX * XBytes;
     static constexpr int OffT = OffLb + NL * LbBytes;
     static constexpr int OffBar = OffT + NL * TBytes;
-    static constexpr int NumBars = 2 * NW + 2 * NX + 2 * NA + 3 * NL + 2 + 2 + 1;
+    static constexpr int NumBars = 2 * NW + 2 * NX + 2 * NA + 3 * NL + 2 + 2 + 2;
     // Who issues the low-rank MMAs.  The two integer issuers spend nine tenths of their time
     // inside barrier and tensor-core instructions (a wait, MMA or commit costs its thread a few
     // hundred cycles under copy traffic), so every operation of a low-rank chunk on one of them
     // sets it back against the other and the whole pipeline with it.  A warp of its own for the
-    // job costs every thread 16 registers (21 warps: six on one scheduler), so at 128-token tiles
-    // lane 1 of the operand producer's warp does it: a third issuing thread that diverges from
-    // lane 0 for the whole kernel and spends nearly all of its time inside barrier waits.
-    // Measured against the low-rank MMAs on issuer 0: gate projection 282 -> 270 us, q/o 92.5 ->
-    // 89 us, K = 14336 224 -> 214 us; the operand producer polling for the chunks between its
-    // stages instead measured the same within 2 %.
-    static constexpr bool LrLane = (BT == 128);
+    // job costs every thread 16 registers (21 warps: six on one scheduler).  A second lane of the
+    // producer's warp as a third issuer measured the same as what is done here, but depends on how
+    // the hardware shares a warp between two diverged spinning lanes: at rank 256 the lane was
+    // starved while lane 0 waited for it, and a bounded wait gave up.  So, with the one-slot
+    // chunk ring, the thread that loads the chunks also multiplies them: it runs a few stages
+    // ahead of the MMAs, has slack, polls the chunk's barriers between its activation stages, and
+    // waits for them only where nothing it still has to do is needed for them to complete.
+    static constexpr bool ProducerLr = (NL == 1);
     static constexpr int SmemBytes = OffBar + NumBars * 8 + 128 + 1024;  // + slack for 1 KiB alignment
     static constexpr int ASlotCols = KA * 32;
     static constexpr int TmemColsUsed = 3 * BT + NA * ASlotCols;
@@ -300,15 +301,16 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     //   READY[a]   A operand of the stage written to tensor memory -> MMA issuer of the stage
     //   FREE[a]    MMAs of the stage retired (commit)         -> unpack warps
     //   FULL_LR / CONV_LR / EMPTY_LR[l]  low-rank chunk landed / converted / multiplied
-    //   ACC_FULL / ACC_EMPTY[2]  accumulators complete (every issuer arrives) / read and zeroed
+    //   ACC_FULL / ACC_EMPTY[2]  integer accumulator complete / read and zeroed by the epilogue
     //   DLR_EMPTY  the epilogue has read the low-rank accumulator -> low-rank issuer
+    //   LR_DONE    the item's low-rank MMAs retired (commit by the producer) -> epilogue
     constexpr int B_W_FULL = 0, B_W_FREE = B_W_FULL + C::NW, B_X_FULL = B_W_FREE + C::NW,
                   B_X_FREE = B_X_FULL + C::NX, B_READY = B_X_FREE + C::NX,
                   B_FREE = B_READY + C::NA, B_FULL_LR = B_FREE + C::NA,
                   B_CONV_LR = B_FULL_LR + C::NL, B_EMPTY_LR = B_CONV_LR + C::NL,
                   B_ACC_FULL = B_EMPTY_LR + C::NL, B_ACC_EMPTY = B_ACC_FULL + 2,
-                  B_DLR_EMPTY = B_ACC_EMPTY + 2;
-    static_assert(B_DLR_EMPTY + 1 == C::NumBars, "barrier count");
+                  B_DLR_EMPTY = B_ACC_EMPTY + 2, B_LR_DONE = B_DLR_EMPTY + 1;
+    static_assert(B_LR_DONE + 1 == C::NumBars, "barrier count");
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + C::OffBar + C::NumBars * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     int* last_flag = reinterpret_cast<int*>(tmem_slot + 2);
@@ -327,8 +329,9 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     if (warp == 0) {
         for (int i = lane; i < C::NumBars; i += 32) {
             const uint32_t count =
-                (i >= B_ACC_EMPTY) ? (uint32_t)C::EW
-                : (i >= B_ACC_FULL && i < B_ACC_EMPTY) ? (C::LrLane ? 3u : 2u) : 1u;
+                (i == B_LR_DONE) ? 1u
+                : (i >= B_ACC_EMPTY) ? (uint32_t)C::EW
+                : (i >= B_ACC_FULL && i < B_ACC_EMPTY) ? 2u : 1u;
             mbar_init(bar(i), count);
         }
         if (lane == 0) {
@@ -410,21 +413,74 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             Work w{};
             uint32_t cx = 0, cl = 0;
             bool ok = true;
+            // ProducerLr: the chunk most recently loaded and not yet multiplied (one slot, so
+            // there is never more than one), and the low-rank items multiplied so far.
+            bool job = false, job_last = false, dlr_ok = false;
+            int job_c = 0;
+            uint32_t job_cl = 0, lr_items = 0;
+            constexpr uint32_t idesc_lr = make_idesc(1, 0, 128, BT);
+            auto run_job = [&]() {          // its conversion is complete: multiply, hand the slot back
+                const int s = job_cl % C::NL;
+                tc_fence_after();
+                const uint64_t adesc = smem_desc_sw128(sbase + C::OffLb + s * C::LbBytes);
+                const uint64_t bdesc = smem_desc_sw128(sbase + C::OffT + s * C::TBytes);
+                int steps = (p.r - job_c * 64) / 16;
+                if (steps > 4) steps = 4;
+                for (int kk = 0; kk < steps; ++kk)
+                    mma_f16_ss(tm_dlr, adesc + 2 * kk, bdesc + 2 * kk, idesc_lr, (job_c != 0 || kk != 0) ? 1u : 0u);
+                tc_commit(bar(B_EMPTY_LR + s));
+                if (job_last) {             // the item's low-rank term is complete when these retire
+                    tc_commit(bar(B_LR_DONE));
+                    ++lr_items;
+                    dlr_ok = false;
+                }
+                job = false;
+            };
+            // without waiting: multiply the pending chunk if it is ready (the first chunk of an
+            // item also needs the previous item's epilogue to have read the accumulator)
+            auto poll_job = [&]() {
+                if (!C::ProducerLr || !job) return;
+                if (job_c == 0 && !dlr_ok) {
+                    if (!mbar_try_wait(bar(B_DLR_EMPTY), (lr_items & 1) ^ 1)) return;
+                    dlr_ok = true;
+                }
+                if (!mbar_try_wait(bar(B_CONV_LR + job_cl % C::NL), (job_cl / C::NL) & 1)) return;
+                run_job();
+            };
+            // the same, waiting: before anything that waits for the slot (this thread frees it)
+            auto finish_job = [&]() -> bool {
+                if (!C::ProducerLr || !job) return true;
+                if (job_c == 0 && !dlr_ok) {
+                    if (!mbar_wait(bar(B_DLR_EMPTY), (lr_items & 1) ^ 1, ab)) return false;
+                    dlr_ok = true;
+                }
+                if (!mbar_wait(bar(B_CONV_LR + job_cl % C::NL), (job_cl / C::NL) & 1, ab)) return false;
+                run_job();
+                return true;
+            };
             auto load_lr = [&](int c) {
                 const int s = cl % C::NL;
                 mbar_arrive_expect_tx(bar(B_FULL_LR + s), C::LbBytes + C::TBytes);
                 tma_load_2d(sbase + C::OffLb + s * C::LbBytes, &map_lb, c * 64, w.nt * 128, bar(B_FULL_LR + s));
                 tma_load_2d(sbase + C::OffT + s * C::TBytes, &map_t, c * 64 + cat_layer(p.cat, w.nt * 128) * p.r, w.tt * BT,
                             bar(B_FULL_LR + s));
+                if (C::ProducerLr) {
+                    job = true;
+                    job_c = c;
+                    job_cl = cl;
+                    job_last = (c == lr_chunks - 1);
+                }
                 ++cl;
             };
             auto issue_lr = [&](int c) {
+                if (!finish_job()) return false;
                 if (!mbar_wait(bar(B_EMPTY_LR + cl % C::NL), ((cl / C::NL) & 1) ^ 1, ab)) return false;
                 load_lr(c);
                 return true;
             };
             // the same without waiting: false when the slot is still in use
             auto try_issue_lr = [&](int c) {
+                if (job) return false;
                 if (!mbar_try_wait(bar(B_EMPTY_LR + cl % C::NL), ((cl / C::NL) & 1) ^ 1)) return false;
                 load_lr(c);
                 return true;
@@ -453,6 +509,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     mbar_arrive_expect_tx(bar(B_X_FULL + s), C::XBytes);
                     tma_load_3d(sbase + C::OffX + s * C::XBytes, &map_x, 0, w.tt * BT, kb, bar(B_X_FULL + s));
                     ++cx;
+                    poll_job();
                     // mid-tile schedule: the next chunk goes out as soon as the slot is free; never
                     // wait here (the activation stages must keep flowing)
                     if (mid && mid_next < lr_chunks && try_issue_lr(mid_next)) ++mid_next;
@@ -465,6 +522,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     for (int c = early; c < lr_chunks && ok; ++c) ok = issue_lr(c);
                 }
             }
+            if (ok) ok = finish_job();      // the last item's last chunk
             if (*abort_flag) dump_role(p.status, 1, cx, cl, (uint32_t)w.tile, (uint32_t)w.kb0, (uint32_t)w.kb1);
             if (!ok || *abort_flag) {
                 // let copies already issued land before the CTA's shared memory goes away
@@ -472,48 +530,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     mbar_wait(bar(B_FULL_LR + i % C::NL), (i / C::NL) & 1, Abort{never_flag, p.status});
                 for (uint32_t i = (cx > (uint32_t)C::NX ? cx - C::NX : 0); i < cx; ++i)
                     mbar_wait(bar(B_X_FULL + i % C::NX), (i / C::NX) & 1, Abort{never_flag, p.status});
-            }
-        }
-        if (C::LrLane && lane == 1) {
-            // =================== low-rank MMA issuer (lane 1 of this warp) ===================
-            // Takes the chunks of a work item as their conversion completes.  It arrives on the
-            // item's accumulator barrier like the integer issuers (a commit where it issued
-            // MMAs), and like them it first waits for the epilogue to have released that
-            // accumulator, so that its arrival can never fall into the phase of the item two
-            // before.
-            constexpr uint32_t idesc_f16 = make_idesc(1, 0, 128, BT);
-            Cursor cur;
-            cur.init(u_begin, u_end, p);
-            Work w;
-            uint32_t cl = 0, ci = 0, clr_items = 0;
-            bool ok = true;
-            while (ok && next_work(cur, p, w)) {
-                const int buf = ci & 1;
-                ok = mbar_wait(bar(B_ACC_EMPTY + buf), (ci >> 1) & 1, ab);
-                if (!ok) break;
-                if (w.has_lr) {
-                    // the epilogue of the previous item with a low-rank term has read its accumulator
-                    ok = mbar_wait(bar(B_DLR_EMPTY), (clr_items & 1) ^ 1, ab);
-                    for (int c = 0; c < lr_chunks && ok; ++c) {
-                        const int s = cl % C::NL;
-                        ok = mbar_wait(bar(B_CONV_LR + s), (cl / C::NL) & 1, ab);
-                        if (!ok) break;
-                        tc_fence_after();
-                        const uint64_t adesc = smem_desc_sw128(sbase + C::OffLb + s * C::LbBytes);
-                        const uint64_t bdesc = smem_desc_sw128(sbase + C::OffT + s * C::TBytes);
-                        int steps = (p.r - c * 64) / 16;
-                        if (steps > 4) steps = 4;
-                        for (int kk = 0; kk < steps; ++kk)
-                            mma_f16_ss(tm_dlr, adesc + 2 * kk, bdesc + 2 * kk, idesc_f16, (c != 0 || kk != 0) ? 1u : 0u);
-                        tc_commit(bar(B_EMPTY_LR + s));
-                        ++cl;
-                    }
-                    ++clr_items;
-                    if (ok) tc_commit(bar(B_ACC_FULL + buf));
-                } else {
-                    mbar_arrive(bar(B_ACC_FULL + buf));
-                }
-                ++ci;
             }
         }
     } else if (warp == 1 || warp == C::WarpIssuer1) {
@@ -535,7 +551,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 if (!ok) break;
                 tc_fence_after();
                 const int nst = (w.kb1 - w.kb0 + KS - 1) / KS;
-                const bool mid = !C::LrLane && MID && issuer == 0 && lr_mid_tile(C::NL, w.has_lr, lr_chunks, nst);
+                const bool mid = !C::ProducerLr && MID && issuer == 0 && lr_mid_tile(C::NL, w.has_lr, lr_chunks, nst);
                 int lc = 0;                // low-rank chunks of this item multiplied so far
                 // one chunk: wait for its conversion, multiply, hand the slot back
                 auto lr_chunk = [&](int c) {
@@ -592,7 +608,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     tc_commit(bar(B_X_FREE + sx));
                     ++ca;
                 }
-                if (!C::LrLane && ok && w.has_lr && issuer == 0) {
+                if (!C::ProducerLr && ok && w.has_lr && issuer == 0) {
                     if (lc == 0) ok = mbar_wait(bar(B_DLR_EMPTY), (clr_items & 1) ^ 1, ab);
                     for (int c = lc; c < lr_chunks && ok; ++c) ok = lr_chunk(c);
                     ++clr_items;
@@ -646,10 +662,21 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             for (int kb = w.kb0; kb < w.kb1 && ok; kb += KS, ++st_idx) {
                 const int nkb = (w.kb1 - kb < KS) ? (w.kb1 - kb) : KS;
                 const int sw = cw % C::NW;   // cw counts stages
-                if (mid && lc < lr_chunks - 1 && st_idx == lr_mma_stage(lc, lr_chunks, nst) - 2) {
-                    ok = convert_chunk();
-                    if (!ok) break;
-                    ++lc;
+                if (mid && lc < lr_chunks - 1 && st_idx >= lr_mma_stage(lc, lr_chunks, nst) - 2) {
+                    // Never WAIT for a chunk in mid-tile: it is loaded only after the chunk before
+                    // it has been multiplied, by the thread that also feeds the activation ring,
+                    // and that thread gets back to the chunks only while the stages keep flowing
+                    // (the first chunk of an item also needs the previous epilogue to have read
+                    // the accumulator).  A chunk that has not landed is looked at again at the
+                    // next stage; what is left at the end of the item is waited for there, when
+                    // every activation stage of the item has been issued.
+                    bool landed = true;
+                    if (leader) landed = mbar_try_wait(bar(B_FULL_LR + cl % C::NL), (cl / C::NL) & 1);
+                    if (group_bar_all(group, landed)) {
+                        ok = convert_chunk();
+                        if (!ok) break;
+                        ++lc;
+                    }
                 }
                 if ((int)(cw & 1u) != group) { ++cw; continue; }
                 ok = group_mbar_wait(bar(B_W_FULL + sw), (cw / C::NW) & 1, ab, leader, group);
@@ -708,7 +735,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         Cursor cur;
         cur.init(u_begin, u_end, p);
         Work w;
-        uint32_t ci = 0;
+        uint32_t ci = 0, lr_seen = 0;
         int partial_idx = 0;                       // 0: first partial item of this CTA, 1: second
         bool ok = true;
         // both integer accumulators start at zero: every integer MMA accumulates
@@ -721,6 +748,10 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         while (ok && next_work(cur, p, w)) {
             const int buf = ci & 1;
             ok = warp_mbar_wait(bar(B_ACC_FULL + buf), (ci >> 1) & 1, ab, lane);
+            if (C::ProducerLr && w.has_lr) {            // ... and the item's low-rank MMAs (the producer commits them)
+                if (ok) ok = warp_mbar_wait(bar(B_LR_DONE), lr_seen & 1, ab, lane);
+                ++lr_seen;
+            }
             ok = named_bar_all(1, C::EpiThreads, ok);   // the 128 epilogue threads go on or give up together
             if (!ok) break;
             tc_fence_after();

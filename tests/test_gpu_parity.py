@@ -364,7 +364,7 @@ def test_config4_block_linears_full_size_all_rows(aser, name):
 C5_POINTS = [  # M, N, r, all rows?
     (1, 8192, 64, True), (16, 8192, 32, True), (16, 28672, 64, True), (128, 8192, 0, True),
     (128, 28672, 256, True), (1024, 8192, 128, True), (1024, 28672, 32, False),
-    (4096, 8192, 128, True), (4096, 8192, 0, False), (4096, 28672, 64, True),
+    (4096, 8192, 128, True), (4096, 8192, 0, False), (4096, 28672, 64, True), (4096, 8192, 256, False),
 ]
 
 
@@ -384,6 +384,32 @@ def test_config5_sweep_points(aser, M, N, r, full):
         rows = np.unique(np.concatenate([base, base + 127, base + 61]).clip(0, M - 1))
     run_path(aser, lay, s, Wq, w_scale, L_A, L_B, "tc", rows=rows, use_dgemm=True,
              timed_config=(M == 4096))
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("M,N,K,r", [(4096, 8192, 8192, 256), (4096, 4096, 4096, 128), (2048, 1024, 14336, 192)])
+def test_many_chunks_on_long_tiles_repeated_launches(aser, M, N, K, r):
+    """Several low-rank chunks per 128-token tile on tiles long enough for the mid-tile schedule,
+    several tiles per CTA, launched back to back: no bounded wait may give up (a chunk that is
+    late must never make a role wait for something only a stalled role can provide) and every
+    launch must give the same bits."""
+    lay = synth.make_layer(M, N, K, seed=900 + r, n_cal=8)
+    s = synth.standin_smoothing_vector(K, lay.outlier_idx, 16.0)
+    L_A, L_B = synth.standin_factors(N, K, r, seed=3, scale_a=0.01, scale_b=0.01)
+    L = aser.AserLinear(to_dev(lay.W), to_dev(s), to_dev(L_A), to_dev(L_B), M)
+    X = to_dev(lay.X)
+    first = L(X).clone()
+    aser.check_status(L.ws)
+    for rep in range(30):
+        L.linear(M, True)
+    torch.cuda.synchronize()
+    aser.check_status(L.ws)
+    assert torch.equal(L.Y[:M], first)
+    for rep in range(10):
+        Y = L(X)
+    torch.cuda.synchronize()
+    aser.check_status(L.ws)
+    assert torch.equal(Y, first)
 
 
 @pytest.mark.gpu

@@ -75,13 +75,14 @@ struct Cfg {
     // inside barrier and tensor-core instructions (a wait, MMA or commit costs its thread a few
     // hundred cycles under copy traffic), so every operation of a low-rank chunk on one of them
     // sets it back against the other and the whole pipeline with it.  A warp of its own for the
-    // job costs every thread 16 registers (21 warps: six on one scheduler).  A second lane of the
-    // producer's warp as a third issuer measured the same as what is done here, but depends on how
-    // the hardware shares a warp between two diverged spinning lanes: at rank 256 the lane was
-    // starved while lane 0 waited for it, and a bounded wait gave up.  So, with the one-slot
-    // chunk ring, the thread that loads the chunks also multiplies them: it runs a few stages
-    // ahead of the MMAs, has slack, polls the chunk's barriers between its activation stages, and
-    // waits for them only where nothing it still has to do is needed for them to complete.
+    // job costs every thread 16 registers (21 warps: six on one scheduler); a second lane of the
+    // producer's warp as a third issuer measured the same as what is done here and leans on how the
+    // hardware shares a warp between two diverged spinning lanes.  So, with the one-slot chunk
+    // ring, the thread that loads the chunks also multiplies them: it runs a few stages ahead of
+    // the MMAs, has slack, polls the chunk's barriers between its activation stages, and waits for
+    // them only where nothing it still has to do is needed for them to complete (after the last
+    // activation stage of the item).  For the same reason no other role waits for a chunk in
+    // mid-tile: see the unpack warps.
     static constexpr bool ProducerLr = (NL == 1);
     static constexpr int SmemBytes = OffBar + NumBars * 8 + 128 + 1024;  // + slack for 1 KiB alignment
     static constexpr int ASlotCols = KA * 32;

@@ -79,9 +79,9 @@ EXTRA_POINTS = ("c2_decode_m8", "c2_decode_m1", "c3_prefill_gate_up", "c3_prefil
 # linear_tc launches; "<workload>/<layers>" is the launch of that layer or fused group.  Workloads
 # without a capture of the current kernel report null.
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    "c4_decoder_block": 1040.6e6 / 5,
-    "c4_decoder_block/q+k+v": 36.4e6, "c4_decoder_block/o": 27.5e6, "c4_decoder_block/gate": 167.3e6,
-    "c4_decoder_block/up": 168.9e6, "c4_decoder_block/down": 640.4e6,
+    "c4_decoder_block": 1056.9e6 / 5,
+    "c4_decoder_block/q+k+v": 36.8e6, "c4_decoder_block/o": 27.6e6, "c4_decoder_block/gate": 166.7e6,
+    "c4_decoder_block/up": 189.1e6, "c4_decoder_block/down": 636.9e6,
 }
 
 

@@ -493,7 +493,13 @@ act_quant_kernel(const __half* __restrict__ X, const float* __restrict__ s, int 
         const float* tp = t_part + ((size_t)(j >> 7) * Mc + row0 + rr) * 128 + (j & 127);
         const size_t slice = (size_t)groups * Mc * 128;
         float t = 0.f;
-        for (int ks = 0; ks < KS; ++ks) t += tp[ks * slice];
+        int ks = 0;
+        for (; ks + 4 <= KS; ks += 4) {         // four loads in flight, summed in slice order
+            const float a0 = tp[ks * slice], a1 = tp[(ks + 1) * slice];
+            const float a2 = tp[(ks + 2) * slice], a3 = tp[(ks + 3) * slice];
+            t += a0; t += a1; t += a2; t += a3;
+        }
+        for (; ks < KS; ++ks) t += tp[ks * slice];
         store_t(T + (size_t)(m_first + row0 + rr) * ldt, j, t, lo_off);
     }
     __syncthreads();
